@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the RTPrune pruning path on B200.
+
+A step is one pass of the whole path (norms + statistics -> ratio -> top-M -> cosine scores ->
+Sinkhorn -> merge + pack) over one synthetic DeepSeek-OCR-Large-shaped batch: 64 images x 400 tokens
+x 1280 bf16, dynamic ratio with mean retention ~0.84.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1 is launched by torch.distributed.run (one rank per GPU); images are independent, so every rank
+prunes its own batch and there is no data-path collective (weak scaling).
+--impl reference times the fp64 CPU oracle on the host cores instead (a deliberately slow program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+WORKLOAD = "large"
+WORKLOAD_DESC = "large: 64 images x 400 tokens x 1280 bf16, dynamic ratio (mean retention 0.84), T=100"
+ROTATE = 4                 # input/output buffer sets cycled so that no step finds its input in L2
+FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
+REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
+NCU_TRAFFIC_BYTES = {}
+
+
+def cpu_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return float(pk["hbm_gbs"]), float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any(r[2 + k] == "Active" for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": reasons,
+                "samples": len(self.rows)}
+
+
+def time_oracle(w, images, threads):
+    from oracle import oracle
+    p = w.params
+    op = oracle.Params(dynamic=bool(p["dynamic"]), r_fixed=p["r_fixed"], phi_lo=p["phi_lo"],
+                       phi_hi=p["phi_hi"], r_max=p["r_max"], z=p["z"], alpha=p["alpha"],
+                       eps=p["eps"], iters=int(p["iters"]))
+    X = w.X_f64()
+    t0 = time.perf_counter()
+    oracle.run_batch(X, w.offsets, op, w.rho, images=images, threads=threads)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, rank: int) -> None:
+    """The oracle as it stands, on the host cores: rank 0 only."""
+    if rank != 0:
+        return
+    from paper_2605_00392_b200 import synth
+    threads = cpu_threads()
+    w = synth.make(WORKLOAD, batch=REFERENCE_SAMPLE)
+    images = list(range(REFERENCE_SAMPLE))
+    for _ in range(args.warmup):
+        time_oracle(w, images, threads)
+    t = 0.0
+    for _ in range(args.steps):
+        t += time_oracle(w, images, threads)
+    ms = 1e3 * t / max(args.steps, 1)
+    value = REFERENCE_SAMPLE / (ms / 1e3)
+    sample = "first %d images of the Large batch per step, all host cores" % REFERENCE_SAMPLE
+    line = {"impl": "reference", "metric": "pruned images/sec", "value": value, "unit": "images/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "tokens_per_s": value * 400,
+            "config": {"workload": WORKLOAD_DESC, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "images/s", "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruning path has no CPU fallback")
+    import torch.distributed as dist
+    from paper_2605_00392_b200 import binding, synth
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- workload: every rank prunes its own Large batch (independent images, no exchange) --------
+    sets = []
+    w0 = None
+    for s in range(ROTATE):
+        w = synth.make(WORKLOAD, seed_offset=rank * ROTATE + s)
+        if w0 is None:
+            w0 = w
+        sets.append(w)
+    batch, total, d = w0.batch, w0.total_tokens, w0.d
+    plan = binding.Plan(d, torch.bfloat16, batch, total, w0.max_tokens, device=dev)
+    fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
+    dev_sets = []
+    for w in sets:
+        rho = torch.from_numpy(w.rho).to(dev)
+        dev_sets.append(dict(X=w.X.to(dev), offs=torch.from_numpy(w.offsets).to(dev), rho=rho,
+                             params=binding.make_params(rho, **fields),
+                             out=binding.Outputs.allocate(total, batch, d, torch.bfloat16, dev)))
+    stream = torch.cuda.current_stream()
+
+    def step(i: int) -> None:
+        s = dev_sets[i % ROTATE]
+        plan.run(s["X"], s["offs"], s["params"], s["out"])
+
+    def barrier() -> None:
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert plan.query_status() == 0
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    # ---- timed region: K steps back to back, CUDA events on the launching stream ------------------
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = plan.last_launch_count * args.steps
+
+    # ---- same steps again with per-kernel events (feeds the roofline of the dominant kernel) -----
+    plan.profile_enable(True)
+    per_kernel = {}
+    nprof = min(args.steps, 50)
+    for i in range(nprof):
+        step(i)
+        for name, ms in plan.profile_read():
+            per_kernel.setdefault(name, []).append(ms)
+    plan.profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host-buffer entry point ------------------------------------------
+    host_out = binding.Outputs.allocate(total, batch, d, torch.bfloat16, "cpu", pin=True)
+    hX = [w.X.pin_memory() for w in sets]
+    hoffs = [torch.from_numpy(w.offsets).pin_memory() for w in sets]
+    hrho = [torch.from_numpy(w.rho).pin_memory() for w in sets]
+    hparams = binding.make_params(None, **fields)
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        plan.run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_out)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    for i in range(e2e_steps):
+        plan.run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_out)
+    e3.record(stream)
+    barrier()
+    ms_e2e = e2.elapsed_time(e3) / e2e_steps
+    kept_total = int(host_out.out_offsets[batch])
+    esz = 2
+    h2d = total * d * esz + (batch + 1) * 4 + batch * 4
+    d2h = total * d * esz + (batch + 1) * 4 + batch * 4 + 4 * total * 4 + batch * 8 * 4
+
+    # ---- max over ranks ---------------------------------------------------------------------------
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    images_s = world * batch / (ms_step / 1e3)
+    e2e_images_s = world * batch / (ms_e2e / 1e3)
+
+    if rank == 0:
+        hbm_peak, tensor_peak, peak_kind = measured_peaks()
+        stats = dev_sets[0]["out"].stats.cpu().numpy()[:batch]
+        M = stats[:, 3].astype(np.int64)
+        B = stats[:, 4].astype(np.int64)
+        iters_run = stats[:, 5]
+        sumM, sumMB = int(M.sum()), int((M * B).sum())
+        avg = {k: float(np.mean(v)) for k, v in per_kernel.items()}
+        dominant = max(avg, key=avg.get)
+        x_bytes = total * d * esz
+        y_bytes = sumM * d * esz
+        algo = {   # algorithmic bytes / flops per launch, by kernel
+            "norm_stats": ("hbm", x_bytes + total * 4),
+            "select": ("hbm", total * 4 * 2 + batch * 48),
+            "scores": ("alu", 2.0 * sumMB * d),
+            "sinkhorn": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
+            "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
+        }
+        bound, units = algo[dominant]
+        dur_s = avg[dominant] / 1e3
+        if bound == "hbm":
+            achieved, peak, unit = units / dur_s / 1e9, hbm_peak, "GB/s"
+        else:
+            achieved, peak, unit = units / dur_s / 1e12, FP32_FMA_PEAK_TFLOPS, "TFLOP/s"
+        path_bytes = x_bytes + y_bytes + 12 * total
+        line = {
+            "metric": "pruned images/sec", "value": images_s, "unit": "images/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "tokens_per_s": images_s * total / batch,
+            "config": {"workload": WORKLOAD_DESC, "global_batch": world * batch,
+                       "accumulate": "fp32", "sinkhorn": "T=100 with exit at the bitwise fixed point",
+                       "mean_iterations_run": float(iters_run.mean()),
+                       "mean_retention": float(sumM) / total,
+                       "l2": "inputs and outputs rotate over %d buffer sets (%.0f MB > L2)"
+                             % (ROTATE, ROTATE * (x_bytes + y_bytes) / 1e6),
+                       "parallelism": "dp%d (independent images, no collective)" % world},
+            "roofline": {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak,
+                         "unit": unit, "frac": achieved / peak, "peak_source": peak_kind,
+                         "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                         "avg_launch_ms": avg[dominant]},
+            "path_roofline": {"bound": "hbm", "algorithmic_bytes": path_bytes,
+                              "achieved": path_bytes / (ms_step / 1e3) / 1e9, "peak": hbm_peak,
+                              "unit": "GB/s", "frac": path_bytes / (ms_step / 1e3) / 1e9 / hbm_peak,
+                              "peak_source": peak_kind},
+            "kernel_ms": avg,
+            "e2e": {"value": e2e_images_s, "unit": "images/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "kept_rows": kept_total},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            threads = cpu_threads()
+            sec = time_oracle(w0, list(range(batch)), threads)
+            line["cpu_baseline"] = {"value": batch / sec, "unit": "images/s", "cores": threads,
+                                    "kind": "oracle",
+                                    "sample": "all %d images of the Large batch, once" % batch}
+        print(json.dumps(line), flush=True)
+    plan.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

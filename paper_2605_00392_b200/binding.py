@@ -1,0 +1,264 @@
+"""Thin ctypes binding of librtprune.so: argument marshalling only.
+
+The names mirror include/rtprune.h.  torch is used for device memory and streams; every step of the
+pruning path runs in the library's CUDA kernels.  There is no CPU fallback: if the library cannot be
+loaded, or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+STATS_STRIDE = 8
+BF16, FP32 = 0, 1
+SINKHORN_AUTO, SINKHORN_LOG, SINKHORN_SCALING = 0, 1, 2
+DEV_NONFINITE, DEV_TIMEOUT, DEV_BAD_OFFSETS = 1, 2, 4
+
+STATUS_NAMES = {0: "RTPRUNE_OK", 1: "RTPRUNE_ERR_INVALID_ARG", 2: "RTPRUNE_ERR_UNSUPPORTED",
+                3: "RTPRUNE_ERR_WORKSPACE", 4: "RTPRUNE_ERR_CUDA", 5: "RTPRUNE_ERR_NONFINITE",
+                6: "RTPRUNE_ERR_TIMEOUT", 7: "RTPRUNE_ERR_BAD_OFFSETS"}
+
+
+class RtpruneError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s returned %s" % (where, STATUS_NAMES.get(status, status)))
+
+
+class CParams(ctypes.Structure):
+    """rtprune_params_t."""
+    _fields_ = [("dynamic", ctypes.c_int32), ("r_fixed", ctypes.c_float),
+                ("rho", ctypes.c_void_p), ("phi_lo", ctypes.c_float), ("phi_hi", ctypes.c_float),
+                ("r_max", ctypes.c_float), ("z", ctypes.c_float), ("alpha", ctypes.c_float),
+                ("eps", ctypes.c_float), ("iters", ctypes.c_int32), ("form", ctypes.c_int32),
+                ("stop_at_fixed_point", ctypes.c_int32), ("tol", ctypes.c_float)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads (building first if the sources are newer) the C-ABI library.  Raises on failure."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if _build.stale():
+        path = _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError("librtprune.so is missing and could not be built")
+    L = ctypes.CDLL(path)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    pp = ctypes.POINTER(CParams)
+    L.rtprune_default_params.argtypes = [pp]
+    L.rtprune_plan.argtypes = [ctypes.POINTER(vp), i32, ctypes.c_int, i32, i64, i32,
+                               ctypes.POINTER(sz)]
+    L.rtprune_run.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.rtprune_workspace_init.argtypes = [vp, vp, vp, sz]
+    L.rtprune_select.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, sz, vp, vp, vp, vp, vp]
+    L.rtprune_run_host.argtypes = [vp, vp, vp, vp, vp, i32, i64, pp, vp, sz,
+                                   vp, vp, vp, vp, vp, vp, vp, vp]
+    L.rtprune_host_arena_bytes.argtypes = [vp, ctypes.POINTER(sz)]
+    L.rtprune_query_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.rtprune_profile_enable.argtypes = [vp, i32]
+    L.rtprune_profile_read.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float),
+                                       ctypes.POINTER(ctypes.c_char_p)]
+    L.rtprune_last_launch_count.argtypes = [vp]
+    L.rtprune_last_cuda_error.argtypes = [vp]
+    L.rtprune_destroy.argtypes = [vp]
+    L.rtprune_destroy.restype = None
+    L.rtprune_status_string.argtypes = [ctypes.c_int]
+    L.rtprune_status_string.restype = ctypes.c_char_p
+    L.rtprune_version.restype = i32
+    _lib = L
+    return L
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise RtpruneError(status, where)
+
+
+def default_params() -> CParams:
+    p = CParams()
+    _check(lib().rtprune_default_params(ctypes.byref(p)), "rtprune_default_params")
+    return p
+
+
+def make_params(rho: Optional[torch.Tensor] = None, **kw) -> CParams:
+    """Paper defaults overridden by keyword (field names of rtprune_params_t)."""
+    p = default_params()
+    for k, v in kw.items():
+        if not hasattr(p, k) or k == "rho":
+            raise KeyError(k)
+        setattr(p, k, v)
+    p.rho = rho.data_ptr() if rho is not None else None
+    return p
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream_handle(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+@dataclass
+class Outputs:
+    """Device (or pinned host) tensors the library fills; see rtprune_run in rtprune.h."""
+    Y: torch.Tensor
+    out_offsets: torch.Tensor
+    counts: torch.Tensor
+    kept_idx: torch.Tensor
+    merged_idx: torch.Tensor
+    merge_partner: torch.Tensor
+    merge_weight: torch.Tensor
+    stats: torch.Tensor
+
+    @staticmethod
+    def allocate(total_tokens: int, batch: int, d: int, dtype: torch.dtype, device,
+                 pin: bool = False) -> "Outputs":
+        kw = dict(device=device, pin_memory=pin) if pin else dict(device=device)
+        n = max(total_tokens, 1)
+        return Outputs(
+            Y=torch.empty((n, d), dtype=dtype, **kw),
+            out_offsets=torch.zeros(batch + 1, dtype=torch.int32, **kw),
+            counts=torch.zeros(max(batch, 1), dtype=torch.int32, **kw),
+            kept_idx=torch.full((n,), -1, dtype=torch.int32, **kw),
+            merged_idx=torch.full((n,), -1, dtype=torch.int32, **kw),
+            merge_partner=torch.full((n,), -1, dtype=torch.int32, **kw),
+            merge_weight=torch.zeros(n, dtype=torch.float32, **kw),
+            stats=torch.zeros((max(batch, 1), STATS_STRIDE), dtype=torch.float32, **kw))
+
+
+class Plan:
+    """rtprune_plan_t plus a torch-allocated workspace on the current device."""
+
+    def __init__(self, d: int, dtype: torch.dtype, max_batch: int, max_total_tokens: int,
+                 max_tokens_per_image: int, device: Optional[torch.device] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("rtprune needs a CUDA device; there is no CPU path")
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+        self.d, self.dtype = d, dtype
+        self.max_batch, self.max_total, self.max_tokens = max_batch, max_total_tokens, max_tokens_per_image
+        code = {torch.bfloat16: BF16, torch.float32: FP32}[dtype]
+        h = ctypes.c_void_p()
+        ws = ctypes.c_size_t()
+        with torch.cuda.device(self.device):
+            _check(lib().rtprune_plan(ctypes.byref(h), d, code, max_batch, max_total_tokens,
+                                      max_tokens_per_image, ctypes.byref(ws)), "rtprune_plan")
+            self.handle = h
+            self.workspace_bytes = ws.value
+            self.workspace = torch.empty(ws.value, dtype=torch.uint8, device=self.device)
+            assert self.workspace.data_ptr() % 256 == 0
+            self.workspace_init()
+        self._arena = None
+
+    # -- rtprune_workspace_init
+    def workspace_init(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(lib().rtprune_workspace_init(self.handle, _stream_handle(stream),
+                                            self.workspace.data_ptr(), self.workspace_bytes),
+               "rtprune_workspace_init")
+
+    # -- rtprune_run
+    def run(self, X: torch.Tensor, offsets: torch.Tensor, params: CParams, out: Outputs,
+            stream: Optional[torch.cuda.Stream] = None) -> None:
+        batch = offsets.numel() - 1
+        _check(lib().rtprune_run(self.handle, _stream_handle(stream), X.data_ptr(),
+                                 offsets.data_ptr(), batch, X.shape[0], ctypes.byref(params),
+                                 self.workspace.data_ptr(), self.workspace_bytes, out.Y.data_ptr(),
+                                 out.out_offsets.data_ptr(), out.counts.data_ptr(),
+                                 out.kept_idx.data_ptr(), out.merged_idx.data_ptr(),
+                                 out.merge_partner.data_ptr(), out.merge_weight.data_ptr(),
+                                 out.stats.data_ptr()), "rtprune_run")
+
+    # -- rtprune_select
+    def select(self, X: torch.Tensor, offsets: torch.Tensor, params: CParams, out: Outputs,
+               norms_out: Optional[torch.Tensor] = None, order_out: Optional[torch.Tensor] = None,
+               stream: Optional[torch.cuda.Stream] = None) -> None:
+        batch = offsets.numel() - 1
+        _check(lib().rtprune_select(self.handle, _stream_handle(stream), X.data_ptr(),
+                                    offsets.data_ptr(), batch, X.shape[0], ctypes.byref(params),
+                                    self.workspace.data_ptr(), self.workspace_bytes,
+                                    out.out_offsets.data_ptr(), out.counts.data_ptr(),
+                                    out.stats.data_ptr(), _ptr(norms_out), _ptr(order_out)),
+               "rtprune_select")
+
+    # -- rtprune_host_arena_bytes / rtprune_run_host
+    def host_arena_bytes(self) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().rtprune_host_arena_bytes(self.handle, ctypes.byref(n)), "rtprune_host_arena_bytes")
+        return n.value
+
+    def run_host(self, X: torch.Tensor, offsets: torch.Tensor, rho: Optional[torch.Tensor],
+                 params: CParams, out: Outputs, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Host tensors in (pinned for speed), host tensors out; asynchronous on the stream."""
+        if self._arena is None:
+            self._arena = torch.empty(self.host_arena_bytes(), dtype=torch.uint8, device=self.device)
+        for t in (X, offsets, out.Y, out.out_offsets):
+            assert t.device.type == "cpu"
+        batch = offsets.numel() - 1
+        _check(lib().rtprune_run_host(self.handle, _stream_handle(stream), X.data_ptr(),
+                                      offsets.data_ptr(), _ptr(rho), batch, X.shape[0],
+                                      ctypes.byref(params), self._arena.data_ptr(),
+                                      self._arena.numel(), out.Y.data_ptr(),
+                                      out.out_offsets.data_ptr(), out.counts.data_ptr(),
+                                      out.kept_idx.data_ptr(), out.merged_idx.data_ptr(),
+                                      out.merge_partner.data_ptr(), out.merge_weight.data_ptr(),
+                                      out.stats.data_ptr()), "rtprune_run_host")
+
+    # -- rtprune_query_status
+    def query_status(self, stream: Optional[torch.cuda.Stream] = None, workspace=None) -> int:
+        """Synchronises, returns the raw device status bits (0 = clean) and clears them."""
+        flags = ctypes.c_uint32()
+        ws = self.workspace.data_ptr() if workspace is None else workspace
+        lib().rtprune_query_status(self.handle, _stream_handle(stream), ws, ctypes.byref(flags))
+        return flags.value
+
+    # -- rtprune_profile_enable / rtprune_profile_read
+    def profile_enable(self, enable: bool = True) -> None:
+        _check(lib().rtprune_profile_enable(self.handle, int(enable)), "rtprune_profile_enable")
+
+    def profile_read(self):
+        """[(kernel name, milliseconds)] of the most recent run (waits for it)."""
+        n = ctypes.c_int32()
+        ms = (ctypes.c_float * 8)()
+        names = (ctypes.c_char_p * 8)()
+        _check(lib().rtprune_profile_read(self.handle, ctypes.byref(n), ms, names),
+               "rtprune_profile_read")
+        return [(names[i].decode(), float(ms[i])) for i in range(n.value)]
+
+    @property
+    def last_launch_count(self) -> int:
+        return lib().rtprune_last_launch_count(self.handle)
+
+    @property
+    def last_cuda_error(self) -> int:
+        return lib().rtprune_last_cuda_error(self.handle)
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            lib().rtprune_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def shard_images(batch: int, world_size: int, rank: int):
+    """Contiguous range of images [lo, hi) owned by `rank`: images are independent, so a multi-GPU
+    run is this split with no exchange."""
+    base, extra = divmod(batch, world_size)
+    lo = rank * base + min(rank, extra)
+    return lo, lo + base + (1 if rank < extra else 0)

@@ -1,0 +1,605 @@
+// C ABI of the RTPrune pruning path: plan, argument checks, workspace layout and kernel launches.
+// Every step of the path runs in the kernels included below; this file only marshals.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "sinkhorn.cuh"
+#include "stage1.cuh"
+
+using namespace rtp;
+
+static_assert(sizeof(rtprune_params_t) == 56, "rtprune_params_t layout is part of the ABI");
+
+struct rtprune_plan_s {
+    int d;
+    rtprune_dtype_t dtype;
+    int max_batch;
+    int64_t max_total;
+    int max_tokens;
+    WsLayout ws;
+    int device;
+    int sm_count;
+    int smem_optin;       // bytes of opt-in shared memory per CTA
+    int sink_smem_bytes;  // dynamic shared memory of the Sinkhorn kernel
+    int last_launches;
+    int last_cuda_error;
+    bool profiling;
+    cudaEvent_t ev[RTPRUNE_PROFILE_MAX + 1];
+    const char *ev_name[RTPRUNE_PROFILE_MAX];
+    int ev_count;  // kernels recorded by the most recent run
+};
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WsLayout make_layout(int d, int max_batch, int64_t max_total, int max_tokens)
+{
+    WsLayout L;
+    L.chunks = (max_tokens + kChunkTokens - 1) / kChunkTokens;
+    L.kmat_stride = (max_tokens + 2 + 3) / 4;
+    size_t off = 0;
+    L.header = off;
+    off = align_up(off + sizeof(WsHeader), 256);
+    L.norms = off;
+    off = align_up(off + sizeof(float) * (size_t)max_total, 256);
+    L.spart = off;
+    off = align_up(off + sizeof(float) * (size_t)max_batch * L.chunks * d, 256);
+    L.order = off;
+    off = align_up(off + sizeof(int32_t) * (size_t)max_total, 256);
+    L.kmat = off;
+    off = align_up(off + sizeof(float) * (size_t)L.kmat_stride * (size_t)(max_total + 2 * (int64_t)max_batch), 256);
+    L.total = off;
+    return L;
+}
+
+struct Checked {
+    rtprune_plan_t *plan;
+    bool ok(cudaError_t e)
+    {
+        if (e == cudaSuccess) return true;
+        plan->last_cuda_error = (int)e;
+        return false;
+    }
+};
+
+// Profiling: event 0 before the first kernel, event k after the k-th.
+void prof_begin(rtprune_plan_t *plan, cudaStream_t st)
+{
+    plan->ev_count = 0;
+    if (plan->profiling) cudaEventRecord(plan->ev[0], st);
+}
+
+void launched(rtprune_plan_t *plan, cudaStream_t st, const char *name)
+{
+    ++plan->last_launches;
+    if (plan->profiling && plan->ev_count < RTPRUNE_PROFILE_MAX) {
+        plan->ev_name[plan->ev_count] = name;
+        cudaEventRecord(plan->ev[++plan->ev_count], st);
+    }
+}
+
+rtprune_status_t check_params(const rtprune_params_t *p)
+{
+    if (!p) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->dynamic != 0 && p->dynamic != 1) return RTPRUNE_ERR_INVALID_ARG;
+    if (!p->dynamic && !(p->r_fixed >= 0.f && p->r_fixed < 1.f)) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->dynamic) {
+        if (!(p->phi_hi > p->phi_lo)) return RTPRUNE_ERR_INVALID_ARG;
+        if (!(p->r_max > 0.f && p->r_max <= 1.f)) return RTPRUNE_ERR_INVALID_ARG;
+    }
+    if (!(p->eps > 0.f) || !std::isfinite(p->eps)) return RTPRUNE_ERR_INVALID_ARG;
+    if (!std::isfinite(p->z) || !std::isfinite(p->alpha)) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->iters < 0) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->form < RTPRUNE_SINKHORN_AUTO || p->form > RTPRUNE_SINKHORN_SCALING)
+        return RTPRUNE_ERR_INVALID_ARG;
+    if (!(p->tol >= 0.f)) return RTPRUNE_ERR_INVALID_ARG;
+    const bool scaling_safe = p->eps >= 0.25f && std::fabs(p->z) <= 4.f;
+    if (p->form == RTPRUNE_SINKHORN_SCALING && !scaling_safe) return RTPRUNE_ERR_INVALID_ARG;
+    return RTPRUNE_OK;
+}
+
+bool use_log_form(const rtprune_params_t *p)
+{
+    if (p->form == RTPRUNE_SINKHORN_LOG) return true;
+    if (p->form == RTPRUNE_SINKHORN_SCALING) return false;
+    return !(p->eps >= 0.25f && std::fabs(p->z) <= 4.f);
+}
+
+// Largest B any image of at most max_tokens tokens can get under these parameters.
+int max_pruned(const rtprune_params_t *p, int max_tokens)
+{
+    const float r = p->dynamic ? std::fmin(p->r_max, 1.f) : p->r_fixed;
+    long b = (long)std::floor((double)r * max_tokens + 0.5) + 1;  // +1: fp32 vs fp64 rounding slack
+    if (b > max_tokens - 1) b = max_tokens - 1;
+    if (b < 0) b = 0;
+    return (int)b;
+}
+
+template <typename T>
+cudaError_t launch_norm_stats(const rtprune_plan_t *pl, cudaStream_t st, const void *X,
+                              const int32_t *offsets, int batch, int total, float *norms,
+                              float *spart, WsHeader *hdr)
+{
+    constexpr int EPV = Elem<T>::kPerVec;
+    const int d = pl->d;
+    const int vpl = (d / EPV + 31) / 32;
+    dim3 grid(pl->ws.chunks, batch);
+    const size_t smem = sizeof(float) * 8 * (size_t)d;
+#define RTP_CASE(V)                                                                              \
+    case V: {                                                                                    \
+        auto k = norm_stats_kernel<T, V>;                                                        \
+        if (smem > 48 * 1024) {                                                                  \
+            cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                 (int)smem);                                     \
+            if (e != cudaSuccess) return e;                                                      \
+        }                                                                                        \
+        k<<<grid, 256, smem, st>>>((const T *)X, offsets, d, pl->ws.chunks, pl->max_tokens,      \
+                                   total, norms, spart, hdr);                                    \
+        break;                                                                                   \
+    }
+    switch (vpl) {
+        RTP_CASE(1) RTP_CASE(2) RTP_CASE(3) RTP_CASE(4) RTP_CASE(5) RTP_CASE(6) RTP_CASE(7)
+        RTP_CASE(8) RTP_CASE(9) RTP_CASE(10) RTP_CASE(11) RTP_CASE(12) RTP_CASE(13) RTP_CASE(14)
+        RTP_CASE(15) RTP_CASE(16)
+    default: return cudaErrorInvalidValue;
+    }
+#undef RTP_CASE
+    return cudaGetLastError();
+}
+
+struct DevOut {
+    void *Y;
+    int32_t *out_offsets, *counts, *kept_idx, *merged_idx, *merge_partner;
+    float *merge_weight, *stats;
+};
+
+rtprune_status_t check_common(rtprune_plan_t *plan, const void *X, const int32_t *offsets,
+                              int32_t batch, int64_t total, const rtprune_params_t *params,
+                              void *workspace, size_t workspace_bytes)
+{
+    if (!plan || !params) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch < 0 || total < 0) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch > plan->max_batch || total > plan->max_total) return RTPRUNE_ERR_INVALID_ARG;
+    if (total < batch) return RTPRUNE_ERR_INVALID_ARG;  // every image has at least one token
+    if (batch > 0 && (!X || !offsets)) return RTPRUNE_ERR_INVALID_ARG;
+    if (!workspace) return RTPRUNE_ERR_INVALID_ARG;
+    if (((uintptr_t)X & 15u) || ((uintptr_t)workspace & 255u)) return RTPRUNE_ERR_INVALID_ARG;
+    if (workspace_bytes < plan->ws.total) return RTPRUNE_ERR_WORKSPACE;
+    return check_params(params);
+}
+
+// Stage 1 launches (norms + statistics, selection).
+rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void *X,
+                               const int32_t *offsets, int32_t batch, int total,
+                               const rtprune_params_t *params, char *ws, int32_t *out_offsets,
+                               int32_t *counts, float *stats, float *norms_out,
+                               int32_t *order_out)
+{
+    Checked c{plan};
+    const WsLayout &L = plan->ws;
+    WsHeader *hdr = (WsHeader *)(ws + L.header);
+    float *norms = (float *)(ws + L.norms);
+    float *spart = (float *)(ws + L.spart);
+    int32_t *order = (int32_t *)(ws + L.order);
+    cudaError_t e = (plan->dtype == RTPRUNE_BF16)
+                        ? launch_norm_stats<__nv_bfloat16>(plan, st, X, offsets, batch, total, norms, spart, hdr)
+                        : launch_norm_stats<float>(plan, st, X, offsets, batch, total, norms, spart, hdr);
+    if (!c.ok(e)) return RTPRUNE_ERR_CUDA;
+    launched(plan, st, "norm_stats");
+    RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
+    const size_t smem = sizeof(float) * (size_t)plan->max_tokens;
+    select_kernel<<<batch, 1024, smem, st>>>(offsets, batch, plan->d, L.chunks, plan->max_tokens,
+                                             total, rp, params->rho, norms, spart, order, counts,
+                                             out_offsets, stats, norms_out, order_out, hdr);
+    if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+    launched(plan, st, "select");
+    return RTPRUNE_OK;
+}
+
+template <typename T>
+rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void *X,
+                               const int32_t *offsets, int32_t batch, int total,
+                               const rtprune_params_t *params, char *ws, const DevOut &o)
+{
+    Checked c{plan};
+    const WsLayout &L = plan->ws;
+    float *norms = (float *)(ws + L.norms);
+    int32_t *order = (int32_t *)(ws + L.order);
+    float *kmat = (float *)(ws + L.kmat);
+    const int maxN = plan->max_tokens;
+    const int maxB = max_pruned(params, maxN);
+    const int mtiles = (maxN + kSimtTile - 1) / kSimtTile;
+
+    if (maxB > 0) {
+        const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
+        dim3 grid(mtiles * btiles, batch);
+        scores_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, btiles,
+                                                   o.counts, order, norms, kmat, L.kmat_stride,
+                                                   maxN, total);
+        if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+        launched(plan, st, "scores");
+
+        OtParams op{params->z, params->alpha, params->eps, params->iters,
+                    params->stop_at_fixed_point, params->tol};
+        const int smem_floats = plan->sink_smem_bytes / (int)sizeof(float);
+        if (use_log_form(params))
+            sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
+                offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
+                smem_floats, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
+        else
+            sinkhorn_kernel<false><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
+                offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
+                smem_floats, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
+        if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+        launched(plan, st, "sinkhorn");
+    }
+
+    const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
+    dim3 grid(mtiles * dtiles, batch);
+    merge_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, dtiles, o.counts,
+                                              o.out_offsets, order, kmat, L.kmat_stride, maxN,
+                                              total, params->alpha, (T *)o.Y, o.kept_idx);
+    if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+    launched(plan, st, "merge");
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X,
+                            const int32_t *offsets, int32_t batch, int total,
+                            const rtprune_params_t *params, char *ws, const DevOut &o)
+{
+    if (batch == 0) {
+        Checked c{plan};
+        if (!c.ok(cudaMemsetAsync(o.out_offsets, 0, sizeof(int32_t), st))) return RTPRUNE_ERR_CUDA;
+        return RTPRUNE_OK;
+    }
+    prof_begin(plan, st);
+    rtprune_status_t s = launch_stage1(plan, st, X, offsets, batch, total, params, ws, o.out_offsets,
+                                       o.counts, o.stats, nullptr, nullptr);
+    if (s != RTPRUNE_OK) return s;
+    return (plan->dtype == RTPRUNE_BF16)
+               ? launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o)
+               : launch_stage2<float>(plan, st, X, offsets, batch, total, params, ws, o);
+}
+
+// Device arena of rtprune_run_host: device copies of the inputs and outputs, then the workspace.
+struct Arena {
+    size_t X, offsets, rho, Y, out_offsets, counts, kept_idx, merged_idx, partner, weight, stats,
+        ws, total;
+};
+
+Arena make_arena(const rtprune_plan_t *p)
+{
+    Arena a;
+    const size_t esz = p->dtype == RTPRUNE_BF16 ? 2 : 4;
+    const size_t tot = (size_t)p->max_total, nb = (size_t)p->max_batch;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    a.X = take(tot * p->d * esz);
+    a.offsets = take((nb + 1) * 4);
+    a.rho = take(nb * 4);
+    a.Y = take(tot * p->d * esz);
+    a.out_offsets = take((nb + 1) * 4);
+    a.counts = take(nb * 4);
+    a.kept_idx = take(tot * 4);
+    a.merged_idx = take(tot * 4);
+    a.partner = take(tot * 4);
+    a.weight = take(tot * 4);
+    a.stats = take(nb * kStats * 4);
+    a.ws = take(p->ws.total);
+    a.total = off;
+    return a;
+}
+
+}  // namespace
+
+extern "C" {
+
+rtprune_status_t rtprune_default_params(rtprune_params_t *p)
+{
+    if (!p) return RTPRUNE_ERR_INVALID_ARG;
+    std::memset(p, 0, sizeof(*p));
+    p->dynamic = 0;
+    p->r_fixed = 0.25f;
+    p->rho = nullptr;
+    p->phi_lo = 0.f;
+    p->phi_hi = 1.f;
+    p->r_max = 1.f;
+    p->z = 0.2f;
+    p->alpha = 0.1f;
+    p->eps = 1.f;
+    p->iters = 100;
+    p->form = RTPRUNE_SINKHORN_AUTO;
+    p->stop_at_fixed_point = 1;
+    p->tol = 0.f;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtype_t dtype,
+                              int32_t max_batch, int64_t max_total_tokens,
+                              int32_t max_tokens_per_image, size_t *workspace_bytes)
+{
+    if (!plan_out || !workspace_bytes) return RTPRUNE_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    if (dtype != RTPRUNE_BF16 && dtype != RTPRUNE_FP32) return RTPRUNE_ERR_INVALID_ARG;
+    if (d <= 0 || max_batch <= 0 || max_total_tokens <= 0 || max_tokens_per_image <= 0)
+        return RTPRUNE_ERR_INVALID_ARG;
+    if (max_total_tokens > 0x7fff0000LL) return RTPRUNE_ERR_UNSUPPORTED;  // int32 offsets
+    if (max_batch > 65535) return RTPRUNE_ERR_UNSUPPORTED;
+    const int epv = dtype == RTPRUNE_BF16 ? 8 : 4;
+    if (d % epv != 0 || d > 16 * 32 * epv) return RTPRUNE_ERR_UNSUPPORTED;
+    if (max_tokens_per_image > 8192) return RTPRUNE_ERR_UNSUPPORTED;
+    if (max_tokens_per_image > max_total_tokens) max_tokens_per_image = (int32_t)max_total_tokens;
+
+    rtprune_plan_t *p = new (std::nothrow) rtprune_plan_t();
+    if (!p) return RTPRUNE_ERR_INVALID_ARG;
+    p->d = d;
+    p->dtype = dtype;
+    p->max_batch = max_batch;
+    p->max_total = max_total_tokens;
+    p->max_tokens = max_tokens_per_image;
+    p->ws = make_layout(d, max_batch, max_total_tokens, max_tokens_per_image);
+    p->last_launches = 0;
+    p->last_cuda_error = 0;
+    p->profiling = false;
+    p->ev_count = 0;
+
+    Checked c{p};
+    int dev = 0, optin = 0, sms = 0;
+    if (!c.ok(cudaGetDevice(&dev)) ||
+        !c.ok(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) ||
+        !c.ok(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) {
+        delete p;
+        return RTPRUNE_ERR_CUDA;
+    }
+    p->device = dev;
+    p->smem_optin = optin;
+    p->sm_count = sms;
+
+    // Sinkhorn shared memory: enough for the largest matrix an image of max_tokens can produce
+    // ((N/2+1)^2 cells at r = 1/2), capped by what one CTA may have.
+    const long long half = max_tokens_per_image / 2 + 2;
+    long long want = (half * (half | 1) + max_tokens_per_image + 2 + 2 * kSinkThreads) * 4 + 64;
+    const long long cap = (long long)optin - 1024;
+    if (want > cap) want = cap;
+    p->sink_smem_bytes = (int)(want / 16 * 16);
+    if (!c.ok(cudaFuncSetAttribute(sinkhorn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   p->sink_smem_bytes)) ||
+        !c.ok(cudaFuncSetAttribute(sinkhorn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   p->sink_smem_bytes))) {
+        delete p;
+        return RTPRUNE_ERR_CUDA;
+    }
+    *workspace_bytes = p->ws.total;
+    *plan_out = p;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_workspace_init(rtprune_plan_t *plan, void *cuda_stream, void *workspace,
+                                        size_t workspace_bytes)
+{
+    if (!plan || !workspace || ((uintptr_t)workspace & 255u)) return RTPRUNE_ERR_INVALID_ARG;
+    if (workspace_bytes < plan->ws.total) return RTPRUNE_ERR_WORKSPACE;
+    Checked c{plan};
+    if (!c.ok(cudaMemsetAsync((char *)workspace + plan->ws.header, 0, sizeof(WsHeader),
+                              (cudaStream_t)cuda_stream)))
+        return RTPRUNE_ERR_CUDA;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_run(rtprune_plan_t *plan, void *cuda_stream, const void *X,
+                             const int32_t *offsets, int32_t batch, int64_t total_tokens,
+                             const rtprune_params_t *params, void *workspace,
+                             size_t workspace_bytes, void *Y, int32_t *out_offsets,
+                             int32_t *counts, int32_t *kept_idx, int32_t *merged_idx,
+                             int32_t *merge_partner, float *merge_weight, float *stats)
+{
+    rtprune_status_t s = check_common(plan, X, offsets, batch, total_tokens, params, workspace,
+                                      workspace_bytes);
+    if (s != RTPRUNE_OK) return s;
+    if (!out_offsets) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch > 0 && (!Y || !counts || !kept_idx || !merged_idx || !merge_partner ||
+                      !merge_weight || !stats))
+        return RTPRUNE_ERR_INVALID_ARG;
+    if ((uintptr_t)Y & 15u) return RTPRUNE_ERR_INVALID_ARG;
+    plan->last_launches = 0;
+    DevOut o{Y, out_offsets, counts, kept_idx, merged_idx, merge_partner, merge_weight, stats};
+    return run_device(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
+                      (char *)workspace, o);
+}
+
+rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const void *X,
+                                const int32_t *offsets, int32_t batch, int64_t total_tokens,
+                                const rtprune_params_t *params, void *workspace,
+                                size_t workspace_bytes, int32_t *out_offsets, int32_t *counts,
+                                float *stats, float *norms_out, int32_t *order_out)
+{
+    rtprune_status_t s = check_common(plan, X, offsets, batch, total_tokens, params, workspace,
+                                      workspace_bytes);
+    if (s != RTPRUNE_OK) return s;
+    if (!out_offsets || (batch > 0 && (!counts || !stats))) return RTPRUNE_ERR_INVALID_ARG;
+    plan->last_launches = 0;
+    if (batch == 0) {
+        Checked c{plan};
+        if (!c.ok(cudaMemsetAsync(out_offsets, 0, sizeof(int32_t), (cudaStream_t)cuda_stream)))
+            return RTPRUNE_ERR_CUDA;
+        return RTPRUNE_OK;
+    }
+    prof_begin(plan, (cudaStream_t)cuda_stream);
+    return launch_stage1(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
+                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out);
+}
+
+rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)
+{
+    if (!plan || !arena_bytes) return RTPRUNE_ERR_INVALID_ARG;
+    *arena_bytes = make_arena(plan).total;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_run_host(rtprune_plan_t *plan, void *cuda_stream, const void *X_host,
+                                  const int32_t *offsets_host, const float *rho_host,
+                                  int32_t batch, int64_t total_tokens,
+                                  const rtprune_params_t *params, void *arena, size_t arena_bytes,
+                                  void *Y_host, int32_t *out_offsets_host, int32_t *counts_host,
+                                  int32_t *kept_idx_host, int32_t *merged_idx_host,
+                                  int32_t *merge_partner_host, float *merge_weight_host,
+                                  float *stats_host)
+{
+    if (!plan || !params || !arena || ((uintptr_t)arena & 255u)) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch < 0 || total_tokens < 0 || batch > plan->max_batch ||
+        total_tokens > plan->max_total || total_tokens < batch)
+        return RTPRUNE_ERR_INVALID_ARG;
+    if (!out_offsets_host) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch > 0 && (!X_host || !offsets_host || !Y_host || !counts_host || !kept_idx_host ||
+                      !merged_idx_host || !merge_partner_host || !merge_weight_host || !stats_host))
+        return RTPRUNE_ERR_INVALID_ARG;
+    const Arena a = make_arena(plan);
+    if (arena_bytes < a.total) return RTPRUNE_ERR_WORKSPACE;
+    rtprune_status_t s = check_params(params);
+    if (s != RTPRUNE_OK) return s;
+    // the host can see the offsets here: check the contract before anything is launched
+    if (batch > 0) {
+        if (offsets_host[0] != 0 || offsets_host[batch] != total_tokens) return RTPRUNE_ERR_INVALID_ARG;
+        for (int i = 0; i < batch; ++i) {
+            const int64_t n = (int64_t)offsets_host[i + 1] - offsets_host[i];
+            if (n < 1 || n > plan->max_tokens) return RTPRUNE_ERR_INVALID_ARG;
+        }
+    }
+    plan->last_launches = 0;
+    Checked c{plan};
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *base = (char *)arena;
+    const size_t esz = plan->dtype == RTPRUNE_BF16 ? 2 : 4;
+    const size_t row = (size_t)plan->d * esz;
+    if (batch == 0) {
+        out_offsets_host[0] = 0;
+        return RTPRUNE_OK;
+    }
+    rtprune_params_t p = *params;
+    p.rho = rho_host ? (const float *)(base + a.rho) : nullptr;
+    if (!c.ok(cudaMemcpyAsync(base + a.X, X_host, (size_t)total_tokens * row, cudaMemcpyHostToDevice, st)) ||
+        !c.ok(cudaMemcpyAsync(base + a.offsets, offsets_host, ((size_t)batch + 1) * 4, cudaMemcpyHostToDevice, st)))
+        return RTPRUNE_ERR_CUDA;
+    if (rho_host && !c.ok(cudaMemcpyAsync(base + a.rho, rho_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st)))
+        return RTPRUNE_ERR_CUDA;
+    if (!c.ok(cudaMemsetAsync(base + a.ws + plan->ws.header, 0, sizeof(WsHeader), st)))
+        return RTPRUNE_ERR_CUDA;
+    DevOut o{base + a.Y,
+             (int32_t *)(base + a.out_offsets),
+             (int32_t *)(base + a.counts),
+             (int32_t *)(base + a.kept_idx),
+             (int32_t *)(base + a.merged_idx),
+             (int32_t *)(base + a.partner),
+             (float *)(base + a.weight),
+             (float *)(base + a.stats)};
+    s = run_device(plan, st, base + a.X, (const int32_t *)(base + a.offsets), batch,
+                   (int)total_tokens, &p,
+                   base + a.ws, o);
+    if (s != RTPRUNE_OK) return s;
+    const size_t tot4 = (size_t)total_tokens * 4;
+    if (!c.ok(cudaMemcpyAsync(out_offsets_host, o.out_offsets, ((size_t)batch + 1) * 4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(counts_host, o.counts, (size_t)batch * 4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(kept_idx_host, o.kept_idx, tot4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(merged_idx_host, o.merged_idx, tot4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(merge_partner_host, o.merge_partner, tot4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(merge_weight_host, o.merge_weight, tot4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(stats_host, o.stats, (size_t)batch * kStats * 4, cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemcpyAsync(Y_host, o.Y, (size_t)total_tokens * row, cudaMemcpyDeviceToHost, st)))
+        return RTPRUNE_ERR_CUDA;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_query_status(rtprune_plan_t *plan, void *cuda_stream, void *workspace,
+                                      uint32_t *flags_out)
+{
+    if (!plan || !workspace) return RTPRUNE_ERR_INVALID_ARG;
+    Checked c{plan};
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint32_t flags = 0;
+    WsHeader *hdr = (WsHeader *)((char *)workspace + plan->ws.header);
+    if (!c.ok(cudaMemcpyAsync(&flags, &hdr->status, sizeof(flags), cudaMemcpyDeviceToHost, st)) ||
+        !c.ok(cudaMemsetAsync(&hdr->status, 0, sizeof(uint32_t), st)) ||
+        !c.ok(cudaStreamSynchronize(st)))
+        return RTPRUNE_ERR_CUDA;
+    if (flags_out) *flags_out = flags;
+    if (flags & RTPRUNE_DEV_NONFINITE) return RTPRUNE_ERR_NONFINITE;
+    if (flags & RTPRUNE_DEV_BAD_OFFSETS) return RTPRUNE_ERR_BAD_OFFSETS;
+    if (flags & RTPRUNE_DEV_TIMEOUT) return RTPRUNE_ERR_TIMEOUT;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_profile_enable(rtprune_plan_t *plan, int32_t enable)
+{
+    if (!plan) return RTPRUNE_ERR_INVALID_ARG;
+    Checked c{plan};
+    if (enable && !plan->profiling) {
+        for (int i = 0; i <= RTPRUNE_PROFILE_MAX; ++i)
+            if (!c.ok(cudaEventCreate(&plan->ev[i]))) {
+                for (int k = 0; k < i; ++k) cudaEventDestroy(plan->ev[k]);
+                return RTPRUNE_ERR_CUDA;
+            }
+        plan->profiling = true;
+        plan->ev_count = 0;
+    } else if (!enable && plan->profiling) {
+        for (int i = 0; i <= RTPRUNE_PROFILE_MAX; ++i) cudaEventDestroy(plan->ev[i]);
+        plan->profiling = false;
+        plan->ev_count = 0;
+    }
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_profile_read(rtprune_plan_t *plan, int32_t *n, float *ms,
+                                      const char **names)
+{
+    if (!plan || !n || !ms || !names) return RTPRUNE_ERR_INVALID_ARG;
+    *n = 0;
+    if (!plan->profiling || plan->ev_count == 0) return RTPRUNE_OK;
+    Checked c{plan};
+    if (!c.ok(cudaEventSynchronize(plan->ev[plan->ev_count]))) return RTPRUNE_ERR_CUDA;
+    for (int i = 0; i < plan->ev_count; ++i) {
+        if (!c.ok(cudaEventElapsedTime(&ms[i], plan->ev[i], plan->ev[i + 1]))) return RTPRUNE_ERR_CUDA;
+        names[i] = plan->ev_name[i];
+    }
+    *n = plan->ev_count;
+    return RTPRUNE_OK;
+}
+
+int32_t rtprune_last_launch_count(const rtprune_plan_t *plan) { return plan ? plan->last_launches : 0; }
+
+int32_t rtprune_last_cuda_error(const rtprune_plan_t *plan) { return plan ? plan->last_cuda_error : 0; }
+
+void rtprune_destroy(rtprune_plan_t *plan)
+{
+    if (!plan) return;
+    if (plan->profiling) rtprune_profile_enable(plan, 0);
+    delete plan;
+}
+
+const char *rtprune_status_string(rtprune_status_t s)
+{
+    switch (s) {
+    case RTPRUNE_OK: return "RTPRUNE_OK";
+    case RTPRUNE_ERR_INVALID_ARG: return "RTPRUNE_ERR_INVALID_ARG";
+    case RTPRUNE_ERR_UNSUPPORTED: return "RTPRUNE_ERR_UNSUPPORTED";
+    case RTPRUNE_ERR_WORKSPACE: return "RTPRUNE_ERR_WORKSPACE";
+    case RTPRUNE_ERR_CUDA: return "RTPRUNE_ERR_CUDA";
+    case RTPRUNE_ERR_NONFINITE: return "RTPRUNE_ERR_NONFINITE";
+    case RTPRUNE_ERR_TIMEOUT: return "RTPRUNE_ERR_TIMEOUT";
+    case RTPRUNE_ERR_BAD_OFFSETS: return "RTPRUNE_ERR_BAD_OFFSETS";
+    }
+    return "RTPRUNE_ERR_UNKNOWN";
+}
+
+int32_t rtprune_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,246 @@
+// Dustbin-augmented optimal transport by Sinkhorn iterations (Eq. 5, Appendix C), one CTA per
+// image.  The (M+1) x (B+1) matrix stays in shared memory across all iterations when it fits, else
+// it is iterated in place in the image's L2-resident workspace tile.
+#pragma once
+#include "common.cuh"
+
+namespace rtp {
+
+struct OtParams {
+    float z, alpha, eps;
+    int iters;
+    int stop_fp;
+    float tol;
+};
+
+constexpr int kSinkThreads = 512;
+
+__device__ inline void lse_merge(float &m, float &s, float m2, float s2)
+{
+    const float mm = fmaxf(m, m2);
+    if (mm == -INFINITY) {
+        s = 0.f;
+        m = mm;
+        return;
+    }
+    s = s * expf(m - mm) + s2 * expf(m2 - mm);
+    m = mm;
+}
+
+// LOG = true : Z_ij = S-bar_ij / eps, duals u, v in the log domain,
+//              u_i = log mu_i - LSE_j(Z_ij + v_j), v_j = log nu_j - LSE_i(Z_ij + u_i).
+// LOG = false: K_ij = exp((S-bar_ij - c)/eps), c = max(1, z); duals carried as U = e^u, V = e^v
+//              (up to the constant e^{c/eps}, which cancels in the plan):
+//              U_i = mu_i / sum_j K_ij V_j, V_j = nu_j / sum_i K_ij U_i.
+// mu = [1_M, B], nu = [1_B, M].  Plan: P_ij = U_i K_ij V_j  (= exp(Z_ij + u_i + v_j)).
+template <bool LOG>
+__global__ void __launch_bounds__(kSinkThreads)
+sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__ counts,
+                const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ order,
+                float *__restrict__ kmat, int kmat_stride, int max_tokens, int total, OtParams p,
+                int smem_floats, int32_t *__restrict__ merged_idx,
+                int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
+                float *__restrict__ stats)
+{
+    extern __shared__ __align__(16) float sm[];
+    __shared__ float s_red[32];
+    const int img = blockIdx.x, tid = threadIdx.x;
+    constexpr int nth = kSinkThreads;
+    const int lane = tid & 31, warp = tid >> 5;
+    constexpr int nwarps = nth / 32;
+    int t_begin, N;
+    if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
+    const int M = counts[img], B = N - M;
+    if (B == 0) return;
+    const int R = M + 1, Cc = B + 1;
+
+    float *u = sm;
+    float *v = u + R;
+    float *part = v + Cc;                       // [2][nth]: partial column results and a second lane
+    constexpr int part_floats = 2 * nth;        // (running maxima for LOG, indices for the pairing)
+    float *Ks = part + part_floats;
+    const int lds = Cc | 1;                     // odd row stride: conflict-free column walks
+    const bool in_smem = (long long)R * lds + (R + Cc + part_floats) <= (long long)smem_floats;
+    float *Kg = kmat + kmat_offset(kmat_stride, t_begin, img);
+    float *Kp = in_smem ? Ks : Kg;
+    const int ld = in_smem ? lds : Cc;
+
+    const float inv_eps = 1.f / p.eps;
+    const float shift = fmaxf(1.f, p.z);
+
+    // build Z or K from the raw cosines (dustbin row and column = z, Eq. 5)
+    for (int idx = tid; idx < R * Cc; idx += nth) {
+        const int i = idx / Cc, j = idx - i * Cc;
+        const float s = (i < M && j < B) ? Kg[(size_t)i * Cc + j] : p.z;
+        Kp[(size_t)i * ld + j] = LOG ? s * inv_eps : expf((s - shift) * inv_eps);
+    }
+    const float init = LOG ? 0.f : 1.f;
+    for (int i = tid; i < R; i += nth) u[i] = init;
+    for (int j = tid; j < Cc; j += nth) v[j] = init;
+    __syncthreads();
+
+    const float mu_last = LOG ? logf((float)B) : (float)B;
+    const float nu_last = LOG ? logf((float)M) : (float)M;
+    const float mu_one = LOG ? 0.f : 1.f;
+
+    const int cols_per_pass = min(Cc, nth);
+    const int G = nth / cols_per_pass;
+    const int passes = (Cc + cols_per_pass - 1) / cols_per_pass;
+    const int cj = tid % cols_per_pass, cg = tid / cols_per_pass;
+    const bool row_per_thread = in_smem && R >= 128;
+
+    int done = 0;
+    float last_move = 0.f;
+    for (int it = 0; it < p.iters; ++it) {
+        // ---- u from v -------------------------------------------------------------------------
+        if (row_per_thread) {
+            for (int i = tid; i < R; i += nth) {
+                const float *row = Kp + (size_t)i * ld;
+                if (LOG) {
+                    float m = -INFINITY;
+                    for (int j = 0; j < Cc; ++j) m = fmaxf(m, row[j] + v[j]);
+                    float s = 0.f;
+                    for (int j = 0; j < Cc; ++j) s += expf(row[j] + v[j] - m);
+                    u[i] = (i < M ? mu_one : mu_last) - (m + logf(s));
+                } else {
+                    float s = 0.f;
+                    for (int j = 0; j < Cc; ++j) s = fmaf(row[j], v[j], s);
+                    u[i] = (i < M ? mu_one : mu_last) / s;
+                }
+            }
+        } else {
+            for (int i = warp; i < R; i += nwarps) {
+                const float *row = Kp + (size_t)i * ld;
+                if (LOG) {
+                    float m = -INFINITY;
+                    for (int j = lane; j < Cc; j += 32) m = fmaxf(m, row[j] + v[j]);
+                    m = warp_max(m);
+                    float s = 0.f;
+                    for (int j = lane; j < Cc; j += 32) s += expf(row[j] + v[j] - m);
+                    s = warp_sum(s);
+                    if (lane == 0) u[i] = (i < M ? mu_one : mu_last) - (m + logf(s));
+                } else {
+                    float s = 0.f;
+                    for (int j = lane; j < Cc; j += 32) s = fmaf(row[j], v[j], s);
+                    s = warp_sum(s);
+                    if (lane == 0) u[i] = (i < M ? mu_one : mu_last) / s;
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- v from u -------------------------------------------------------------------------
+        int cont = 0;
+        last_move = 0.f;
+        for (int ps = 0; ps < passes; ++ps) {
+            const int j = ps * cols_per_pass + cj;
+            const bool active = (cg < G) && (j < Cc);
+            float m = -INFINITY, s = 0.f;
+            if (active) {
+                if (LOG) {
+                    for (int i = cg; i < R; i += G) m = fmaxf(m, Kp[(size_t)i * ld + j] + u[i]);
+                    for (int i = cg; i < R; i += G) s += expf(Kp[(size_t)i * ld + j] + u[i] - m);
+                } else {
+                    for (int i = cg; i < R; i += G) s = fmaf(Kp[(size_t)i * ld + j], u[i], s);
+                }
+            }
+            if (G > 1) {
+                if (active) {
+                    part[cg * cols_per_pass + cj] = s;
+                    if (LOG) part[nth + cg * cols_per_pass + cj] = m;
+                }
+                __syncthreads();
+                if (active && cg == 0) {
+                    for (int g = 1; g < G; ++g) {
+                        if (LOG) lse_merge(m, s, part[nth + g * cols_per_pass + cj],
+                                           part[g * cols_per_pass + cj]);
+                        else s += part[g * cols_per_pass + cj];
+                    }
+                }
+            }
+            if (active && cg == 0) {
+                const float nu = (j < B) ? mu_one : nu_last;
+                const float nv = LOG ? nu - (m + logf(s)) : nu / s;
+                const float ov = v[j];
+                const float move = LOG ? fabsf(nv - ov) : fabsf(nv - ov) / fabsf(ov);
+                last_move = fmaxf(last_move, move);
+                if (p.tol > 0.f) cont |= (move > p.tol) ? 1 : 0;
+                else cont |= p.stop_fp ? (__float_as_uint(nv) != __float_as_uint(ov)) : 1;
+                v[j] = nv;
+            }
+            if (passes > 1 && G > 1) __syncthreads();
+        }
+        ++done;
+        if (!__syncthreads_or(cont)) break;
+    }
+    __syncthreads();
+
+    // largest dual move of the last executed iteration
+    {
+        float mv = warp_max(last_move);
+        if (lane == 0) s_red[warp] = mv;
+        __syncthreads();
+        if (warp == 0) {
+            mv = warp_max(lane < nwarps ? s_red[lane] : 0.f);
+            if (lane == 0) {
+                stats[(size_t)img * kStats + 5] = (float)done;
+                stats[(size_t)img * kStats + 6] = mv;
+            }
+        }
+    }
+
+    // ---- pairing: partner_j = argmax_i P_ij = argmax_i (Z_ij + u_i), ties to the lower i -------
+    // weight_j = (U_i K_ij) V_j, the same product the plan below stores, so weight == P there.
+    const int seg = t_begin - out_offsets[img];
+    const int32_t *ord = order + t_begin;
+    int *parti = reinterpret_cast<int *>(part + nth);
+    for (int ps = 0; ps < passes; ++ps) {
+        const int j = ps * cols_per_pass + cj;
+        const bool active = (cg < G) && (j < B);
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
+        if (active) {
+            for (int i = cg; i < M; i += G) {
+                const float k = Kp[(size_t)i * ld + j];
+                const float key = LOG ? k + u[i] : k * u[i];
+                if (key > best) {   // i ascends within a thread: strict > keeps the lower index
+                    best = key;
+                    bi = i;
+                }
+            }
+        }
+        if (G > 1) {
+            __syncthreads();    // part[] may still be read by the previous pass / the sweeps
+            if (active) {
+                part[cg * cols_per_pass + cj] = best;
+                parti[cg * cols_per_pass + cj] = bi;
+            }
+            __syncthreads();
+            if (active && cg == 0) {
+                for (int g = 1; g < G; ++g) {
+                    const float ob = part[g * cols_per_pass + cj];
+                    const int oi = parti[g * cols_per_pass + cj];
+                    if (ob > best || (ob == best && oi < bi)) {
+                        best = ob;
+                        bi = oi;
+                    }
+                }
+            }
+        }
+        if (active && cg == 0) {
+            merged_idx[seg + j] = ord[M + j];
+            merge_partner[seg + j] = bi;
+            merge_weight[seg + j] = LOG ? expf(best + v[j]) : best * v[j];
+        }
+    }
+    __syncthreads();
+
+    // ---- plan P (non-dustbin block), written to the workspace tile with row stride B+1 --------
+    for (int idx = tid; idx < M * B; idx += nth) {
+        const int i = idx / B, j = idx - i * B;
+        const float k = Kp[(size_t)i * ld + j];
+        Kg[(size_t)i * Cc + j] = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
+    }
+}
+
+}  // namespace rtp

@@ -1,0 +1,198 @@
+"""Helpers of the GPU parity tests: run the CUDA path through the C ABI, run the CPU oracle on the
+same seeded inputs, and compare element by element.
+
+Tolerances (stated once, used by every parity test):
+  * counts, out_offsets, kept_idx, merged_idx: bit-exact.
+  * merge_partner: bit-exact where the oracle's top-2 gap of log P over the kept tokens is at least
+    PARTNER_GAP (1e-3); below that several answers are correct to working precision, and the GPU's
+    choice must lie in the oracle's within-gap candidate set.
+  * merged features Y: |y - y*| <= tol * max(|y*|, rms(y* row)) with tol = 1e-2 for bf16 storage
+    (fp32 accumulation) and 1e-5 for fp32 storage; y* is the oracle's fp64 value.
+  * phi: 2e-5 absolute (fp32 sum of ~N unit vectors); r: 1e-5; plan weights: 1e-4 relative.
+Inputs have sorted-norm gaps >= 1.2e-3 (generator) and, for dynamic ratios, |frac(r N) - 1/2| >= 1e-3
+(enforced here by nudging rho, an input), so every integer decision is the same in fp32 and fp64.
+"""
+from __future__ import annotations
+
+import os
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from oracle import oracle
+from paper_2605_00392_b200 import binding, synth
+
+PARTNER_GAP = 1e-3
+FEATURE_TOL = {torch.bfloat16: 1e-2, torch.float32: 1e-5}
+ROUND_MARGIN = 1e-3
+
+
+def oracle_params(p: Dict[str, float]) -> oracle.Params:
+    return oracle.Params(dynamic=bool(p["dynamic"]), r_fixed=float(np.float32(p["r_fixed"])),
+                         phi_lo=float(np.float32(p["phi_lo"])), phi_hi=float(np.float32(p["phi_hi"])),
+                         r_max=float(np.float32(p["r_max"])), z=float(np.float32(p["z"])),
+                         alpha=float(np.float32(p["alpha"])), eps=float(np.float32(p["eps"])),
+                         iters=int(p["iters"]))
+
+
+def cpu_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return os.cpu_count() or 1
+
+
+def settle_rho(w: synth.Workload, images: Sequence[int]) -> None:
+    """Move rho (an input) of any image whose r*N sits within ROUND_MARGIN of a rounding boundary,
+    so that fp32 and fp64 evaluate B = floor(r N + 1/2) alike.  Only dynamic runs depend on rho."""
+    if not w.params["dynamic"]:
+        return
+    p = oracle_params(w.params)
+    for i in images:
+        T = w.image_f64(i)
+        ph = oracle.phi(T)
+        for _ in range(50):
+            r, _, _ = oracle.ratio(ph, float(w.rho[i]), T.shape[0], dynamic=True, phi_lo=p.phi_lo,
+                                   phi_hi=p.phi_hi, r_max=p.r_max)
+            frac = r * T.shape[0] - np.floor(r * T.shape[0])
+            if abs(frac - 0.5) >= ROUND_MARGIN or r in (0.0, p.r_max):
+                break
+            w.rho[i] = np.float32(min(1.0, float(w.rho[i]) + 0.003))
+
+
+@dataclass
+class GpuResult:
+    out: binding.Outputs           # tensors copied to the CPU
+    launches: int
+    status_bits: int
+
+
+def run_gpu(w: synth.Workload, *, overrides: Optional[Dict[str, float]] = None,
+            host_path: bool = False, plan: Optional[binding.Plan] = None) -> GpuResult:
+    dev = torch.device("cuda", 0)
+    p = dict(w.params)
+    if overrides:
+        p.update(overrides)
+    own = plan is None
+    if own:
+        plan = binding.Plan(w.d, w.X.dtype, max(w.batch, 1), max(w.total_tokens, 1),
+                            max(w.max_tokens, 1), device=dev)
+    rho_dev = torch.from_numpy(w.rho.copy()).to(dev) if w.batch else None
+    fields = {k: (int(v) if k in ("dynamic", "iters", "form", "stop_at_fixed_point") else float(v))
+              for k, v in p.items()}
+    if host_path:
+        params = binding.make_params(None, **fields)
+        out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, "cpu", pin=True)
+        X = w.X.pin_memory()
+        offs = torch.from_numpy(w.offsets.copy()).pin_memory()
+        rho = torch.from_numpy(w.rho.copy()).pin_memory()
+        plan.run_host(X, offs, rho, params, out)
+        torch.cuda.synchronize()
+        res = GpuResult(out=out, launches=plan.last_launch_count, status_bits=0)
+    else:
+        params = binding.make_params(rho_dev, **fields)
+        out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, dev)
+        X = w.X.to(dev)
+        offs = torch.from_numpy(w.offsets.copy()).to(dev)
+        plan.run(X, offs, params, out)
+        bits = plan.query_status()
+        cpu = binding.Outputs(**{k: getattr(out, k).cpu() for k in out.__dataclass_fields__})
+        res = GpuResult(out=cpu, launches=plan.last_launch_count, status_bits=bits)
+    if own:
+        plan.close()
+    return res
+
+
+def compare_image(w: synth.Workload, i: int, ref: oracle.ImageResult, g: binding.Outputs,
+                  report: Dict[str, float]) -> None:
+    """Element-by-element comparison of image i; raises AssertionError with context."""
+    tag = "%s image %d" % (w.name, i)
+    N = ref.N
+    o0, o1 = int(g.out_offsets[i]), int(g.out_offsets[i + 1])
+    assert int(g.counts[i]) == ref.M, (tag, int(g.counts[i]), ref.M)
+    assert o1 - o0 == ref.M, tag
+    st = g.stats[i].numpy()
+    assert abs(st[0] - ref.phi) <= 2e-5, (tag, st[0], ref.phi)
+    assert abs(st[2] - ref.r) <= 1e-5, (tag, st[2], ref.r)
+    assert int(st[3]) == ref.M and int(st[4]) == ref.B, tag
+    np.testing.assert_array_equal(g.kept_idx[o0:o1].numpy(), ref.kept, err_msg=tag)
+    seg = int(w.offsets[i]) - o0
+    np.testing.assert_array_equal(g.merged_idx[seg:seg + ref.B].numpy(), ref.prop, err_msg=tag)
+
+    # merged features
+    y = g.Y[o0:o1].to(torch.float64).numpy()
+    ystar = ref.Y
+    rms = np.sqrt(np.mean(ystar * ystar, axis=1, keepdims=True))
+    denom = np.maximum(np.abs(ystar), rms)
+    err = np.abs(y - ystar) / np.where(denom > 0, denom, 1.0)
+    tol = FEATURE_TOL[w.X.dtype]
+    worst = float(err.max()) if err.size else 0.0
+    report["max_feature_err"] = max(report.get("max_feature_err", 0.0), worst)
+    assert worst <= tol, (tag, worst, tol)
+    if ref.B == 0:   # retention 1: output rows are the input rows, bit for bit
+        assert torch.equal(g.Y[o0:o1], w.X[int(w.offsets[i]):int(w.offsets[i + 1])]), tag
+        return
+
+    # pairs
+    gp = g.merge_partner[seg:seg + ref.B].numpy()
+    gw = g.merge_weight[seg:seg + ref.B].numpy().astype(np.float64)
+    decisive = ref.gap >= PARTNER_GAP
+    np.testing.assert_array_equal(gp[decisive], ref.partner[decisive], err_msg=tag)
+    report["pairs"] = report.get("pairs", 0) + ref.B
+    report["pairs_within_gap"] = report.get("pairs_within_gap", 0) + int((~decisive).sum())
+    if (~decisive).any():
+        assert ref.Pbar is not None, "oracle must be run with want_plan for near-tie columns"
+        logP = np.log(ref.Pbar[:-1, :-1])
+        for j in np.nonzero(~decisive)[0]:
+            assert 0 <= gp[j] < ref.M and logP[gp[j], j] >= logP[:, j].max() - PARTNER_GAP, (tag, j)
+    same = gp == ref.partner
+    np.testing.assert_allclose(gw[same], ref.weight[same], rtol=1e-4, err_msg=tag)
+    assert st[5] >= 1 or w.params.get("iters", 100) == 0, tag
+
+
+def check_workload(w: synth.Workload, *, images: Optional[Sequence[int]] = None,
+                   overrides: Optional[Dict[str, float]] = None, host_path: bool = False,
+                   plan: Optional[binding.Plan] = None) -> Dict[str, float]:
+    """GPU run of the whole workload + oracle on `images` (default: all); returns a small report."""
+    imgs = list(range(w.batch)) if images is None else list(images)
+    if overrides:
+        w.params.update(overrides)
+    settle_rho(w, imgs)
+    res = run_gpu(w, host_path=host_path, plan=plan)
+    assert res.status_bits == 0, res.status_bits
+    g = res.out
+    # whole-batch structure (any size)
+    counts = g.counts[:w.batch].numpy().astype(np.int64)
+    offs = g.out_offsets.numpy().astype(np.int64)
+    np.testing.assert_array_equal(offs, np.concatenate([[0], np.cumsum(counts)]))
+    lens = np.diff(w.offsets.astype(np.int64))
+    assert np.all(counts >= 1) and np.all(counts <= lens)
+    for i in range(w.batch):      # kept and merged partition {0..N_i-1}, each ascending
+        o0, o1 = offs[i], offs[i + 1]
+        seg = int(w.offsets[i]) - o0
+        k = g.kept_idx[o0:o1].numpy()
+        m = g.merged_idx[seg:seg + lens[i] - counts[i]].numpy()
+        assert np.all(np.diff(k) > 0) and np.all(np.diff(m) > 0)
+        both = np.concatenate([k, m])
+        assert len(both) == lens[i] and np.array_equal(np.sort(both), np.arange(lens[i]))
+    refs = oracle.run_batch(w.X_f64() if images is None else _SparseX(w), w.offsets,
+                            oracle_params(w.params), w.rho, images=imgs, threads=cpu_threads(),
+                            want_plan=True)
+    report: Dict[str, float] = {"launches": res.launches}
+    for i, ref in zip(imgs, refs.images):
+        compare_image(w, i, ref, g, report)
+    report["mean_retention"] = float(counts.sum()) / float(lens.sum())
+    report["mean_iters"] = float(g.stats[:w.batch, 5].mean())
+    return report
+
+
+class _SparseX:
+    """Lazily converts only the requested images of a big batch to fp64."""
+
+    def __init__(self, w: synth.Workload):
+        self.w = w
+
+    def __getitem__(self, sl: slice):
+        return self.w.X[sl.start:sl.stop].to(torch.float64).numpy()

@@ -1,0 +1,215 @@
+"""Edge cases, parameter ranges and device-side error reporting of the CUDA path.  Marked gpu."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_00392_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def parity():
+    import parity as _p
+    return _p
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2605_00392_b200 import binding as _b
+    return _b
+
+
+RAGGED = [1, 2, 3, 5, 63, 64, 65, 127, 129, 400, 1]
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_ragged_lengths_fixed_ratio(parity, dtype):
+    w = synth.ragged(RAGGED, dtype=dtype, params=dict(r_fixed=0.3))
+    parity.check_workload(w)
+
+
+def test_ragged_dynamic(parity):
+    w = synth.ragged(RAGGED, params=dict(dynamic=1, phi_lo=0.0, phi_hi=0.6, r_max=0.5))
+    parity.check_workload(w)
+
+
+def test_retention_one_is_identity(parity):
+    w = synth.ragged([7, 64, 200], params=dict(r_fixed=0.0))
+    rep = parity.check_workload(w)
+    assert rep["mean_retention"] == 1.0 and rep["launches"] == 3   # stage 2 is not launched
+
+
+def test_rho_one_prunes_nothing(parity):
+    w = synth.ragged([50, 70], params=dict(dynamic=1, phi_hi=0.5))
+    w.rho[:] = 1.0
+    assert parity.check_workload(w)["mean_retention"] == 1.0
+
+
+def test_single_kept_token(parity):
+    w = synth.ragged([9, 40], params=dict(r_fixed=0.999))
+    rep = parity.check_workload(w)
+    assert rep["mean_retention"] == pytest.approx(2.0 / 49.0)
+
+
+def test_alpha_zero_is_plain_pruning(parity, binding):
+    w = synth.ragged([33, 90], params=dict(r_fixed=0.25, alpha=0.0))
+    parity.check_workload(w)
+    g = parity.run_gpu(w).out
+    for i in range(2):
+        o0, o1 = int(g.out_offsets[i]), int(g.out_offsets[i + 1])
+        rows = w.X[int(w.offsets[i]):int(w.offsets[i + 1])][g.kept_idx[o0:o1].long()]
+        assert torch.equal(g.Y[o0:o1], rows)
+
+
+@pytest.mark.parametrize("over", [dict(form=1), dict(eps=0.1), dict(eps=0.3, z=0.6),
+                                  dict(iters=0), dict(iters=1), dict(iters=7, stop_at_fixed_point=0),
+                                  dict(z=1.0), dict(z=0.0, alpha=0.5), dict(eps=0.05, iters=300)])
+def test_ot_parameter_ranges(parity, over):
+    w = synth.ragged([64, 150, 31], params=dict(r_fixed=0.25))
+    parity.check_workload(w, overrides=over)
+
+
+def test_fixed_point_stop_equals_all_iterations(parity):
+    w = synth.make("base", batch=6)
+    a = parity.run_gpu(w, overrides=dict(stop_at_fixed_point=1)).out
+    b = parity.run_gpu(w, overrides=dict(stop_at_fixed_point=0)).out
+    assert torch.equal(a.Y, b.Y) and torch.equal(a.merge_partner, b.merge_partner)
+    assert torch.equal(a.merge_weight, b.merge_weight)
+    assert float(b.stats[:6, 5].min()) == 100.0 and float(a.stats[:6, 5].max()) <= 100.0
+
+
+def test_tolerance_stop_runs_fewer_iterations(parity):
+    w = synth.make("base", batch=4)
+    a = parity.run_gpu(w, overrides=dict(tol=1e-4)).out
+    assert 1.0 <= float(a.stats[:4, 5].max()) < 30.0 and float(a.stats[:4, 6].max()) <= 1e-4
+    parity.check_workload(w, overrides=dict(tol=1e-6))
+
+
+def test_large_tile_leaves_shared_memory(parity):
+    # N = 1156 at r = 0.5: a 579 x 579 matrix (1.3 MB) that cannot stay in one CTA's shared memory
+    w = synth.ragged([1156, 456], params=dict(r_fixed=0.5))
+    parity.check_workload(w)
+
+
+def test_exact_ties_keep_lower_index(parity):
+    w = synth.ragged([40], params=dict(r_fixed=0.5))
+    w.X[21] = w.X[3]
+    w.X[30] = w.X[3]
+    w.X[35] = w.X[8]
+    parity.check_workload(w)
+    w.X[:] = w.X[0]                      # every token identical
+    g = parity.run_gpu(w).out
+    assert g.kept_idx[:20].tolist() == list(range(20))
+    assert g.merge_partner[:20].tolist() == [0] * 20
+    parity.check_workload(w)
+
+
+@pytest.mark.parametrize("d,dtype", [(8, torch.bfloat16), (64, torch.float32), (264, torch.bfloat16),
+                                     (1000, torch.float32), (4096, torch.bfloat16)])
+def test_other_widths(parity, d, dtype):
+    w = synth.ragged([70, 33], d=d, dtype=dtype, params=dict(r_fixed=0.3))
+    parity.check_workload(w)
+
+
+def test_select_entry_point(parity, binding):
+    w = synth.make("base", batch=3)
+    parity.settle_rho(w, range(3))
+    dev = torch.device("cuda", 0)
+    plan = binding.Plan(w.d, w.X.dtype, 3, w.total_tokens, 256, device=dev)
+    out = binding.Outputs.allocate(w.total_tokens, 3, w.d, w.X.dtype, dev)
+    norms = torch.zeros(w.total_tokens, device=dev)
+    order = torch.zeros(w.total_tokens, dtype=torch.int32, device=dev)
+    rho = torch.from_numpy(w.rho).to(dev)
+    fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w.params.items()}
+    plan.select(w.X.to(dev), torch.from_numpy(w.offsets).to(dev), binding.make_params(rho, **fields),
+                out, norms, order)
+    assert plan.query_status() == 0 and plan.last_launch_count == 2
+    from oracle import oracle
+    ref = oracle.run_batch(w.X_f64(), w.offsets, parity.oracle_params(w.params), w.rho)
+    for i, im in enumerate(ref.images):
+        a = int(w.offsets[i])
+        np.testing.assert_allclose(norms[a:a + 256].cpu().numpy(), im.C, rtol=2e-6)
+        assert int(out.counts[i]) == im.M
+        np.testing.assert_array_equal(order[a:a + im.M].cpu().numpy(), im.kept)
+        np.testing.assert_array_equal(order[a + im.M:a + 256].cpu().numpy(), im.prop)
+    plan.close()
+
+
+def test_empty_batch(binding):
+    dev = torch.device("cuda", 0)
+    plan = binding.Plan(1280, torch.bfloat16, 4, 100, 50, device=dev)
+    out = binding.Outputs.allocate(0, 0, 1280, torch.bfloat16, dev)
+    out.out_offsets.fill_(9)
+    plan.run(torch.empty((0, 1280), dtype=torch.bfloat16, device=dev),
+             torch.zeros(1, dtype=torch.int32, device=dev), binding.make_params(), out)
+    torch.cuda.synchronize()
+    assert out.out_offsets.tolist() == [0] and plan.last_launch_count == 0
+    plan.close()
+
+
+def test_device_status_word(parity, binding):
+    dev = torch.device("cuda", 0)
+    w = synth.ragged([20, 30])
+    plan = binding.Plan(w.d, w.X.dtype, 2, 50, 30, device=dev)
+    out = binding.Outputs.allocate(50, 2, w.d, w.X.dtype, dev)
+    X = w.X.to(dev)
+    X[25, 7] = float("nan")
+    offs = torch.from_numpy(w.offsets).to(dev)
+    plan.run(X, offs, binding.make_params(), out)
+    assert plan.query_status() & binding.DEV_NONFINITE
+    assert plan.query_status() == 0                        # reading clears it
+    # offsets that break the contract (image longer than the plan allows) are reported, not chased
+    bad = torch.tensor([0, 45, 50], dtype=torch.int32, device=dev)
+    plan.run(w.X.to(dev), bad, binding.make_params(), out)
+    assert plan.query_status() & binding.DEV_BAD_OFFSETS
+    # and the plan still works afterwards
+    plan.run(w.X.to(dev), offs, binding.make_params(), out)
+    assert plan.query_status() == 0 and int(out.out_offsets[2]) == 15 + 22
+    plan.close()
+
+
+def test_host_side_argument_errors(binding):
+    dev = torch.device("cuda", 0)
+    with pytest.raises(binding.RtpruneError) as e:
+        binding.Plan(1281, torch.bfloat16, 1, 10, 10, device=dev)
+    assert e.value.status == 2
+    with pytest.raises(binding.RtpruneError):
+        binding.Plan(1280, torch.bfloat16, 1, 10 ** 5, 9000, device=dev)
+    plan = binding.Plan(1280, torch.bfloat16, 2, 100, 60, device=dev)
+    out = binding.Outputs.allocate(100, 2, 1280, torch.bfloat16, dev)
+    X = torch.zeros((100, 1280), dtype=torch.bfloat16, device=dev)
+    offs = torch.tensor([0, 50, 100], dtype=torch.int32, device=dev)
+    for bad in [dict(r_fixed=1.0), dict(r_fixed=-0.1), dict(eps=0.0), dict(iters=-1), dict(form=7),
+                dict(dynamic=1, phi_lo=0.5, phi_hi=0.5), dict(dynamic=1, r_max=0.0),
+                dict(form=2, eps=0.1), dict(tol=-1.0), dict(z=float("inf"))]:
+        with pytest.raises(binding.RtpruneError) as e:
+            plan.run(X, offs, binding.make_params(**bad), out)
+        assert e.value.status == 1, bad
+    with pytest.raises(binding.RtpruneError):                 # more tokens than planned
+        plan.run(torch.zeros((101, 1280), dtype=torch.bfloat16, device=dev), offs,
+                 binding.make_params(), out)
+    with pytest.raises(binding.RtpruneError):                 # misaligned X
+        lib = binding.lib()
+        p = binding.make_params()
+        binding._check(lib.rtprune_run(plan.handle, None, X.data_ptr() + 2, offs.data_ptr(), 2, 100,
+                                       ctypes.byref(p), plan.workspace.data_ptr(),
+                                       plan.workspace_bytes, out.Y.data_ptr(),
+                                       out.out_offsets.data_ptr(), out.counts.data_ptr(),
+                                       out.kept_idx.data_ptr(), out.merged_idx.data_ptr(),
+                                       out.merge_partner.data_ptr(), out.merge_weight.data_ptr(),
+                                       out.stats.data_ptr()), "rtprune_run")
+    with pytest.raises(binding.RtpruneError) as e:            # workspace too small
+        lib = binding.lib()
+        p = binding.make_params()
+        binding._check(lib.rtprune_run(plan.handle, None, X.data_ptr(), offs.data_ptr(), 2, 100,
+                                       ctypes.byref(p), plan.workspace.data_ptr(), 1024,
+                                       out.Y.data_ptr(), out.out_offsets.data_ptr(),
+                                       out.counts.data_ptr(), out.kept_idx.data_ptr(),
+                                       out.merged_idx.data_ptr(), out.merge_partner.data_ptr(),
+                                       out.merge_weight.data_ptr(), out.stats.data_ptr()),
+                       "rtprune_run")
+    assert e.value.status == 3
+    plan.close()

@@ -1,0 +1,59 @@
+"""Multi-process use of the path: images are independent, so N ranks each take a contiguous slice of
+the batch and nothing is exchanged on the data path.  Two gloo ranks on CPU check the host-side
+logic: the slices cover the batch, and per-rank results (here from the CPU oracle, standing in for
+the GPU path) concatenate to the single-process result once the packed offsets are shifted by the
+counts of the lower ranks."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2605_00392_b200 import binding, synth
+
+
+def _free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank: int, world: int, port: int, ret):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import oracle
+    w = synth.ragged([40, 17, 64, 9, 33], d=32, dtype=torch.float32, params=dict(r_fixed=0.25))
+    lo, hi = binding.shard_images(w.batch, world, rank)
+    res = oracle.run_batch(w.X_f64(), w.offsets, oracle.Params(r_fixed=0.25), w.rho,
+                           images=list(range(lo, hi)))
+    counts = torch.tensor([im.M for im in res.images], dtype=torch.int64)
+    # the only cross-rank datum: how many packed rows the lower ranks produce
+    mine = torch.tensor([int(counts.sum())])
+    allc = [torch.zeros(1, dtype=torch.int64) for _ in range(world)]
+    dist.all_gather(allc, mine)
+    base = int(sum(int(c) for c in allc[:rank]))
+    offs = base + np.concatenate([[0], np.cumsum(counts.numpy())])
+    ret[rank] = (lo, hi, offs.tolist(), [im.kept.tolist() for im in res.images])
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_partition_the_batch():
+    world = 2
+    port = _free_port()
+    mgr = mp.Manager()
+    ret = mgr.dict()
+    mp.spawn(_worker, args=(world, port, ret), nprocs=world, join=True)
+    from oracle import oracle
+    w = synth.ragged([40, 17, 64, 9, 33], d=32, dtype=torch.float32, params=dict(r_fixed=0.25))
+    ref = oracle.run_batch(w.X_f64(), w.offsets, oracle.Params(r_fixed=0.25), w.rho)
+    assert ret[0][0] == 0 and ret[0][1] == ret[1][0] and ret[1][1] == w.batch
+    got_offs = ret[0][2][:-1] + ret[1][2]
+    assert got_offs == ref.out_offsets.tolist()
+    kept = ret[0][3] + ret[1][3]
+    assert kept == [im.kept.tolist() for im in ref.images]
