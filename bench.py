@@ -150,6 +150,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -235,8 +236,8 @@ def main() -> None:
     hoffs = [torch.from_numpy(w.offsets).pin_memory() for w in sets]
     hrho = [torch.from_numpy(w.rho).pin_memory() for w in sets]
     hparams = binding.make_params(None, **fields)
-    e2e_steps = max(3, min(args.steps, 20))
-    for i in range(2):
+    e2e_steps = 1 if args.no_e2e else max(3, min(args.steps, 20))
+    for i in range(0 if args.no_e2e else 2):
         plan.run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_out)
     barrier()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

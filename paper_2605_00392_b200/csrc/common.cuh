@@ -25,18 +25,24 @@ struct WsLayout {
     size_t norms;      // float [total]            C_k
     size_t spart;      // float [batch][chunks][d] partial sums of the unit tokens
     size_t order;      // int32 [total]            per image: kept indices then pruned indices
+    size_t kpos;       // int32 [total]            per token: position among kept, or -1 - position
+                       //                          among pruned
     size_t kmat;       // float [kmat_floats]      per-image score / kernel / plan matrix
     size_t total;      // bytes
     int chunks;        // chunks per image = ceil(max_tokens_per_image / kChunkTokens)
     int kmat_stride;   // floats of kmat per token-unit, see kmat_offset()
 };
 
-// Image i's matrix starts at float offset kmat_stride * (offsets[i] + 2 i).  Its (M+1) x (B+1)
-// cells always fit because (M+1)(B+1) <= (N+2)^2 / 4 <= kmat_stride * (N+2), kmat_stride being
-// ceil((maxN+2)/4).
+// Row pitch (floats) of an image's score / plan matrix: B real columns + the dustbin column,
+// rounded up to a multiple of 4 so that rows can be written as 16-byte vectors.
+__host__ __device__ inline int score_pitch(int B) { return (B + 4) & ~3; }
+
+// Image i's matrix starts at float offset kmat_stride * (offsets[i] + 8 i), a multiple of 4.  Its
+// (M+1) rows of score_pitch(B) floats always fit: (M+1)(B+4) <= (N+5)^2 / 4 <= kmat_stride * (N+8),
+// kmat_stride being 4 * ceil((maxN+8)/16).
 __host__ __device__ inline size_t kmat_offset(int kmat_stride, int tok_offset, int img)
 {
-    return (size_t)kmat_stride * (size_t)(tok_offset + 2 * img);
+    return (size_t)kmat_stride * (size_t)(tok_offset + 8 * img);
 }
 
 // Reads image `img`'s token range and checks it against the contract (1 <= N <= max_tokens, rows

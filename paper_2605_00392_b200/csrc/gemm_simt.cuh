@@ -11,7 +11,7 @@ constexpr int kSimtBK = 32;
 
 // ---------------------------------------------------------------------------------------------
 // S_ij = x_i . x_j / (|x_i| |x_j|), i in T_kept, j in T_prop.  grid = (mtiles * btiles, batch).
-// Rows are gathered through the image's order[] list.  Output: kmat[i * (B+1) + j].
+// Rows are gathered through the image's order[] list.  Output: kmat[i * score_pitch(B) + j].
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -89,7 +89,7 @@ scores_simt_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets,
     }
 
     float *Kimg = kmat + kmat_offset(kmat_stride, t_begin, img);
-    const int ld = B + 1;
+    const int ld = score_pitch(B);
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
         const int i = i0 + ty * 4 + p;
@@ -107,7 +107,7 @@ scores_simt_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets,
 
 // ---------------------------------------------------------------------------------------------
 // y_i = x_i + alpha * sum_j P_ij x_j (Eq. 7), written packed: Y row out_offsets[img] + i, together
-// with kept_idx.  grid = (mtiles * dtiles, batch).  P is read from kmat (row stride B+1).
+// with kept_idx.  grid = (mtiles * dtiles, batch).  P is read from kmat (row pitch score_pitch(B)).
 // With B = 0 the rows are copied unchanged.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
@@ -149,7 +149,7 @@ merge_simt_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, 
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
     const float *Pimg = kmat + kmat_offset(kmat_stride, t_begin, img);
-    const int ld = B + 1;
+    const int ld = score_pitch(B);
     for (int j0 = 0; j0 < B; j0 += BK) {
         for (int v = tid; v < BK * kSimtTile; v += 256) {
             {   // P tile: consecutive threads walk j (contiguous in memory)

@@ -4,9 +4,11 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <type_traits>
 
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "scores_umma.cuh"
 #include "sinkhorn.cuh"
 #include "stage1.cuh"
 
@@ -25,6 +27,7 @@ struct rtprune_plan_s {
     int sm_count;
     int smem_optin;       // bytes of opt-in shared memory per CTA
     int sink_smem_bytes;  // dynamic shared memory of the Sinkhorn kernel
+    void *encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
     int last_launches;
     int last_cuda_error;
     bool profiling;
@@ -41,7 +44,7 @@ WsLayout make_layout(int d, int max_batch, int64_t max_total, int max_tokens)
 {
     WsLayout L;
     L.chunks = (max_tokens + kChunkTokens - 1) / kChunkTokens;
-    L.kmat_stride = (max_tokens + 2 + 3) / 4;
+    L.kmat_stride = 4 * ((max_tokens + 8 + 15) / 16);
     size_t off = 0;
     L.header = off;
     off = align_up(off + sizeof(WsHeader), 256);
@@ -51,8 +54,10 @@ WsLayout make_layout(int d, int max_batch, int64_t max_total, int max_tokens)
     off = align_up(off + sizeof(float) * (size_t)max_batch * L.chunks * d, 256);
     L.order = off;
     off = align_up(off + sizeof(int32_t) * (size_t)max_total, 256);
+    L.kpos = off;
+    off = align_up(off + sizeof(int32_t) * (size_t)max_total, 256);
     L.kmat = off;
-    off = align_up(off + sizeof(float) * (size_t)L.kmat_stride * (size_t)(max_total + 2 * (int64_t)max_batch), 256);
+    off = align_up(off + sizeof(float) * (size_t)L.kmat_stride * (size_t)(max_total + 8 * (int64_t)max_batch), 256);
     L.total = off;
     return L;
 }
@@ -81,6 +86,32 @@ void launched(rtprune_plan_t *plan, cudaStream_t st, const char *name)
         plan->ev_name[plan->ev_count] = name;
         cudaEventRecord(plan->ev[++plan->ev_count], st);
     }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix with the given row pitch, boxes of
+// box_cols x box_rows elements, 128-byte swizzle, out-of-range elements read as zero.
+bool make_tmap_bf16(rtprune_plan_t *plan, CUtensorMap *map, const void *base, uint64_t rows,
+                    uint64_t cols, uint64_t pitch_bytes, uint32_t box_cols, uint32_t box_rows)
+{
+    if (!plan->encode_tiled) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch_bytes};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = ((EncodeTiledFn)plan->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        plan->last_cuda_error = (int)cudaErrorInvalidValue;
+        return false;
+    }
+    return true;
 }
 
 rtprune_status_t check_params(const rtprune_params_t *p)
@@ -114,6 +145,7 @@ bool use_log_form(const rtprune_params_t *p)
 int max_pruned(const rtprune_params_t *p, int max_tokens)
 {
     const float r = p->dynamic ? std::fmin(p->r_max, 1.f) : p->r_fixed;
+    if (r <= 0.f) return 0;  // nothing can be pruned: stage 2 is not launched
     long b = (long)std::floor((double)r * max_tokens + 0.5) + 1;  // +1: fp32 vs fp64 rounding slack
     if (b > max_tokens - 1) b = max_tokens - 1;
     if (b < 0) b = 0;
@@ -186,6 +218,7 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
     float *norms = (float *)(ws + L.norms);
     float *spart = (float *)(ws + L.spart);
     int32_t *order = (int32_t *)(ws + L.order);
+    int32_t *kpos = (int32_t *)(ws + L.kpos);
     cudaError_t e = (plan->dtype == RTPRUNE_BF16)
                         ? launch_norm_stats<__nv_bfloat16>(plan, st, X, offsets, batch, total, norms, spart, hdr)
                         : launch_norm_stats<float>(plan, st, X, offsets, batch, total, norms, spart, hdr);
@@ -194,7 +227,7 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
     RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
     const size_t smem = sizeof(float) * (size_t)plan->max_tokens;
     select_kernel<<<batch, 1024, smem, st>>>(offsets, batch, plan->d, L.chunks, plan->max_tokens,
-                                             total, rp, params->rho, norms, spart, order, counts,
+                                             total, rp, params->rho, norms, spart, order, kpos, counts,
                                              out_offsets, stats, norms_out, order_out, hdr);
     if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
     launched(plan, st, "select");
@@ -216,11 +249,24 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     const int mtiles = (maxN + kSimtTile - 1) / kSimtTile;
 
     if (maxB > 0) {
-        const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
-        dim3 grid(mtiles * btiles, batch);
-        scores_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, btiles,
-                                                   o.counts, order, norms, kmat, L.kmat_stride,
-                                                   maxN, total);
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            // tensor-core path: one CTA per (128 consecutive tokens, image)
+            CUtensorMap tmapX;
+            if (!make_tmap_bf16(plan, &tmapX, X, (uint64_t)total, (uint64_t)plan->d,
+                                (uint64_t)plan->d * 2, kScBK, kScTileM))
+                return RTPRUNE_ERR_CUDA;
+            dim3 grid((maxN + kScTileM - 1) / kScTileM, batch);
+            scores_umma_kernel<<<grid, kScThreads, kScSmemBytes, st>>>(
+                tmapX, (const __nv_bfloat16 *)X, offsets, plan->d, o.counts, order,
+                (const int32_t *)(ws + L.kpos), norms, kmat, L.kmat_stride, maxN, total,
+                (WsHeader *)(ws + L.header));
+        } else {
+            const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
+            dim3 grid(mtiles * btiles, batch);
+            scores_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, btiles,
+                                                       o.counts, order, norms, kmat,
+                                                       L.kmat_stride, maxN, total);
+        }
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
         launched(plan, st, "scores");
 
@@ -378,6 +424,25 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
                                    p->sink_smem_bytes))) {
         delete p;
         return RTPRUNE_ERR_CUDA;
+    }
+    p->encode_tiled = nullptr;
+    {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            p->encode_tiled = fn;
+        else
+            (void)cudaGetLastError();
+    }
+    if (dtype == RTPRUNE_BF16) {
+        if (!p->encode_tiled ||
+            !c.ok(cudaFuncSetAttribute(scores_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kScSmemBytes))) {
+            if (!p->last_cuda_error) p->last_cuda_error = (int)cudaErrorNotSupported;
+            delete p;
+            return RTPRUNE_ERR_CUDA;
+        }
     }
     *workspace_bytes = p->ws.total;
     *plan_out = p;

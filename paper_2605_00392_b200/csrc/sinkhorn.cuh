@@ -29,8 +29,9 @@ __device__ inline void lse_merge(float &m, float &s, float m2, float s2)
 
 // LOG = true : Z_ij = S-bar_ij / eps, duals u, v in the log domain,
 //              u_i = log mu_i - LSE_j(Z_ij + v_j), v_j = log nu_j - LSE_i(Z_ij + u_i).
-// LOG = false: K_ij = exp((S-bar_ij - c)/eps), c = max(1, z); duals carried as U = e^u, V = e^v
-//              (up to the constant e^{c/eps}, which cancels in the plan):
+// LOG = false: K_ij = exp((S-bar_ij - c)/eps), c = max(1, z); duals carried as U = e^u and
+//              V = e^{v + c/eps} (V starts at e^{c/eps}, i.e. v = 0), so that U K V = exp(Z + u + v)
+//              after any number of iterations, zero included:
 //              U_i = mu_i / sum_j K_ij V_j, V_j = nu_j / sum_i K_ij U_i.
 // mu = [1_M, B], nu = [1_B, M].  Plan: P_ij = U_i K_ij V_j  (= exp(Z_ij + u_i + v_j)).
 template <bool LOG>
@@ -63,7 +64,8 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     const bool in_smem = (long long)R * lds + (R + Cc + part_floats) <= (long long)smem_floats;
     float *Kg = kmat + kmat_offset(kmat_stride, t_begin, img);
     float *Kp = in_smem ? Ks : Kg;
-    const int ld = in_smem ? lds : Cc;
+    const int ldg = score_pitch(B);             // pitch of the workspace tile
+    const int ld = in_smem ? lds : ldg;
 
     const float inv_eps = 1.f / p.eps;
     const float shift = fmaxf(1.f, p.z);
@@ -71,12 +73,12 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     // build Z or K from the raw cosines (dustbin row and column = z, Eq. 5)
     for (int idx = tid; idx < R * Cc; idx += nth) {
         const int i = idx / Cc, j = idx - i * Cc;
-        const float s = (i < M && j < B) ? Kg[(size_t)i * Cc + j] : p.z;
+        const float s = (i < M && j < B) ? Kg[(size_t)i * ldg + j] : p.z;
         Kp[(size_t)i * ld + j] = LOG ? s * inv_eps : expf((s - shift) * inv_eps);
     }
-    const float init = LOG ? 0.f : 1.f;
-    for (int i = tid; i < R; i += nth) u[i] = init;
-    for (int j = tid; j < Cc; j += nth) v[j] = init;
+    const float v_init = LOG ? 0.f : expf(shift * inv_eps);
+    for (int i = tid; i < R; i += nth) u[i] = LOG ? 0.f : 1.f;
+    for (int j = tid; j < Cc; j += nth) v[j] = v_init;
     __syncthreads();
 
     const float mu_last = LOG ? logf((float)B) : (float)B;
@@ -235,11 +237,11 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     }
     __syncthreads();
 
-    // ---- plan P (non-dustbin block), written to the workspace tile with row stride B+1 --------
+    // ---- plan P (non-dustbin block), written to the workspace tile (row pitch score_pitch(B)) --
     for (int idx = tid; idx < M * B; idx += nth) {
         const int i = idx / B, j = idx - i * B;
         const float k = Kp[(size_t)i * ld + j];
-        Kg[(size_t)i * Cc + j] = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
+        Kg[(size_t)i * ldg + j] = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
     }
 }
 

@@ -89,7 +89,8 @@ norm_stats_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, 
 // Kernel (a2)-(a4): one CTA per image, 1024 threads.
 //   phi from the chunk partials; r and B = floor(r N + 1/2) clamped to [0, N-1], M = N - B;
 //   rank of every token under (norm descending, index ascending) by counting; the M best are
-//   T_kept.  Writes order[] = kept indices ascending, then pruned indices ascending; counts, stats;
+//   T_kept.  Writes order[] = kept indices ascending, then pruned indices ascending, and its
+//   inverse kpos[]; counts, stats;
 //   the last CTA to finish turns counts into out_offsets (exclusive prefix sum).
 // Shared memory: float keys[max_tokens] (dynamic) + static scratch.
 // ---------------------------------------------------------------------------------------------
@@ -102,7 +103,7 @@ __global__ void __launch_bounds__(1024)
 select_kernel(const int32_t *__restrict__ offsets, int batch, int d, int chunks, int max_tokens,
               int total, RatioParams rp, const float *__restrict__ rho, const float *__restrict__ norms,
               const float *__restrict__ spart, int32_t *__restrict__ order,
-              int32_t *__restrict__ counts, int32_t *__restrict__ out_offsets,
+              int32_t *__restrict__ kpos, int32_t *__restrict__ counts, int32_t *__restrict__ out_offsets,
               float *__restrict__ stats, float *__restrict__ norms_out,
               int32_t *__restrict__ order_out, WsHeader *__restrict__ hdr)
 {
@@ -201,14 +202,15 @@ select_kernel(const int32_t *__restrict__ offsets, int batch, int d, int chunks,
             s_redi[lane] = wi - w;
         }
         __syncthreads();
-        int kpos = s_redi[warp] + incl - nkept;  // kept tokens before k0
+        int kpos_run = s_redi[warp] + incl - nkept;  // kept tokens before k0
         int32_t *ord = order + t_begin;
         for (int k = k0; k < k1; ++k) {
             const bool kept = (keptmask >> (k - k0)) & 1u;
-            const int pos = kept ? kpos : (M + (k - kpos));
+            const int pos = kept ? kpos_run : (M + (k - kpos_run));
             ord[pos] = k;
+            kpos[t_begin + k] = kept ? kpos_run : -1 - (k - kpos_run);
             if (order_out) order_out[t_begin + pos] = k;
-            kpos += kept ? 1 : 0;
+            kpos_run += kept ? 1 : 0;
         }
     } else if (tid == 0) {
         atomicOr(&hdr->status, RTPRUNE_DEV_BAD_OFFSETS);  // offsets broke the contract: the image yields no output

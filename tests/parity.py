@@ -4,8 +4,9 @@ same seeded inputs, and compare element by element.
 Tolerances (stated once, used by every parity test):
   * counts, out_offsets, kept_idx, merged_idx: bit-exact.
   * merge_partner: bit-exact where the oracle's top-2 gap of log P over the kept tokens is at least
-    PARTNER_GAP (1e-3); below that several answers are correct to working precision, and the GPU's
-    choice must lie in the oracle's within-gap candidate set.
+    PARTNER_GAP (1e-3); below that several answers are correct to working precision (near-duplicate
+    background tokens make most columns of the document batches such near-ties), so in addition
+    EVERY chosen partner must reach the oracle's column maximum of log P to within PARTNER_REGRET.
   * merged features Y: |y - y*| <= tol * max(|y*|, rms(y* row)) with tol = 1e-2 for bf16 storage
     (fp32 accumulation) and 1e-5 for fp32 storage; y* is the oracle's fp64 value.
   * phi: 2e-5 absolute (fp32 sum of ~N unit vectors); r: 1e-5; plan weights: 1e-4 relative.
@@ -25,6 +26,7 @@ from oracle import oracle
 from paper_2605_00392_b200 import binding, synth
 
 PARTNER_GAP = 1e-3
+PARTNER_REGRET = 5e-5      # every chosen partner's log P must be this close to the column maximum
 FEATURE_TOL = {torch.bfloat16: 1e-2, torch.float32: 1e-5}
 ROUND_MARGIN = 1e-3
 
@@ -142,11 +144,14 @@ def compare_image(w: synth.Workload, i: int, ref: oracle.ImageResult, g: binding
     np.testing.assert_array_equal(gp[decisive], ref.partner[decisive], err_msg=tag)
     report["pairs"] = report.get("pairs", 0) + ref.B
     report["pairs_within_gap"] = report.get("pairs_within_gap", 0) + int((~decisive).sum())
-    if (~decisive).any():
-        assert ref.Pbar is not None, "oracle must be run with want_plan for near-tie columns"
+    if ref.Pbar is not None:
+        # stronger than the masked rule: whatever the gap, the GPU's choice must be a maximiser of
+        # the oracle's plan column to within PARTNER_REGRET (fp32 working precision with margin)
         logP = np.log(ref.Pbar[:-1, :-1])
-        for j in np.nonzero(~decisive)[0]:
-            assert 0 <= gp[j] < ref.M and logP[gp[j], j] >= logP[:, j].max() - PARTNER_GAP, (tag, j)
+        assert np.all((gp >= 0) & (gp < ref.M)), tag
+        regret = logP.max(axis=0) - logP[gp, np.arange(ref.B)]
+        report["max_partner_regret"] = max(report.get("max_partner_regret", 0.0), float(regret.max()))
+        assert regret.max() <= PARTNER_REGRET, (tag, float(regret.max()))
     same = gp == ref.partner
     np.testing.assert_allclose(gw[same], ref.weight[same], rtol=1e-4, err_msg=tag)
     assert st[5] >= 1 or w.params.get("iters", 100) == 0, tag
