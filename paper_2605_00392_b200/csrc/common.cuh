@@ -28,6 +28,8 @@ struct WsLayout {
     size_t kpos;       // int32 [total]            per token: position among kept, or -1 - position
                        //                          among pruned
     size_t kmat;       // float [kmat_floats]      per-image score / kernel / plan matrix
+    size_t pbuf;       // bf16 [total][pbuf_pitch] plan rows for the tensor-core merge (bf16 mode)
+    int pbuf_pitch_max;  // elements; a run uses round_up(its largest possible B, 64) <= this
     size_t total;      // bytes
     int chunks;        // chunks per image = ceil(max_tokens_per_image / kChunkTokens)
     int kmat_stride;   // floats of kmat per token-unit, see kmat_offset()

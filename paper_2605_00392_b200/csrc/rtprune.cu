@@ -1,5 +1,6 @@
 // C ABI of the RTPrune pruning path: plan, argument checks, workspace layout and kernel launches.
 // Every step of the path runs in the kernels included below; this file only marshals.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -8,6 +9,7 @@
 
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "merge_umma.cuh"
 #include "scores_umma.cuh"
 #include "sinkhorn.cuh"
 #include "stage1.cuh"
@@ -40,7 +42,7 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-WsLayout make_layout(int d, int max_batch, int64_t max_total, int max_tokens)
+WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_total, int max_tokens)
 {
     WsLayout L;
     L.chunks = (max_tokens + kChunkTokens - 1) / kChunkTokens;
@@ -58,6 +60,10 @@ WsLayout make_layout(int d, int max_batch, int64_t max_total, int max_tokens)
     off = align_up(off + sizeof(int32_t) * (size_t)max_total, 256);
     L.kmat = off;
     off = align_up(off + sizeof(float) * (size_t)L.kmat_stride * (size_t)(max_total + 8 * (int64_t)max_batch), 256);
+    L.pbuf = off;
+    L.pbuf_pitch_max = (max_tokens + 63) / 64 * 64;
+    if (dtype == RTPRUNE_BF16)
+        off = align_up(off + sizeof(__nv_bfloat16) * (size_t)max_total * L.pbuf_pitch_max, 256);
     L.total = off;
     return L;
 }
@@ -247,6 +253,9 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     const int maxN = plan->max_tokens;
     const int maxB = max_pruned(params, maxN);
     const int mtiles = (maxN + kSimtTile - 1) / kSimtTile;
+    constexpr bool kTensor = std::is_same<T, __nv_bfloat16>::value;
+    __nv_bfloat16 *pbuf = kTensor ? (__nv_bfloat16 *)(ws + L.pbuf) : nullptr;
+    const int pbuf_pitch = (std::max(maxB, 1) + 63) / 64 * 64;   // <= L.pbuf_pitch_max
 
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
@@ -276,20 +285,33 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
-                smem_floats, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
+                smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
+                o.stats);
         else
             sinkhorn_kernel<false><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
-                smem_floats, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
+                smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
+                o.stats);
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
         launched(plan, st, "sinkhorn");
     }
 
-    const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
-    dim3 grid(mtiles * dtiles, batch);
-    merge_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, dtiles, o.counts,
-                                              o.out_offsets, order, kmat, L.kmat_stride, maxN,
-                                              total, params->alpha, (T *)o.Y, o.kept_idx);
+    if constexpr (kTensor) {
+        CUtensorMap tmapP;
+        if (!make_tmap_bf16(plan, &tmapP, pbuf, (uint64_t)total, (uint64_t)pbuf_pitch,
+                            (uint64_t)pbuf_pitch * 2, kMgBK, kMgTileM))
+            return RTPRUNE_ERR_CUDA;
+        dim3 grid((maxN + kMgTileM - 1) / kMgTileM, batch);
+        merge_umma_kernel<<<grid, kMgThreads, kMgSmemBytes, st>>>(
+            tmapP, (const __nv_bfloat16 *)X, offsets, plan->d, o.counts, o.out_offsets, order, maxN,
+            total, params->alpha, (__nv_bfloat16 *)o.Y, o.kept_idx, (WsHeader *)(ws + L.header));
+    } else {
+        const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
+        dim3 grid(mtiles * dtiles, batch);
+        merge_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)X, offsets, plan->d, dtiles, o.counts,
+                                                  o.out_offsets, order, kmat, L.kmat_stride, maxN,
+                                                  total, params->alpha, (T *)o.Y, o.kept_idx);
+    }
     if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
     launched(plan, st, "merge");
     return RTPRUNE_OK;
@@ -393,7 +415,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     p->max_batch = max_batch;
     p->max_total = max_total_tokens;
     p->max_tokens = max_tokens_per_image;
-    p->ws = make_layout(d, max_batch, max_total_tokens, max_tokens_per_image);
+    p->ws = make_layout(d, dtype, max_batch, max_total_tokens, max_tokens_per_image);
     p->last_launches = 0;
     p->last_cuda_error = 0;
     p->profiling = false;
@@ -438,7 +460,9 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     if (dtype == RTPRUNE_BF16) {
         if (!p->encode_tiled ||
             !c.ok(cudaFuncSetAttribute(scores_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kScSmemBytes))) {
+                                       kScSmemBytes)) ||
+            !c.ok(cudaFuncSetAttribute(merge_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kMgSmemBytes))) {
             if (!p->last_cuda_error) p->last_cuda_error = (int)cudaErrorNotSupported;
             delete p;
             return RTPRUNE_ERR_CUDA;

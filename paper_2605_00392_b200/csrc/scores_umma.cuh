@@ -10,7 +10,8 @@
 //   * D: 128 TMEM lanes x BN columns (BN = B rounded up to 16, at most 256 per pass).
 // Warp roles (192 threads): warps 0-3 gather B, then run the epilogue (TMEM -> registers -> divide by
 // the two norms -> global); warp 4 lane 0 issues the TMA loads; warp 5 owns TMEM and lane 0 issues
-// the UMMAs.  A 4-stage ring of shared-memory buffers is handed over with mbarriers.
+// the UMMAs.  A ring of shared-memory stages (as many as fit: 8 for B <= 64, 4 for B = 256) is handed
+// over with mbarriers; the gather keeps kScLag stages of copies in flight per thread.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -19,21 +20,22 @@ namespace rtp {
 
 constexpr int kScTileM = 128;
 constexpr int kScBK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int kScStages = 4;
+constexpr int kScMaxStages = 8;
+constexpr int kScLag = 3;            // stages of gather copies in flight per thread (< stages)
 constexpr int kScBNMax = 256;
 constexpr int kScThreads = 192;
 constexpr int kScABytes = kScTileM * 128;    // 16 KB
-constexpr int kScBBytes = kScBNMax * 128;    // 32 KB
-constexpr int kScStageBytes = kScABytes + kScBBytes;
-constexpr int kScSmemBytes = kScStages * kScStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int kScRingBytes = 4 * (kScABytes + kScBNMax * 128);   // 192 KB of stage buffers
+constexpr int kScSmemBytes = kScRingBytes + 1024 /*alignment*/ + 2048 /*barriers, norms*/;
 
 struct ScoresBarriers {
-    uint64_t full[kScStages];
-    uint64_t empty[kScStages];
+    uint64_t full[kScMaxStages];
+    uint64_t empty[kScMaxStages];
     uint64_t accum_full;
     uint64_t tmem_empty;
     uint32_t tmem_base;
     volatile int abort_flag;
+    float inv_nj[kScBNMax];          // 1 / |x_j| of the first pass's pruned tokens
 };
 
 __global__ void __launch_bounds__(kScThreads, 1)
@@ -51,14 +53,17 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
     if (B == 0 || mt * kScTileM >= N) return;
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    ScoresBarriers *bars = reinterpret_cast<ScoresBarriers *>(smem + kScStages * kScStageBytes);
+    ScoresBarriers *bars = reinterpret_cast<ScoresBarriers *>(smem + kScRingBytes);
+    // stage = A tile + this image's B tile; as many stages as fit in the ring
+    const int stage_bytes = kScABytes + min(kScBNMax, (B + 15) & ~15) * 128;
+    const int kScStages = min(kScMaxStages, kScRingBytes / stage_bytes);   // 4 .. 8
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nkb = (d + kScBK - 1) / kScBK;
     const int nbt = (B + kScBNMax - 1) / kScBNMax;
     const int32_t *ord = order + t_begin;
 
     if (tid == 0) {
-        for (int s = 0; s < kScStages; ++s) {
+        for (int s = 0; s < kScMaxStages; ++s) {
             ptx::mbar_init(&bars->full[s], 1 + 128);
             ptx::mbar_init(&bars->empty[s], 1);
         }
@@ -92,7 +97,7 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
                         break;
                     }
                     ptx::mbar_arrive_expect_tx(&bars->full[s], kScABytes);
-                    ptx::tma_load_2d(smem_base + s * kScStageBytes, &tmapX, &bars->full[s], kb * kScBK,
+                    ptx::tma_load_2d(smem_base + s * stage_bytes, &tmapX, &bars->full[s], kb * kScBK,
                                      t_begin + mt * kScTileM);
                 }
             }
@@ -120,7 +125,7 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
                         break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t a_base = smem_base + s * kScStageBytes;
+                    const uint32_t a_base = smem_base + s * stage_bytes;
                     const uint32_t b_base = a_base + kScABytes;
 #pragma unroll
                     for (int k = 0; k < kScBK / 16; ++k) {
@@ -137,15 +142,19 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
         // ---------------- warps 0-3: gather B, then epilogue ------------------------------------
         const int c = tid & 7, rbase = tid >> 3;
         uint32_t it = 0;
-        int prev_s = -1;
         float *Simg = kmat + kmat_offset(kmat_stride, t_begin, img);
         const int ldS = score_pitch(B);
         const int row = tid;                       // TMEM lane = tile row
         const int k_tok = mt * kScTileM + row;
         const int p = (k_tok < N) ? kpos[t_begin + k_tok] : -1;
-        const float ni = (p >= 0) ? fmaxf(norms[t_begin + k_tok], kNormFloor) : 1.f;
+        const float inv_ni = (p >= 0) ? 1.f / fmaxf(norms[t_begin + k_tok], kNormFloor) : 1.f;
+        // 1/|x_j| of the first pass's columns, shared by the 128 epilogue threads.  The barrier is
+        // reached unconditionally: nothing can have failed yet.
+        for (int j = tid; j < min(B, kScBNMax); j += 128)
+            bars->inv_nj[j] = 1.f / fmaxf(norms[t_begin + ord[M + j]], kNormFloor);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         for (int bt = 0; bt < nbt; ++bt) {
-            if (__any_sync(0xffffffffu, bars->abort_flag != 0)) break;  // warp-uniform exit
+            if (bt > 0 && __any_sync(0xffffffffu, bars->abort_flag != 0)) break;  // warp-uniform
             const int j0 = bt * kScBNMax;
             const int BN = min(kScBNMax, (B - j0 + 15) & ~15);
             int tok[kScBNMax / 16];
@@ -155,6 +164,7 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
                 tok[q] = (16 * q < BN && j < B) ? t_begin + ord[M + j] : -1;
             }
             bool failed = false;
+            const uint32_t it0 = it;
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % kScStages;
                 if (it >= (uint32_t)kScStages &&
@@ -162,7 +172,7 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
                     failed = true;
                     break;
                 }
-                const uint32_t b_base = smem_base + s * kScStageBytes + kScABytes;
+                const uint32_t b_base = smem_base + s * stage_bytes + kScABytes;
                 const int kcol = kb * kScBK + c * 8;
 #pragma unroll
                 for (int q = 0; q < kScBNMax / 16; ++q) {
@@ -175,18 +185,17 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
                     }
                 }
                 ptx::cp_async_commit();
-                if (prev_s >= 0) {
-                    ptx::cp_async_wait<1>();
+                if (kb >= kScLag) {     // the copies issued kScLag k-blocks ago have landed
+                    ptx::cp_async_wait<kScLag>();
                     ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(&bars->full[prev_s]);
+                    ptx::mbar_arrive(&bars->full[(it - kScLag) % kScStages]);
                 }
-                prev_s = s;
             }
             ptx::cp_async_wait<0>();
-            if (prev_s >= 0 && !failed) {
+            if (!failed) {
                 ptx::fence_proxy_async_smem();
-                ptx::mbar_arrive(&bars->full[prev_s]);
-                prev_s = -1;
+                for (uint32_t q = (it - it0 > (uint32_t)kScLag ? it - kScLag : it0); q < it; ++q)
+                    ptx::mbar_arrive(&bars->full[q % kScStages]);
             }
             // the TMEM loads below are warp-collective: take the go / no-go decision per warp
             bool ok = !__any_sync(0xffffffffu, failed);
@@ -210,8 +219,10 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __nv_bfloat1
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 const int je = min(j + e, B - 1);
-                                const float nj = fmaxf(__ldg(norms + t_begin + ord[M + je]), kNormFloor);
-                                o[e] = __uint_as_float(r[4 * g + e]) / (ni * nj);
+                                const float inv_nj =
+                                    (bt == 0) ? bars->inv_nj[je]
+                                              : 1.f / fmaxf(__ldg(norms + t_begin + ord[M + je]), kNormFloor);
+                                o[e] = __uint_as_float(r[4 * g + e]) * inv_ni * inv_nj;
                             }
                             *reinterpret_cast<float4 *>(Simg + (size_t)p * ldS + j) =
                                 make_float4(o[0], o[1], o[2], o[3]);

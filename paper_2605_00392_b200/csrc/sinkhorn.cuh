@@ -39,7 +39,8 @@ __global__ void __launch_bounds__(kSinkThreads)
 sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__ counts,
                 const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ order,
                 float *__restrict__ kmat, int kmat_stride, int max_tokens, int total, OtParams p,
-                int smem_floats, int32_t *__restrict__ merged_idx,
+                int smem_floats, __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch,
+                int32_t *__restrict__ merged_idx,
                 int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
                 float *__restrict__ stats)
 {
@@ -237,11 +238,28 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     }
     __syncthreads();
 
-    // ---- plan P (non-dustbin block), written to the workspace tile (row pitch score_pitch(B)) --
-    for (int idx = tid; idx < M * B; idx += nth) {
-        const int i = idx / B, j = idx - i * B;
-        const float k = Kp[(size_t)i * ld + j];
-        Kg[(size_t)i * ldg + j] = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
+    // ---- plan P (non-dustbin block) ---------------------------------------------------------------
+    if (pbuf) {
+        // bf16 rows for the tensor-core merge: row = packed output row, columns padded with zeros to
+        // the next multiple of 64 (the contraction runs over whole 64-column blocks)
+        const int kpad = (B + 63) & ~63;
+        __nv_bfloat16 *Pimg = pbuf + (size_t)out_offsets[img] * pbuf_pitch;
+        for (int idx = tid; idx < M * kpad; idx += nth) {
+            const int i = idx / kpad, j = idx - i * kpad;
+            float pv = 0.f;
+            if (j < B) {
+                const float k = Kp[(size_t)i * ld + j];
+                pv = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
+            }
+            Pimg[(size_t)i * pbuf_pitch + j] = __float2bfloat16_rn(pv);
+        }
+    } else {
+        // fp32, in place in the workspace tile (row pitch score_pitch(B))
+        for (int idx = tid; idx < M * B; idx += nth) {
+            const int i = idx / B, j = idx - i * B;
+            const float k = Kp[(size_t)i * ld + j];
+            Kg[(size_t)i * ldg + j] = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
+        }
     }
 }
 
