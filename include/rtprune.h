@@ -157,6 +157,36 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
                                 float *stats, float *norms_out, int32_t *order_out);
 
 /*
+ * Stage 1 for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * convenience of the library).  Some hosts of this code own no allocator at the point where they
+ * call it: a plug-in running inside another framework's memory pool that must not be disturbed, a
+ * real-time loop in which cudaMalloc's implicit synchronisation is forbidden, a process whose
+ * memory budget was fixed at start-up.  For them this entry point does what rtprune_select does,
+ * with the same arguments minus the workspace: its scratch is a fixed array of
+ * RTPRUNE_STATIC_SCRATCH_BYTES that is part of the library's device image (every GPU that loads the
+ * library holds it until the process exits).  It calls no cudaMalloc / cudaFree and no allocating
+ * library routine; inputs and outputs are still the caller's buffers.
+ *
+ *   - Limit: the plan's stage-1 scratch (norms, unit-token partial sums, selection lists; it grows
+ *     with max_total_tokens and with max_batch * max_tokens_per_image * d) must fit the array, else
+ *     RTPRUNE_ERR_WORKSPACE is returned and nothing is launched.  A 64-image x 400-token x 1280
+ *     plan needs about 2.6 MiB.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - Every call on a device shares the one array, which keeps the previous call's contents; the
+ *     call clears the words that must start at zero itself.  Two calls that overlap on the same
+ *     GPU (different streams, or threads) race on it: serialise them.
+ *   - The device status word lives in the array too and cannot be read with rtprune_query_status;
+ *     a batch that breaks the offsets contract yields counts of 0 for the offending image.
+ */
+#define RTPRUNE_STATIC_SCRATCH_BYTES (4u << 20)
+rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
+                                       const int32_t *offsets, int32_t batch, int64_t total_tokens,
+                                       const rtprune_params_t *params, int32_t *out_offsets,
+                                       int32_t *counts, float *stats, float *norms_out,
+                                       int32_t *order_out);
+
+/*
  * The same run, from and to HOST buffers (pinned memory recommended): copies X, offsets and rho to
  * the device arena, runs, and copies every output back, all asynchronously on the stream; the
  * caller synchronises the stream before reading.  `rho_host` may be NULL (params->rho is ignored

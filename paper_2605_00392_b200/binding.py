@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
     L.rtprune_run.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp]
     L.rtprune_workspace_init.argtypes = [vp, vp, vp, sz]
     L.rtprune_select.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, sz, vp, vp, vp, vp, vp]
+    L.rtprune_select_static.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, vp, vp, vp, vp]
     L.rtprune_run_host.argtypes = [vp, vp, vp, vp, vp, i32, i64, pp, vp, sz,
                                    vp, vp, vp, vp, vp, vp, vp, vp]
     L.rtprune_host_arena_bytes.argtypes = [vp, ctypes.POINTER(sz)]
@@ -191,6 +192,20 @@ class Plan:
                                     out.out_offsets.data_ptr(), out.counts.data_ptr(),
                                     out.stats.data_ptr(), _ptr(norms_out), _ptr(order_out)),
                "rtprune_select")
+
+    # -- rtprune_select_static
+    def select_static(self, X: torch.Tensor, offsets: torch.Tensor, params: CParams, out: Outputs,
+                      norms_out: Optional[torch.Tensor] = None,
+                      order_out: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Stage 1 on the library's built-in scratch array: nothing is allocated by the call."""
+        batch = offsets.numel() - 1
+        _check(lib().rtprune_select_static(self.handle, _stream_handle(stream), X.data_ptr(),
+                                           offsets.data_ptr(), batch, X.shape[0],
+                                           ctypes.byref(params), out.out_offsets.data_ptr(),
+                                           out.counts.data_ptr(), out.stats.data_ptr(),
+                                           _ptr(norms_out), _ptr(order_out)),
+               "rtprune_select_static")
 
     # -- rtprune_host_arena_bytes / rtprune_run_host
     def host_arena_bytes(self) -> int:

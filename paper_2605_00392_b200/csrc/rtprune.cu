@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 
@@ -38,7 +39,16 @@ struct rtprune_plan_s {
     int ev_count;  // kernels recorded by the most recent run
 };
 
+// Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[RTPRUNE_STATIC_SCRATCH_BYTES];
+
 namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_scratch_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -526,6 +536,53 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
     prof_begin(plan, (cudaStream_t)cuda_stream);
     return launch_stage1(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
                          (char *)workspace, out_offsets, counts, stats, norms_out, order_out);
+}
+
+rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
+                                       const int32_t *offsets, int32_t batch, int64_t total_tokens,
+                                       const rtprune_params_t *params, int32_t *out_offsets,
+                                       int32_t *counts, float *stats, float *norms_out,
+                                       int32_t *order_out)
+{
+    if (!plan || !params) return RTPRUNE_ERR_INVALID_ARG;
+    if (batch < 0 || total_tokens < 0 || batch > plan->max_batch || total_tokens > plan->max_total ||
+        total_tokens < batch)
+        return RTPRUNE_ERR_INVALID_ARG;
+    if (batch > 0 && (!X || !offsets)) return RTPRUNE_ERR_INVALID_ARG;
+    if ((uintptr_t)X & 15u) return RTPRUNE_ERR_INVALID_ARG;
+    if (!out_offsets || (batch > 0 && (!counts || !stats))) return RTPRUNE_ERR_INVALID_ARG;
+    // Stage 1 uses the workspace regions that precede the score tiles; they must fit the array.
+    if (plan->ws.kmat > (size_t)RTPRUNE_STATIC_SCRATCH_BYTES) return RTPRUNE_ERR_WORKSPACE;
+    rtprune_status_t s = check_params(params);
+    if (s != RTPRUNE_OK) return s;
+
+    Checked c{plan};
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    if (!c.ok(cudaGetDevice(&dev))) return RTPRUNE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return RTPRUNE_ERR_UNSUPPORTED;
+    char *scratch = nullptr;
+    {
+        // first call on this device: ask the runtime where this device keeps the array
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_scratch_addr[dev]) {
+            void *p = nullptr;
+            if (!c.ok(cudaGetSymbolAddress(&p, g_static_scratch)) || !p) return RTPRUNE_ERR_CUDA;
+            g_static_scratch_addr[dev] = p;
+        }
+        scratch = (char *)g_static_scratch_addr[dev];
+    }
+    plan->last_launches = 0;
+    if (batch == 0) {
+        if (!c.ok(cudaMemsetAsync(out_offsets, 0, sizeof(int32_t), st))) return RTPRUNE_ERR_CUDA;
+        return RTPRUNE_OK;
+    }
+    // the array keeps whatever the last call left: the status word and the counters must start at 0
+    if (!c.ok(cudaMemsetAsync(scratch + plan->ws.header, 0, sizeof(WsHeader), st)))
+        return RTPRUNE_ERR_CUDA;
+    prof_begin(plan, st);
+    return launch_stage1(plan, st, X, offsets, batch, (int)total_tokens, params, scratch, out_offsets,
+                         counts, stats, norms_out, order_out);
 }
 
 rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)
