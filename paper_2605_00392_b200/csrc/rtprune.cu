@@ -13,6 +13,7 @@
 #include "merge_umma.cuh"
 #include "scores_umma.cuh"
 #include "sinkhorn.cuh"
+#include "sinkhorn_fast.cuh"
 #include "stage1.cuh"
 
 using namespace rtp;
@@ -29,7 +30,8 @@ struct rtprune_plan_s {
     int device;
     int sm_count;
     int smem_optin;       // bytes of opt-in shared memory per CTA
-    int sink_smem_bytes;  // dynamic shared memory of the Sinkhorn kernel
+    int sink_smem_bytes;  // dynamic shared memory of the general Sinkhorn kernel
+    int fast_smem_bytes;  // dynamic shared memory of the one-pass Sinkhorn kernel
     void *encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
     int last_launches;
     int last_cuda_error;
@@ -292,18 +294,34 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         OtParams op{params->z, params->alpha, params->eps, params->iters,
                     params->stop_at_fixed_point, params->tol};
         const int smem_floats = plan->sink_smem_bytes / (int)sizeof(float);
+        // Scaling form: tiles that fit one CTA's shared memory go to the one-pass kernel; the general
+        // kernel then takes what is left (it skips the images already solved).
+        int fast_nc = 0;
+        const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
+        bool all_fast = false;
+        if (!use_log_form(params)) {
+            fast_nc = kSfMaxNc;
+            all_fast = maxB <= 32 * fast_nc;
+            for (int b = 1; b <= maxB && all_fast; ++b)
+                all_fast = sinkhorn_fast_fits(std::max(maxN - b, 1), b, fast_nc, fast_floats);
+            sinkhorn_fast_kernel<<<batch, kSfThreads, plan->fast_smem_bytes, st>>>(
+                offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op, fast_floats,
+                pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
+            if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "sinkhorn_fast");
+        }
         if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                o.stats);
-        else
+                o.stats, 0, 0);
+        else if (!all_fast)
             sinkhorn_kernel<false><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                o.stats);
+                o.stats, fast_nc, fast_floats);
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
-        launched(plan, st, "sinkhorn");
+        if (use_log_form(params) || !all_fast) launched(plan, st, "sinkhorn");
     }
 
     if constexpr (kTensor) {
@@ -454,6 +472,12 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
                                    p->sink_smem_bytes)) ||
         !c.ok(cudaFuncSetAttribute(sinkhorn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    p->sink_smem_bytes))) {
+        delete p;
+        return RTPRUNE_ERR_CUDA;
+    }
+    p->fast_smem_bytes = (int)(cap / 16 * 16);
+    if (!c.ok(cudaFuncSetAttribute(sinkhorn_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   p->fast_smem_bytes))) {
         delete p;
         return RTPRUNE_ERR_CUDA;
     }
