@@ -28,6 +28,9 @@ struct WsLayout {
     size_t kpos;       // int32 [total]            per token: position among kept, or -1 - position
                        //                          among pruned
     size_t kmat;       // float [kmat_floats]      per-image score / kernel / plan matrix
+    size_t xp;         // bf16 [total + 64 batch][d] compact copy of the pruned tokens (bf16 mode): image
+                       //                          i's B rows start at row xp_row0(offsets[i], i), followed
+                       //                          by zero rows up to a multiple of 64
     size_t pbuf;       // bf16 [total][pbuf_pitch] plan rows for the tensor-core merge (bf16 mode)
     int pbuf_pitch_max;  // elements; a run uses round_up(its largest possible B, 64) <= this
     size_t total;      // bytes
@@ -46,6 +49,10 @@ __host__ __device__ inline size_t kmat_offset(int kmat_stride, int tok_offset, i
 {
     return (size_t)kmat_stride * (size_t)(tok_offset + 8 * img);
 }
+
+// First row of image `img`'s segment in the compact copy of pruned tokens.  Each image owns
+// N + 64 rows there, enough for its B <= N - 1 rows rounded up to a multiple of 64.
+__host__ __device__ inline int xp_row0(int tok_offset, int img) { return tok_offset + 64 * img; }
 
 // Reads image `img`'s token range and checks it against the contract (1 <= N <= max_tokens, rows
 // inside [0, total)).  Kernels skip an image that fails; the selection kernel reports it.

@@ -72,6 +72,9 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(int32_t) * (size_t)max_total, 256);
     L.kmat = off;
     off = align_up(off + sizeof(float) * (size_t)L.kmat_stride * (size_t)(max_total + 8 * (int64_t)max_batch), 256);
+    L.xp = off;
+    if (dtype == RTPRUNE_BF16)
+        off = align_up(off + sizeof(__nv_bfloat16) * (size_t)(max_total + 64 * (int64_t)max_batch) * d, 256);
     L.pbuf = off;
     L.pbuf_pitch_max = (max_tokens + 63) / 64 * 64;
     if (dtype == RTPRUNE_BF16)
@@ -228,7 +231,7 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
                                const int32_t *offsets, int32_t batch, int total,
                                const rtprune_params_t *params, char *ws, int32_t *out_offsets,
                                int32_t *counts, float *stats, float *norms_out,
-                               int32_t *order_out)
+                               int32_t *order_out, bool with_xp)
 {
     Checked c{plan};
     const WsLayout &L = plan->ws;
@@ -244,9 +247,12 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
     launched(plan, st, "norm_stats");
     RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
     const size_t smem = sizeof(float) * (size_t)plan->max_tokens;
+    const bool bf16 = with_xp && plan->dtype == RTPRUNE_BF16;   // the compact copy of T_prop feeds stage 2 only
     select_kernel<<<batch, 1024, smem, st>>>(offsets, batch, plan->d, L.chunks, plan->max_tokens,
                                              total, rp, params->rho, norms, spart, order, kpos, counts,
-                                             out_offsets, stats, norms_out, order_out, hdr);
+                                             out_offsets, stats, norms_out, order_out, hdr,
+                                             bf16 ? (const __nv_bfloat16 *)X : nullptr,
+                                             bf16 ? (__nv_bfloat16 *)(ws + L.xp) : nullptr);
     if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
     launched(plan, st, "select");
     return RTPRUNE_OK;
@@ -272,15 +278,16 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
             // tensor-core path: one CTA per (128 consecutive tokens, image)
-            CUtensorMap tmapX;
+            CUtensorMap tmapX, tmapXp;
             if (!make_tmap_bf16(plan, &tmapX, X, (uint64_t)total, (uint64_t)plan->d,
-                                (uint64_t)plan->d * 2, kScBK, kScTileM))
+                                (uint64_t)plan->d * 2, kScBK, kScTileM) ||
+                !make_tmap_bf16(plan, &tmapXp, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
+                                (uint64_t)plan->d * 2, kScBK, kScBBoxRows))
                 return RTPRUNE_ERR_CUDA;
             dim3 grid((maxN + kScTileM - 1) / kScTileM, batch);
             scores_umma_kernel<<<grid, kScThreads, kScSmemBytes, st>>>(
-                tmapX, (const __nv_bfloat16 *)X, offsets, plan->d, o.counts, order,
-                (const int32_t *)(ws + L.kpos), norms, kmat, L.kmat_stride, maxN, total,
-                (WsHeader *)(ws + L.header));
+                tmapX, tmapXp, offsets, plan->d, o.counts, order, (const int32_t *)(ws + L.kpos), norms,
+                kmat, L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header));
         } else {
             const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
             dim3 grid(mtiles * btiles, batch);
@@ -356,7 +363,7 @@ rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X
     }
     prof_begin(plan, st);
     rtprune_status_t s = launch_stage1(plan, st, X, offsets, batch, total, params, ws, o.out_offsets,
-                                       o.counts, o.stats, nullptr, nullptr);
+                                       o.counts, o.stats, nullptr, nullptr, true);
     if (s != RTPRUNE_OK) return s;
     return (plan->dtype == RTPRUNE_BF16)
                ? launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o)
@@ -559,7 +566,7 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
     }
     prof_begin(plan, (cudaStream_t)cuda_stream);
     return launch_stage1(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
-                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out);
+                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out, false);
 }
 
 rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
@@ -606,7 +613,7 @@ rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, 
         return RTPRUNE_ERR_CUDA;
     prof_begin(plan, st);
     return launch_stage1(plan, st, X, offsets, batch, (int)total_tokens, params, scratch, out_offsets,
-                         counts, stats, norms_out, order_out);
+                         counts, stats, norms_out, order_out, false);
 }
 
 rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)

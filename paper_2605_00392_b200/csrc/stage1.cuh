@@ -90,7 +90,7 @@ norm_stats_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, 
 //   phi from the chunk partials; r and B = floor(r N + 1/2) clamped to [0, N-1], M = N - B;
 //   rank of every token under (norm descending, index ascending) by counting; the M best are
 //   T_kept.  Writes order[] = kept indices ascending, then pruned indices ascending, and its
-//   inverse kpos[]; counts, stats;
+//   inverse kpos[]; counts, stats; for bf16 storage also the compact copy of T_prop's rows;
 //   the last CTA to finish turns counts into out_offsets (exclusive prefix sum).
 // Shared memory: float keys[max_tokens] (dynamic) + static scratch.
 // ---------------------------------------------------------------------------------------------
@@ -105,7 +105,8 @@ select_kernel(const int32_t *__restrict__ offsets, int batch, int d, int chunks,
               const float *__restrict__ spart, int32_t *__restrict__ order,
               int32_t *__restrict__ kpos, int32_t *__restrict__ counts, int32_t *__restrict__ out_offsets,
               float *__restrict__ stats, float *__restrict__ norms_out,
-              int32_t *__restrict__ order_out, WsHeader *__restrict__ hdr)
+              int32_t *__restrict__ order_out, WsHeader *__restrict__ hdr,
+              const __nv_bfloat16 *__restrict__ Xb, __nv_bfloat16 *__restrict__ xp)
 {
     extern __shared__ uint32_t s_keys[];  // norm bits: for non-negative floats the unsigned order
     __shared__ float s_redf[32];          // is the float order, and a NaN still ranks somewhere
@@ -211,6 +212,32 @@ select_kernel(const int32_t *__restrict__ offsets, int batch, int d, int chunks,
             kpos[t_begin + k] = kept ? kpos_run : -1 - (k - kpos_run);
             if (order_out) order_out[t_begin + pos] = k;
             kpos_run += kept ? 1 : 0;
+        }
+
+        // compact copy of T_prop for the tensor-core kernels (bf16 storage): a warp per row, then rows
+        // of zeros up to a multiple of 64 so that whole 64-row tiles can be fetched
+        if (xp != nullptr && M < N) {
+            __syncthreads();                      // this CTA's writes to ord[] are visible to it
+            const int B = N - M, Bpad = (B + 63) & ~63;
+            const int nvec = d >> 3;
+            uint4 *seg = reinterpret_cast<uint4 *>(xp + (size_t)xp_row0(t_begin, img) * d);
+            for (int j = warp; j < Bpad; j += (nth >> 5)) {
+                uint4 *dst = seg + (size_t)j * nvec;
+                if (j < B) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(Xb + (size_t)(t_begin + ord[M + j]) * d);
+                    for (int v0 = lane; v0 < nvec; v0 += 128) {
+                        uint4 t[4];
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+                            t[a] = (v0 + 32 * a < nvec) ? __ldg(src + v0 + 32 * a) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+                            if (v0 + 32 * a < nvec) dst[v0 + 32 * a] = t[a];
+                    }
+                } else {
+                    for (int v = lane; v < nvec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+                }
+            }
         }
     } else if (tid == 0) {
         atomicOr(&hdr->status, RTPRUNE_DEV_BAD_OFFSETS);  // offsets broke the contract: the image yields no output
