@@ -332,14 +332,23 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     }
 
     if constexpr (kTensor) {
-        CUtensorMap tmapP;
-        if (!make_tmap_bf16(plan, &tmapP, pbuf, (uint64_t)total, (uint64_t)pbuf_pitch,
+        // every operand by tiled TMA: X rows (token tiles), the compact copy of pruned rows, the plan
+        CUtensorMap tmapXm, tmapXpm, tmapP;
+        if (!make_tmap_bf16(plan, &tmapXm, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2,
+                            64, kMgBK) ||
+            !make_tmap_bf16(plan, &tmapXpm, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
+                            (uint64_t)plan->d * 2, 64, kMgBK) ||
+            !make_tmap_bf16(plan, &tmapP, pbuf, (uint64_t)total, (uint64_t)pbuf_pitch,
                             (uint64_t)pbuf_pitch * 2, kMgBK, kMgTileM))
             return RTPRUNE_ERR_CUDA;
-        dim3 grid((maxN + kMgTileM - 1) / kMgTileM, batch);
+        const int mtiles_m = (maxN + kMgTileM - 1) / kMgTileM;
+        const int nct = (plan->d + kMgTileN - 1) / kMgTileN;
+        const long long nunits = (long long)batch * mtiles_m * nct;
+        const int grid = (int)std::min<long long>(nunits, plan->sm_count);
         merge_umma_kernel<<<grid, kMgThreads, kMgSmemBytes, st>>>(
-            tmapP, (const __nv_bfloat16 *)X, offsets, plan->d, o.counts, o.out_offsets, order, maxN,
-            total, params->alpha, (__nv_bfloat16 *)o.Y, o.kept_idx, (WsHeader *)(ws + L.header));
+            tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
+            (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
+            (WsHeader *)(ws + L.header));
     } else {
         const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
         dim3 grid(mtiles * dtiles, batch);

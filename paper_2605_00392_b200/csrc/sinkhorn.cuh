@@ -258,10 +258,10 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
 
     // ---- plan P (non-dustbin block) ---------------------------------------------------------------
     if (pbuf) {
-        // bf16 rows for the tensor-core merge: row = packed output row, columns padded with zeros to
+        // alpha P in bf16 for the tensor-core merge: row = the kept token's position in X, columns padded with zeros to
         // the next multiple of 64 (the contraction runs over whole 64-column blocks)
         const int kpad = (B + 63) & ~63;
-        __nv_bfloat16 *Pimg = pbuf + (size_t)out_offsets[img] * pbuf_pitch;
+        __nv_bfloat16 *Pimg = pbuf + (size_t)t_begin * pbuf_pitch;
         for (int idx = tid; idx < M * kpad; idx += nth) {
             const int i = idx / kpad, j = idx - i * kpad;
             float pv = 0.f;
@@ -269,7 +269,7 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
                 const float k = Kp[(size_t)i * ld + j];
                 pv = LOG ? expf(k + u[i] + v[j]) : (k * u[i]) * v[j];
             }
-            Pimg[(size_t)i * pbuf_pitch + j] = __float2bfloat16_rn(pv);
+            Pimg[(size_t)ord[i] * pbuf_pitch + j] = __float2bfloat16_rn(p.alpha * pv);
         }
     } else {
         // fp32, in place in the workspace tile (row pitch score_pitch(B))

@@ -300,13 +300,14 @@ sinkhorn_fast_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
 
     // ---- plan P = U K V (non-dustbin block) ---------------------------------------------------------
     if (pbuf) {
-        // bf16 rows for the tensor-core merge: row = packed output row; columns up to the next multiple
-        // of 64 are written (zeros past B), 8 columns = 16 bytes per store
+        // alpha P in bf16 for the tensor-core merge: row = the kept token's position in X; columns up to
+        // the next multiple of 64 are written (zeros past B), 8 columns = 16 bytes per store
         const int kpad = (B + 63) & ~63;
         const int vpr = kpad >> 3;
-        __nv_bfloat16 *Pimg = pbuf + (size_t)out0 * pbuf_pitch;
+        __nv_bfloat16 *Pimg = pbuf + (size_t)t_begin * pbuf_pitch;
         for (int idx = tid; idx < M * vpr; idx += kSfThreads) {
             const int i = idx / vpr, j0 = (idx - i * vpr) << 3;
+            const int tok = __ldg(order + t_begin + i);
             const float ui = us[i];
             __align__(16) float kk[8];
             __align__(16) float vv[8];
@@ -325,9 +326,9 @@ sinkhorn_fast_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
                 // K is zero past column B, so those products are zero
                 const float a = (kk[2 * e] * ui) * vv[2 * e];
                 const float b = (kk[2 * e + 1] * ui) * vv[2 * e + 1];
-                o[e] = __floats2bfloat162_rn(a, b);
+                o[e] = __floats2bfloat162_rn(p.alpha * a, p.alpha * b);
             }
-            *reinterpret_cast<uint4 *>(Pimg + (size_t)i * pbuf_pitch + j0) = *reinterpret_cast<uint4 *>(o);
+            *reinterpret_cast<uint4 *>(Pimg + (size_t)tok * pbuf_pitch + j0) = *reinterpret_cast<uint4 *>(o);
         }
     } else {
         // fp32, in place in the workspace tile (row pitch score_pitch(B))
