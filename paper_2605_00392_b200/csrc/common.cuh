@@ -8,20 +8,22 @@
 
 namespace rtp {
 
-constexpr int kChunkTokens = 64;       // tokens per CTA of the norm/statistics pass
+constexpr int kChunkTokens = 32;       // tokens per CTA of the norm/statistics pass
 constexpr float kNormFloor = 1e-12f;   // divisor floor for a zero-norm token
 constexpr int kStats = RTPRUNE_STATS_STRIDE;
 
 // Workspace header (first 256 bytes of the workspace).
 struct WsHeader {
     uint32_t status;       // RTPRUNE_DEV_* bits
-    uint32_t select_done;  // CTAs of the selection kernel that have published their count
+    uint32_t select_done;  // images whose selection has been published
     uint32_t pad[62];
 };
 
 // Byte offsets of the workspace regions; computed on the host from the plan's maxima.
 struct WsLayout {
     size_t header;     // WsHeader
+    size_t img_done;   // uint32 [batch]           chunks of each image that have finished their pass
+    size_t clear_bytes;  // the workspace's first clear_bytes bytes (header, counters) start at zero
     size_t norms;      // float [total]            C_k
     size_t spart;      // float [batch][chunks][d] partial sums of the unit tokens
     size_t order;      // int32 [total]            per image: kept indices then pruned indices

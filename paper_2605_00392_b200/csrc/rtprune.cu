@@ -62,6 +62,9 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     size_t off = 0;
     L.header = off;
     off = align_up(off + sizeof(WsHeader), 256);
+    L.img_done = off;
+    off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
+    L.clear_bytes = off;
     L.norms = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
     L.spart = off;
@@ -174,25 +177,37 @@ int max_pruned(const rtprune_params_t *p, int max_tokens)
 }
 
 template <typename T>
-cudaError_t launch_norm_stats(const rtprune_plan_t *pl, cudaStream_t st, const void *X,
-                              const int32_t *offsets, int batch, int total, float *norms,
-                              float *spart, WsHeader *hdr)
+cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, const void *X,
+                                 const int32_t *offsets, int batch, int total, const RatioParams &rp,
+                                 const float *rho, char *ws, int32_t *out_offsets, int32_t *counts,
+                                 float *stats, float *norms_out, int32_t *order_out)
 {
     constexpr int EPV = Elem<T>::kPerVec;
+    const WsLayout &L = pl->ws;
     const int d = pl->d;
     const int vpl = (d / EPV + 31) / 32;
-    dim3 grid(pl->ws.chunks, batch);
-    const size_t smem = sizeof(float) * 8 * (size_t)d;
+    // tokens per CTA: about one wave of CTAs (two per SM) for small batches, never fewer than
+    // kChunkTokens (the partial-sum region is sized for that) nor more than 128
+    const int slots = 2 * pl->sm_count;
+    const int per_image = std::max(1, slots / std::max(batch, 1));
+    int chunk_tokens = (pl->max_tokens + per_image - 1) / per_image;
+    chunk_tokens = std::min(128, std::max(kChunkTokens, (chunk_tokens + 7) / 8 * 8));
+    const int chunks_run = (pl->max_tokens + chunk_tokens - 1) / chunk_tokens;   // <= L.chunks
+    dim3 grid(chunks_run, batch);
+    const size_t smem = sizeof(float) * stage1_smem_floats(d, pl->max_tokens);
 #define RTP_CASE(V)                                                                              \
     case V: {                                                                                    \
-        auto k = norm_stats_kernel<T, V>;                                                        \
+        auto k = stage1_kernel<T, V>;                                                            \
         if (smem > 48 * 1024) {                                                                  \
             cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                  (int)smem);                                     \
             if (e != cudaSuccess) return e;                                                      \
         }                                                                                        \
-        k<<<grid, 256, smem, st>>>((const T *)X, offsets, d, pl->ws.chunks, pl->max_tokens,      \
-                                   total, norms, spart, hdr);                                    \
+        k<<<grid, kS1Threads, smem, st>>>(                                                       \
+            (const T *)X, offsets, batch, d, L.chunks, chunk_tokens, pl->max_tokens, total, rp, rho, \
+            (float *)(ws + L.norms), (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),     \
+            (int32_t *)(ws + L.order), (int32_t *)(ws + L.kpos), counts, out_offsets, stats,     \
+            norms_out, order_out, (WsHeader *)(ws + L.header));                                  \
         break;                                                                                   \
     }
     switch (vpl) {
@@ -226,35 +241,22 @@ rtprune_status_t check_common(rtprune_plan_t *plan, const void *X, const int32_t
     return check_params(params);
 }
 
-// Stage 1 launches (norms + statistics, selection).
+// Stage 1: norms, statistics, ratio and selection in one kernel.
 rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void *X,
                                const int32_t *offsets, int32_t batch, int total,
                                const rtprune_params_t *params, char *ws, int32_t *out_offsets,
                                int32_t *counts, float *stats, float *norms_out,
-                               int32_t *order_out, bool with_xp)
+                               int32_t *order_out)
 {
     Checked c{plan};
-    const WsLayout &L = plan->ws;
-    WsHeader *hdr = (WsHeader *)(ws + L.header);
-    float *norms = (float *)(ws + L.norms);
-    float *spart = (float *)(ws + L.spart);
-    int32_t *order = (int32_t *)(ws + L.order);
-    int32_t *kpos = (int32_t *)(ws + L.kpos);
-    cudaError_t e = (plan->dtype == RTPRUNE_BF16)
-                        ? launch_norm_stats<__nv_bfloat16>(plan, st, X, offsets, batch, total, norms, spart, hdr)
-                        : launch_norm_stats<float>(plan, st, X, offsets, batch, total, norms, spart, hdr);
-    if (!c.ok(e)) return RTPRUNE_ERR_CUDA;
-    launched(plan, st, "norm_stats");
     RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
-    const size_t smem = sizeof(float) * (size_t)plan->max_tokens;
-    const bool bf16 = with_xp && plan->dtype == RTPRUNE_BF16;   // the compact copy of T_prop feeds stage 2 only
-    select_kernel<<<batch, 1024, smem, st>>>(offsets, batch, plan->d, L.chunks, plan->max_tokens,
-                                             total, rp, params->rho, norms, spart, order, kpos, counts,
-                                             out_offsets, stats, norms_out, order_out, hdr,
-                                             bf16 ? (const __nv_bfloat16 *)X : nullptr,
-                                             bf16 ? (__nv_bfloat16 *)(ws + L.xp) : nullptr);
-    if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
-    launched(plan, st, "select");
+    cudaError_t e = (plan->dtype == RTPRUNE_BF16)
+                        ? launch_stage1_kernel<__nv_bfloat16>(plan, st, X, offsets, batch, total, rp, params->rho,
+                                                              ws, out_offsets, counts, stats, norms_out, order_out)
+                        : launch_stage1_kernel<float>(plan, st, X, offsets, batch, total, rp, params->rho, ws,
+                                                      out_offsets, counts, stats, norms_out, order_out);
+    if (!c.ok(e)) return RTPRUNE_ERR_CUDA;
+    launched(plan, st, "stage1");
     return RTPRUNE_OK;
 }
 
@@ -277,7 +279,16 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
 
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-            // tensor-core path: one CTA per (128 consecutive tokens, image)
+            // compact copy of the pruned rows for the tensor-core kernels
+            {
+                const int rows_max = (maxB + 63) & ~63;
+                dim3 ggrid((rows_max + kGpRows - 1) / kGpRows, batch);
+                gather_prop_kernel<<<ggrid, 128, 0, st>>>((const __nv_bfloat16 *)X, offsets, o.counts, order,
+                                                         plan->d, maxN, total, (__nv_bfloat16 *)(ws + L.xp));
+                if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+                launched(plan, st, "gather");
+            }
+            // scores: one CTA per (128 consecutive tokens, image)
             CUtensorMap tmapX, tmapXp;
             if (!make_tmap_bf16(plan, &tmapX, X, (uint64_t)total, (uint64_t)plan->d,
                                 (uint64_t)plan->d * 2, kScBK, kScTileM) ||
@@ -372,7 +383,7 @@ rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X
     }
     prof_begin(plan, st);
     rtprune_status_t s = launch_stage1(plan, st, X, offsets, batch, total, params, ws, o.out_offsets,
-                                       o.counts, o.stats, nullptr, nullptr, true);
+                                       o.counts, o.stats, nullptr, nullptr);
     if (s != RTPRUNE_OK) return s;
     return (plan->dtype == RTPRUNE_BF16)
                ? launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o)
@@ -529,7 +540,7 @@ rtprune_status_t rtprune_workspace_init(rtprune_plan_t *plan, void *cuda_stream,
     if (!plan || !workspace || ((uintptr_t)workspace & 255u)) return RTPRUNE_ERR_INVALID_ARG;
     if (workspace_bytes < plan->ws.total) return RTPRUNE_ERR_WORKSPACE;
     Checked c{plan};
-    if (!c.ok(cudaMemsetAsync((char *)workspace + plan->ws.header, 0, sizeof(WsHeader),
+    if (!c.ok(cudaMemsetAsync((char *)workspace + plan->ws.header, 0, plan->ws.clear_bytes,
                               (cudaStream_t)cuda_stream)))
         return RTPRUNE_ERR_CUDA;
     return RTPRUNE_OK;
@@ -575,7 +586,7 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
     }
     prof_begin(plan, (cudaStream_t)cuda_stream);
     return launch_stage1(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
-                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out, false);
+                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out);
 }
 
 rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
@@ -618,11 +629,11 @@ rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, 
         return RTPRUNE_OK;
     }
     // the array keeps whatever the last call left: the status word and the counters must start at 0
-    if (!c.ok(cudaMemsetAsync(scratch + plan->ws.header, 0, sizeof(WsHeader), st)))
+    if (!c.ok(cudaMemsetAsync(scratch + plan->ws.header, 0, plan->ws.clear_bytes, st)))
         return RTPRUNE_ERR_CUDA;
     prof_begin(plan, st);
     return launch_stage1(plan, st, X, offsets, batch, (int)total_tokens, params, scratch, out_offsets,
-                         counts, stats, norms_out, order_out, false);
+                         counts, stats, norms_out, order_out);
 }
 
 rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)
@@ -678,7 +689,7 @@ rtprune_status_t rtprune_run_host(rtprune_plan_t *plan, void *cuda_stream, const
         return RTPRUNE_ERR_CUDA;
     if (rho_host && !c.ok(cudaMemcpyAsync(base + a.rho, rho_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st)))
         return RTPRUNE_ERR_CUDA;
-    if (!c.ok(cudaMemsetAsync(base + a.ws + plan->ws.header, 0, sizeof(WsHeader), st)))
+    if (!c.ok(cudaMemsetAsync(base + a.ws + plan->ws.header, 0, plan->ws.clear_bytes, st)))
         return RTPRUNE_ERR_CUDA;
     DevOut o{base + a.Y,
              (int32_t *)(base + a.out_offsets),

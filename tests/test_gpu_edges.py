@@ -39,7 +39,7 @@ def test_ragged_dynamic(parity):
 def test_retention_one_is_identity(parity):
     w = synth.ragged([7, 64, 200], params=dict(r_fixed=0.0))
     rep = parity.check_workload(w)
-    assert rep["mean_retention"] == 1.0 and rep["launches"] == 3   # stage 2 is not launched
+    assert rep["mean_retention"] == 1.0 and rep["launches"] == 2   # stage 1 + merge: stage 2 is not launched
 
 
 def test_rho_one_prunes_nothing(parity):
@@ -126,7 +126,7 @@ def test_select_entry_point(parity, binding):
     fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w.params.items()}
     plan.select(w.X.to(dev), torch.from_numpy(w.offsets).to(dev), binding.make_params(rho, **fields),
                 out, norms, order)
-    assert plan.query_status() == 0 and plan.last_launch_count == 2
+    assert plan.query_status() == 0 and plan.last_launch_count == 1
     from oracle import oracle
     ref = oracle.run_batch(w.X_f64(), w.offsets, parity.oracle_params(w.params), w.rho)
     for i, im in enumerate(ref.images):
