@@ -87,6 +87,15 @@ __device__ inline void tma_load_2d(uint32_t dst_smem, const CUtensorMap *map, ui
         ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
 }
+// 1-D bulk load global -> shared (both 16-byte aligned, size a multiple of 16); completion is counted
+// in bytes on the mbarrier.
+__device__ inline void bulk_load(uint32_t dst_smem, const void *src_global, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     dst_smem),
+                 "l"(src_global), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 // 1-D bulk store shared -> global (both 16-byte aligned, size a multiple of 16), tracked by the
 // thread's bulk async-group.
 __device__ inline void bulk_store(void *dst_global, uint32_t src_smem, uint32_t bytes)

@@ -194,7 +194,7 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
     chunk_tokens = std::min(128, std::max(kChunkTokens, (chunk_tokens + 7) / 8 * 8));
     const int chunks_run = (pl->max_tokens + chunk_tokens - 1) / chunk_tokens;   // <= L.chunks
     dim3 grid(chunks_run, batch);
-    const size_t smem = sizeof(float) * stage1_smem_floats(d, pl->max_tokens);
+    const size_t smem = sizeof(float) * stage1_smem_floats(d, pl->max_tokens, sizeof(T));
 #define RTP_CASE(V)                                                                              \
     case V: {                                                                                    \
         auto k = stage1_kernel<T, V>;                                                            \

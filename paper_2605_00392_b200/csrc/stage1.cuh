@@ -3,6 +3,7 @@
 // the compact copy of the pruned rows for the tensor-core kernels.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace rtp {
 
@@ -14,19 +15,60 @@ struct RatioParams {
 constexpr int kS1Threads = 256;
 constexpr int kS1Warps = kS1Threads / 32;
 
-// Dynamic shared memory (floats) of stage1_kernel: the 8 warps' partial sums of unit tokens, later the
-// image's norm keys for the ranking.
-__host__ __device__ inline size_t stage1_smem_floats(int d, int max_tokens)
+constexpr int kS1StageRows = kS1Warps;   // rows per stage of the streaming ring: one per warp
+constexpr int kS1MaxStages = 4;
+
+// Stages of the streaming ring for rows of row_bytes: as many as fit in 96 KB, 2 to 4.
+__host__ __device__ inline int stage1_stages(size_t row_bytes)
 {
+    const size_t s = (96u * 1024u) / (kS1StageRows * row_bytes);
+    return s < 2 ? 2 : (s > (size_t)kS1MaxStages ? kS1MaxStages : (int)s);
+}
+
+// Dynamic shared memory (floats) of stage1_kernel: the ring of row stages, reused for the 8 warps'
+// partial sums of unit tokens and then for the image's norm keys of the ranking.
+__host__ __device__ inline size_t stage1_smem_floats(int d, int max_tokens, size_t elem_bytes)
+{
+    const size_t ring = (size_t)stage1_stages((size_t)d * elem_bytes) * kS1StageRows * d * elem_bytes / 4;
     const size_t a = (size_t)kS1Warps * d, b = (size_t)max_tokens + 64;
-    return a > b ? a : b;
+    const size_t m = a > b ? a : b;
+    return ring > m ? ring : m;
+}
+
+// Exclusive prefix sum of one int per thread over the CTA (256 threads); `scratch` holds 32 ints.
+__device__ inline int block_excl_scan(int v, int *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();                       // scratch may still be read from an earlier scan
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < kS1Warps) ? scratch[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        scratch[lane] = wi - w;
+    }
+    __syncthreads();
+    return scratch[warp] + incl - v;
 }
 
 // ---------------------------------------------------------------------------------------------
 // Selection of one image by one CTA (256 threads): phi from the chunk partials; r and
-// B = floor(r N + 1/2) clamped to [0, N-1], M = N - B; rank of every token under (norm descending,
-// index ascending) by counting; the M best are T_kept.  Writes order[] = kept indices ascending, then
-// pruned indices ascending, and its inverse kpos[]; counts, stats.
+// B = floor(r N + 1/2) clamped to [0, N-1], M = N - B; the M tokens of largest norm (ties to the lower
+// index) are T_kept.  The M-th largest norm is found by a radix select over the norm bits (four
+// 8-bit digits, a 256-bin histogram each), tokens equal to it are admitted in index order.  Writes
+// order[] = kept indices ascending, then pruned indices ascending, and its inverse kpos[]; counts,
+// stats.
 // ---------------------------------------------------------------------------------------------
 __device__ inline void select_image(int img, int t_begin, int N, int d, int chunks, int chunk_tokens,
                                     const RatioParams &rp,
@@ -38,10 +80,21 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
 {
     __shared__ float s_redf[32];
     __shared__ int s_redi[32];
+    __shared__ int s_hist[256];
     __shared__ int s_M;
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_need;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int nth = kS1Threads;
 
+    // every global read is issued up front: rho, the norms (keys of the ranking), the chunk partials
+    const float rho_i = (tid == 0 && rho) ? __ldg(rho + img) : 0.f;
+    // norm bits: for non-negative floats the unsigned order is the float order, and a NaN still ranks
+    for (int k = tid; k < N; k += nth) {
+        const float key = __ldcg(norms + t_begin + k);
+        s_keys[k] = __float_as_uint(key) & 0x7fffffffu;
+        if (norms_out) norms_out[t_begin + k] = key;
+    }
     // phi (Eq. 8) via |sum of unit tokens|^2; the partials were written by other CTAs: read them from L2
     const int nchunk = (N + chunk_tokens - 1) / chunk_tokens;
     const float *sp = spart + (size_t)img * chunks * d;
@@ -56,7 +109,6 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
     if (tid == 0) {
         const float Nf = (float)N;
         const float phi = (N >= 2) ? (ssum - Nf) / (Nf * (Nf - 1.f)) : 0.f;
-        const float rho_i = rho ? rho[img] : 0.f;
         float r;
         if (rp.dynamic) {
             float f = (phi - rp.phi_lo) / (rp.phi_hi - rp.phi_lo);
@@ -80,69 +132,76 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
         st[7] = 0.f;
         counts[img] = N - B;
     }
-    // norm bits: for non-negative floats the unsigned order is the float order, and a NaN still ranks
-    for (int k = tid; k < N; k += nth) {
-        const float key = __ldcg(norms + t_begin + k);
-        s_keys[k] = __float_as_uint(key) & 0x7fffffffu;
-        if (norms_out) norms_out[t_begin + k] = key;
-    }
-    if (tid < 4) s_keys[N + tid] = 0u;   // padding read by the 4-wide ranking loop; never outranks a token
     __syncthreads();
     const int M = s_M;
 
-    // Each thread owns a contiguous range of tokens so that a block scan of its kept count gives
-    // output positions in ascending index.
+    // radix select: after the four digits `prefix` is the M-th largest key and `need` is how many
+    // tokens equal to it are kept
+    uint32_t prefix = 0;
+    int need = M;
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        s_hist[tid] = 0;
+        __syncthreads();
+        for (int k = tid; k < N; k += nth) {
+            const uint32_t key = s_keys[k];
+            if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns the bins 255 - 8 l down to 248 - 8 l: largest digits first
+            int h[8], sum8 = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                h[q] = s_hist[255 - 8 * lane - q];
+                sum8 += h[q];
+            }
+            int incl = sum8;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            int c = incl - sum8;
+            if (c < need && need <= incl) {            // exactly one lane
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (c < need && need <= c + h[q]) {
+                        s_prefix = (prefix << 8) | (uint32_t)(255 - 8 * lane - q);
+                        s_need = need - c;
+                    }
+                    c += h[q];
+                }
+            }
+        }
+        __syncthreads();
+        prefix = s_prefix;
+        need = s_need;
+    }
+    const uint32_t thr = prefix;
+
+    // Each thread owns a contiguous range of tokens so that block scans give positions in ascending
+    // index: first among the tokens equal to the threshold, then among the kept ones.
     const int ipt = (N + nth - 1) / nth;          // <= 32 for N <= 8192
     const int k0 = min(tid * ipt, N), k1 = min(k0 + ipt, N);
+    int neq = 0;
+    for (int k = k0; k < k1; ++k) neq += (s_keys[k] == thr) ? 1 : 0;
+    int eq_run = block_excl_scan(neq, s_redi);
     uint32_t keptmask = 0;
     int nkept = 0;
     for (int k = k0; k < k1; ++k) {
-        const uint32_t my = s_keys[k];
-        int rank = 0;
-        // tokens that outrank k: a larger key anywhere, or an equal key at a lower index.  Below k the
-        // test is >=, above it >; only the 4-wide group that holds k needs the index.
-        const int kb = k & ~3;
-        for (int l = 0; l < kb; l += 4) {
-            const uint4 o = *reinterpret_cast<const uint4 *>(s_keys + l);
-            rank += (o.x >= my) + (o.y >= my) + (o.z >= my) + (o.w >= my);
+        const uint32_t key = s_keys[k];
+        bool kept = key > thr;
+        if (key == thr) {
+            kept = eq_run < need;
+            ++eq_run;
         }
-        {
-            const uint4 o = *reinterpret_cast<const uint4 *>(s_keys + kb);
-            rank += (o.x > my || (o.x == my && kb + 0 < k)) ? 1 : 0;
-            rank += (o.y > my || (o.y == my && kb + 1 < k)) ? 1 : 0;
-            rank += (o.z > my || (o.z == my && kb + 2 < k)) ? 1 : 0;
-            rank += (o.w > my || (o.w == my && kb + 3 < k)) ? 1 : 0;
-        }
-        for (int l = kb + 4; l < N; l += 4) {
-            const uint4 o = *reinterpret_cast<const uint4 *>(s_keys + l);
-            rank += (o.x > my) + (o.y > my) + (o.z > my) + (o.w > my);
-        }
-        if (rank < M) {
+        if (kept) {
             keptmask |= 1u << (k - k0);
             ++nkept;
         }
     }
-    // exclusive block scan of nkept
-    int incl = nkept;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) s_redi[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int w = (lane < (nth >> 5)) ? s_redi[lane] : 0;
-        int wi = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, wi, o);
-            if (lane >= o) wi += t;
-        }
-        s_redi[lane] = wi - w;
-    }
-    __syncthreads();
-    int kpos_run = s_redi[warp] + incl - nkept;  // kept tokens before k0
+    int kpos_run = block_excl_scan(nkept, s_redi);   // kept tokens before k0
     int32_t *ord = order + t_begin;
     for (int k = k0; k < k1; ++k) {
         const bool kept = (keptmask >> (k - k0)) & 1u;
@@ -158,14 +217,15 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
 // ---------------------------------------------------------------------------------------------
 // grid = (chunks of this run, batch), 256 threads; CTA (c, i) owns chunk_tokens consecutive tokens of
 // image i (a multiple of 8, at least kChunkTokens, chosen by the host so that the grid is about one wave).
-//   Pass over X: a warp holds one token in registers and the next in flight (128-bit loads), fp32 sum of squares
-//   by shuffle reduction; while the rows are still in registers they are added, divided by their
+//   Pass over X: the chunk's rows stream through a shared-memory ring (bulk copies issued by one
+//   thread); a warp takes one row of each stage: fp32 sum of squares
+//   by shuffle reduction; while the row is still in registers it is added, divided by its
 //   norm, into per-lane accumulators; the CTA writes the partial sum of unit tokens of its chunk to
 //   spart[img][chunk][d].  phi needs only |sum_k x_k/|x_k||^2:
 //       sum_{k<l} cos(x_k, x_l) = (|sum_k xhat_k|^2 - N) / 2.
 //   The CTA that finishes an image last (a counter per image) runs the selection of that image; the
 //   CTA that finishes the last image turns counts into out_offsets (exclusive prefix sum).
-// Dynamic shared memory: stage1_smem_floats(d, max_tokens) floats.
+// Dynamic shared memory: stage1_smem_floats(d, max_tokens, sizeof(T)) floats.
 // ---------------------------------------------------------------------------------------------
 template <typename T, int VPL>  // VPL = 16-byte vectors per lane = ceil(d / (32 * kPerVec))
 __global__ void __launch_bounds__(kS1Threads, 2)
@@ -180,6 +240,7 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
     extern __shared__ __align__(16) float s_dyn[];
     __shared__ bool s_last;
     __shared__ int s_scan[32];
+    __shared__ uint64_t s_full[kS1MaxStages], s_empty[kS1MaxStages];
     const int img = blockIdx.y, chunk = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int t_begin, n_img;
@@ -202,53 +263,75 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
         float acc[VPL * EPV];
 #pragma unroll
         for (int i = 0; i < VPL * EPV; ++i) acc[i] = 0.f;
-        bool bad = false;
-        // the warp's tokens t0 + warp, + 8, ...: the next row is requested before the current one is
-        // reduced, so that every warp always has loads in flight
-        uint4 cur[VPL], nxt[VPL];
-        int t = t0 + warp;
-        if (t < t1) {
-            const uint4 *row = reinterpret_cast<const uint4 *>(X + (size_t)t * d);
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) {
-                const int vi = lane + 32 * j;
-                cur[j] = (vi < nvec) ? __ldg(row + vi) : make_uint4(0, 0, 0, 0);
+        bool bad = false, gave_up = false;
+
+        // The chunk's rows are contiguous in X: thread 0 streams them through a ring of shared-memory
+        // stages (8 rows each, one per warp) with bulk copies, a few stages ahead of the warps.
+        const size_t row_bytes = (size_t)d * sizeof(T);
+        const int nstage = stage1_stages(row_bytes);
+        const uint32_t stage_bytes = (uint32_t)(kS1StageRows * row_bytes);
+        const uint32_t ring_u32 = ptx::smem_u32(s_dyn);
+        const int nit = (t1 - t0 + kS1StageRows - 1) / kS1StageRows;
+        if (tid == 0) {
+            for (int s = 0; s < kS1MaxStages; ++s) {
+                ptx::mbar_init(&s_full[s], 1);
+                ptx::mbar_init(&s_empty[s], kS1Warps);
             }
+            ptx::fence_mbar_init();
         }
-        while (t < t1) {
-            const int tn = t + kS1Warps;
-            if (tn < t1) {
-                const uint4 *row = reinterpret_cast<const uint4 *>(X + (size_t)tn * d);
+        __syncthreads();
+        auto issue = [&](int it) {
+            const int s = it % nstage;
+            const int r0 = t0 + it * kS1StageRows;
+            const uint32_t bytes = (uint32_t)(min(kS1StageRows, t1 - r0) * row_bytes);
+            ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
+            ptx::bulk_load(ring_u32 + s * stage_bytes, X + (size_t)r0 * d, bytes, &s_full[s]);
+        };
+        if (tid == 0)
+            for (int it = 0; it < min(nstage, nit); ++it) issue(it);
+        for (int it = 0; it < nit; ++it) {
+            const int s = it % nstage;
+            if (!gave_up && !ptx::mbar_wait(&s_full[s], (it / nstage) & 1)) gave_up = true;
+            const int t = t0 + it * kS1StageRows + warp;
+            if (t < t1 && !gave_up) {
+                const uint4 *row = reinterpret_cast<const uint4 *>(
+                    reinterpret_cast<const uint8_t *>(s_dyn) + s * stage_bytes + warp * row_bytes);
+                uint4 cur[VPL];
 #pragma unroll
                 for (int j = 0; j < VPL; ++j) {
                     const int vi = lane + 32 * j;
-                    nxt[j] = (vi < nvec) ? __ldg(row + vi) : make_uint4(0, 0, 0, 0);
+                    cur[j] = (vi < nvec) ? row[vi] : make_uint4(0, 0, 0, 0);
+                }
+                float ss = 0.f;
+#pragma unroll
+                for (int j = 0; j < VPL; ++j) {
+                    float f[EPV];
+                    Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+                }
+                ss = warp_sum(ss);
+                const float n = sqrtf(ss);
+                if (!(ss <= 3.0e38f)) bad = true;  // inf or NaN
+                const float inv = 1.f / fmaxf(n, kNormFloor);
+                if (lane == 0) norms[t] = n;
+#pragma unroll
+                for (int j = 0; j < VPL; ++j) {
+                    float f[EPV];
+                    Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc[j * EPV + e] = fmaf(f[e], inv, acc[j * EPV + e]);
                 }
             }
-            float ss = 0.f;
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) {
-                float f[EPV];
-                Elem<T>::unpack(cur[j], f);
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&s_empty[s]);
+            if (tid == 0 && it + nstage < nit) {     // refill the stage once all eight warps have left it
+                if (!gave_up && !ptx::mbar_wait(&s_empty[s], (it / nstage) & 1)) gave_up = true;
+                if (!gave_up) issue(it + nstage);
             }
-            ss = warp_sum(ss);
-            const float n = sqrtf(ss);
-            if (!(ss <= 3.0e38f)) bad = true;  // inf or NaN
-            const float inv = 1.f / fmaxf(n, kNormFloor);
-            if (lane == 0) norms[t] = n;
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) {
-                float f[EPV];
-                Elem<T>::unpack(cur[j], f);
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) acc[j * EPV + e] = fmaf(f[e], inv, acc[j * EPV + e]);
-            }
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) cur[j] = nxt[j];
-            t = tn;
         }
+        if (gave_up && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+        __syncthreads();      // the ring is free: it now holds the warps' partial sums
         if (bad && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_NONFINITE);
 
         // reduce the 8 warps' accumulators through shared memory
