@@ -277,7 +277,7 @@ def main() -> None:
             "select": ("hbm", total * 4 * 2 + batch * 48),
             "scores": ("alu", 2.0 * sumMB * d),
             "sinkhorn": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
-            "sinkhorn_fast": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
+            "sinkhorn_cluster": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
             "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
         }
         bound, units = algo[dominant]

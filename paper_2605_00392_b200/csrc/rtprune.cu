@@ -13,7 +13,7 @@
 #include "merge_umma.cuh"
 #include "scores_umma.cuh"
 #include "sinkhorn.cuh"
-#include "sinkhorn_fast.cuh"
+#include "sinkhorn_cluster.cuh"
 #include "stage1.cuh"
 
 using namespace rtp;
@@ -314,19 +314,34 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         const int smem_floats = plan->sink_smem_bytes / (int)sizeof(float);
         // Scaling form: tiles that fit one CTA's shared memory go to the one-pass kernel; the general
         // kernel then takes what is left (it skips the images already solved).
-        int fast_nc = 0;
+        int fast_c = 0;
         const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
         bool all_fast = false;
         if (!use_log_form(params)) {
-            fast_nc = kSfMaxNc;
-            all_fast = maxB <= 32 * fast_nc;
+            // CTAs per image: as many as keep the whole batch on the chip at once, 8 at most
+            fast_c = 1;
+            while (fast_c < 8 && (long long)batch * fast_c * 2 <= plan->sm_count) fast_c *= 2;
+            all_fast = maxB <= 32 * kSfMaxNc;
             for (int b = 1; b <= maxB && all_fast; ++b)
-                all_fast = sinkhorn_fast_fits(std::max(maxN - b, 1), b, fast_nc, fast_floats);
-            sinkhorn_fast_kernel<<<batch, kSfThreads, plan->fast_smem_bytes, st>>>(
-                offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op, fast_floats,
-                pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats);
-            if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
-            launched(plan, st, "sinkhorn_fast");
+                all_fast = sinkhorn_cluster_fits(std::max(maxN - b, 1), b, fast_c, fast_floats);
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(batch * fast_c));
+            cfg.blockDim = dim3(kSfThreads);
+            cfg.dynamicSmemBytes = (size_t)plan->fast_smem_bytes;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)fast_c;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (!c.ok(cudaLaunchKernelEx(&cfg, sinkhorn_cluster_kernel, offsets, (const int32_t *)o.counts,
+                                         (const int32_t *)o.out_offsets, (const int32_t *)order, kmat,
+                                         L.kmat_stride, maxN, total, op, fast_floats, pbuf, pbuf_pitch,
+                                         o.merged_idx, o.merge_partner, o.merge_weight, o.stats)))
+                return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "sinkhorn_cluster");
         }
         if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
@@ -337,7 +352,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             sinkhorn_kernel<false><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                o.stats, fast_nc, fast_floats);
+                o.stats, fast_c, fast_floats);
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
         if (use_log_form(params) || !all_fast) launched(plan, st, "sinkhorn");
     }
@@ -503,7 +518,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         return RTPRUNE_ERR_CUDA;
     }
     p->fast_smem_bytes = (int)(cap / 16 * 16);
-    if (!c.ok(cudaFuncSetAttribute(sinkhorn_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (!c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    p->fast_smem_bytes))) {
         delete p;
         return RTPRUNE_ERR_CUDA;

@@ -19,16 +19,18 @@ constexpr int kSfThreads = 512;
 constexpr int kSfWarps = kSfThreads / 32;
 constexpr int kSfMaxNc = 8;            // the one-pass kernel takes tiles of at most 32 * 8 columns
 
-// Shared-memory floats the one-pass kernel (sinkhorn_fast.cuh) needs for an M x B tile: K padded to
-// 32-column multiples, cross-warp partials for the column sums and for the pairing, duals, scratch.
-__host__ __device__ inline long long sinkhorn_fast_floats(int M, int B)
+// Shared-memory floats one CTA of the cluster kernel (sinkhorn_cluster.cuh) needs for an M x B tile
+// split over C CTAs: its rows of K padded to 32-column multiples, per-warp and per-CTA partials of the
+// column sums (the same space serves the pairing), duals, scratch.
+__host__ __device__ inline long long sinkhorn_cluster_floats(int M, int B, int C)
 {
     const long long ldk = (B + 31) & ~31;
-    return (long long)M * ldk + 2 * kSfWarps * ldk + (M + 8) + (ldk + 4) + 2 * kSfWarps + 32 + 16;
+    const long long rows_per = (M + C - 1) / C;
+    return rows_per * ldk + 2 * kSfWarps * ldk + 2 * C * ldk + (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
 }
-__host__ __device__ inline bool sinkhorn_fast_fits(int M, int B, int ncmax, int smem_floats)
+__host__ __device__ inline bool sinkhorn_cluster_fits(int M, int B, int C, int smem_floats)
 {
-    return B >= 1 && B <= 32 * ncmax && sinkhorn_fast_floats(M, B) <= (long long)smem_floats;
+    return B >= 1 && B <= 32 * kSfMaxNc && sinkhorn_cluster_floats(M, B, C) <= (long long)smem_floats;
 }
 
 __device__ inline void lse_merge(float &m, float &s, float m2, float s2)
@@ -58,7 +60,7 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
                 int smem_floats, __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch,
                 int32_t *__restrict__ merged_idx,
                 int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
-                float *__restrict__ stats, int fast_ncmax, int fast_smem_floats)
+                float *__restrict__ stats, int fast_cluster, int fast_smem_floats)
 {
     extern __shared__ __align__(16) float sm[];
     __shared__ float s_red[32];
@@ -70,8 +72,8 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;
     if (B == 0) return;
-    // images whose tile fits the shared-memory kernel launched before this one were solved there
-    if (fast_ncmax > 0 && sinkhorn_fast_fits(M, B, fast_ncmax, fast_smem_floats)) return;
+    // images whose tile fits the cluster kernel launched before this one were solved there
+    if (fast_cluster > 0 && sinkhorn_cluster_fits(M, B, fast_cluster, fast_smem_floats)) return;
     const int R = M + 1, Cc = B + 1;
 
     float *u = sm;
