@@ -25,21 +25,24 @@ namespace rtp {
 constexpr int kMgTileM = 128;
 constexpr int kMgTileN = 256;        // output columns per unit
 constexpr int kMgBK = 64;            // contraction rows per k-block
-constexpr int kMgStages = 2;
+constexpr int kMgBStages = 3;        // ring of B tiles (every k-block)
+constexpr int kMgAStages = 2;        // ring of plan tiles (k-blocks after the identity ones)
 constexpr int kMgThreads = 192;
 constexpr int kMgABytes = kMgTileM * 128;            // A tile: 128 rows x 64 bf16
 constexpr int kMgBBytes = kMgBK * kMgTileN * 2;      // B tile: 64 rows x 256 bf16 = 32 KB
 constexpr int kMgBBoxBytes = kMgBK * 128;            // one 64-column slab of it
-constexpr int kMgStageBytes = kMgABytes + kMgBBytes; // 48 KB
-constexpr int kMgIdentBytes = 2 * kMgABytes;         // I_128 as two 128 x 64 K-major tiles
+// I_128 as two 128 x 64 K-major views of [64 zero rows][I_64][64 zero rows]: the view that starts at
+// the I_64 block has its ones in rows 0-63, the view that starts 64 rows earlier in rows 64-127.
+constexpr int kMgIdentBytes = 3 * (kMgABytes / 2);
 constexpr int kMgIdentKb = 2;                        // k-blocks that carry the token tile's own rows
 constexpr int kMgStagePitch = kMgTileN * 2 + 16;     // bytes per staging row: padded, conflict-free
 constexpr int kMgStagingBytes = kMgTileM * kMgStagePitch;
-constexpr int kMgSmemBytes = kMgStages * kMgStageBytes + kMgIdentBytes + kMgStagingBytes + 1024 + 256;
+constexpr int kMgSmemBytes = kMgBStages * kMgBBytes + kMgAStages * kMgABytes + kMgIdentBytes +
+                             kMgStagingBytes + 1024 + 256;
 
 struct MergeBarriers {
-    uint64_t full[kMgStages];
-    uint64_t empty[kMgStages];
+    uint64_t full[kMgBStages];       // B tile (and, for plan k-blocks, the A tile) of a k-block has landed
+    uint64_t empty[kMgBStages];      // the k-block's UMMAs have read them
     uint64_t accum_full[2];
     uint64_t accum_empty[2];
     uint32_t tmem_base;
@@ -79,25 +82,27 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *ident = smem + kMgStages * kMgStageBytes;
+    uint8_t *a_ring = smem + kMgBStages * kMgBBytes;
+    uint8_t *ident = a_ring + kMgAStages * kMgABytes;
     uint8_t *staging = ident + kMgIdentBytes;
     MergeBarriers *bars = reinterpret_cast<MergeBarriers *>(staging + kMgStagingBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nct = (d + kMgTileN - 1) / kMgTileN;
     const int nunits = batch * mtiles * nct;
 
-    // identity tiles: tile h holds ones at (row r, k = r - 64 h), in the swizzled K-major layout
+    // identity block: rows 64 .. 127 of the 192-row region hold I_64 (ones at (64 + r, k = r)), in the
+    // swizzled K-major layout; the other rows are zero
     for (int v = tid; v < kMgIdentBytes / 16; v += kMgThreads)
         reinterpret_cast<uint4 *>(ident)[v] = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    if (tid < kMgTileM) {
-        const int r = tid, h = r >> 6, k = r & 63;
-        const uint32_t off = h * kMgABytes + (r >> 3) * 1024 + (r & 7) * 128 + (((k >> 3) ^ (r & 7)) << 4) + (k & 7) * 2;
+    if (tid < 64) {
+        const int r = 64 + tid, k = tid;
+        const uint32_t off = (r >> 3) * 1024 + (r & 7) * 128 + (((k >> 3) ^ (r & 7)) << 4) + (k & 7) * 2;
         *reinterpret_cast<uint16_t *>(ident + off) = 0x3F80;   // bf16 1.0
     }
     ptx::fence_proxy_async_smem();
     if (tid == 0) {
-        for (int s = 0; s < kMgStages; ++s) {
+        for (int s = 0; s < kMgBStages; ++s) {
             ptx::mbar_init(&bars->full[s], 1);
             ptx::mbar_init(&bars->empty[s], 1);
         }
@@ -124,7 +129,11 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
             ptx::prefetch_tensormap(&tmapX);
             ptx::prefetch_tensormap(&tmapXp);
             ptx::prefetch_tensormap(&tmapP);
-            uint32_t it = 0;
+            // `it` counts k-blocks (B ring), `ia` plan k-blocks (A ring).  a_user[slot] is the k-block that
+            // last read the A slot: its UMMAs must have finished before the slot is refilled.
+            uint32_t it = 0, ia = 0;
+            uint32_t a_user[kMgAStages];
+            for (int s = 0; s < kMgAStages; ++s) a_user[s] = 0xffffffffu;
             for (int u = blockIdx.x; u < nunits && !bars->abort_flag; u += gridDim.x) {
                 const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total);
                 if (!q.valid) continue;
@@ -134,19 +143,32 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                 const int col0 = q.ct * kMgTileN;
                 const int nslab = min(kMgTileN, d - col0 + 63) / 64;   // 64-column slabs with any column < d
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % kMgStages;
-                    if (it >= (uint32_t)kMgStages &&
-                        !ptx::mbar_wait(&bars->empty[s], ((it / kMgStages) - 1) & 1)) {
+                    const int s = it % kMgBStages;
+                    if (it >= (uint32_t)kMgBStages &&
+                        !ptx::mbar_wait(&bars->empty[s], ((it / kMgBStages) - 1) & 1)) {
                         bars->abort_flag = 1;
                         atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
                         break;
                     }
-                    const uint32_t a_dst = smem_base + s * kMgStageBytes;
-                    const uint32_t b_dst = a_dst + kMgABytes;
+                    const uint32_t b_dst = smem_base + s * kMgBBytes;
                     const bool own = kb < kMgIdentKb;       // the token tile's own rows: A is the identity
                     ptx::mbar_arrive_expect_tx(&bars->full[s], (own ? 0 : kMgABytes) + nslab * kMgBBoxBytes);
-                    if (!own)
-                        ptx::tma_load_2d(a_dst, &tmapP, &bars->full[s], (kb - kMgIdentKb) * kMgBK, row0);
+                    if (!own) {
+                        const int sa = ia % kMgAStages;
+                        const uint32_t prev = a_user[sa];
+                        // k-blocks up to it - kMgBStages are known to be done (the wait above); a younger
+                        // reader of this A slot is the latest user of its B slot: wait for that phase
+                        if (prev != 0xffffffffu && prev + kMgBStages > it &&
+                            !ptx::mbar_wait(&bars->empty[prev % kMgBStages], (prev / kMgBStages) & 1)) {
+                            bars->abort_flag = 1;
+                            atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                            break;
+                        }
+                        a_user[sa] = it;
+                        ptx::tma_load_2d(ptx::smem_u32(a_ring) + sa * kMgABytes, &tmapP, &bars->full[s],
+                                         (kb - kMgIdentKb) * kMgBK, row0);
+                        ++ia;
+                    }
                     const CUtensorMap *bm = own ? &tmapX : &tmapXp;
                     const int brow = own ? row0 + kb * kMgBK : xp0 + (kb - kMgIdentKb) * kMgBK;
                     for (int sl = 0; sl < nslab; ++sl)
@@ -158,7 +180,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
         // ---------------- UMMA issuer -----------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = ptx::idesc_bf16(kMgTileM, kMgTileN, false, true);
-            uint32_t it = 0, acc = 0;
+            uint32_t it = 0, ia = 0, acc = 0;
             for (int u = blockIdx.x; u < nunits && !bars->abort_flag; u += gridDim.x) {
                 const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total);
                 if (!q.valid) continue;
@@ -175,15 +197,21 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kMgTileN);
                 bool failed = false;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % kMgStages;
-                    if (!ptx::mbar_wait(&bars->full[s], (it / kMgStages) & 1)) {
+                    const int s = it % kMgBStages;
+                    if (!ptx::mbar_wait(&bars->full[s], (it / kMgBStages) & 1)) {
                         failed = true;
                         break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t a_base = (kb < kMgIdentKb) ? ptx::smem_u32(ident) + kb * kMgABytes
-                                                              : smem_base + s * kMgStageBytes;
-                    const uint32_t b_base = smem_base + s * kMgStageBytes + kMgABytes;
+                    // identity k-block 0: the view whose rows 0-63 are I_64; k-block 1: rows 64-127
+                    uint32_t a_base;
+                    if (kb < kMgIdentKb) {
+                        a_base = ptx::smem_u32(ident) + (1 - kb) * (kMgABytes / 2);
+                    } else {
+                        a_base = ptx::smem_u32(a_ring) + (ia % kMgAStages) * kMgABytes;
+                        ++ia;
+                    }
+                    const uint32_t b_base = smem_base + s * kMgBBytes;
 #pragma unroll
                     for (int k = 0; k < kMgBK / 16; ++k) {
                         // A: K-major, 32 bytes further along the 128-byte row per 16 k.
