@@ -122,6 +122,10 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
     ptx::tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     const uint32_t smem_base = ptx::smem_u32(smem);
+    // everything above is local set-up; the plan, the selection and the compact copy come from the
+    // kernels ahead in the stream
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();
 
     if (warp == 4) {
         // ---------------- producer: tiled TMA for every operand -------------------------------------

@@ -115,6 +115,15 @@ template <int N> __device__ inline void bulk_wait()
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// ---- programmatic dependent launch --------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start before the kernel
+// ahead of it in the stream has finished.  grid_dep_wait() returns once that kernel has completed and
+// its writes are visible (at once if there is no such dependency); nothing it wrote may be read, and
+// nothing it reads may be written, before the call.  grid_dep_launch() lets the next kernel in the
+// stream begin its own prologue once every CTA of this grid has called it or exited.
+__device__ inline void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- thread-block clusters: ranks, distributed shared memory, cluster barrier ------------------------
 __device__ inline uint32_t cluster_ctarank()
 {

@@ -112,6 +112,35 @@ void launched(rtprune_plan_t *plan, cudaStream_t st, const char *name)
     }
 }
 
+// Launch with programmatic stream serialization (the kernel may begin while the one ahead of it in the
+// stream drains; it calls grid_dep_wait() before touching anything that kernel produced), optionally
+// as thread-block clusters of `cluster` CTAs.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       unsigned cluster, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -203,11 +232,12 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
                                                  (int)smem);                                     \
             if (e != cudaSuccess) return e;                                                      \
         }                                                                                        \
-        k<<<grid, kS1Threads, smem, st>>>(                                                       \
+        cudaError_t e = launch_pdl(k, grid, dim3(kS1Threads), smem, st, 1u,                      \
             (const T *)X, offsets, batch, d, L.chunks, chunk_tokens, pl->max_tokens, total, rp, rho, \
             (float *)(ws + L.norms), (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),     \
             (int32_t *)(ws + L.order), (int32_t *)(ws + L.kpos), counts, out_offsets, stats,     \
             norms_out, order_out, (WsHeader *)(ws + L.header));                                  \
+        if (e != cudaSuccess) return e;                                                          \
         break;                                                                                   \
     }
     switch (vpl) {
@@ -283,9 +313,10 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             {
                 const int rows_max = (maxB + 63) & ~63;
                 dim3 ggrid((rows_max + kGpRows - 1) / kGpRows, batch);
-                gather_prop_kernel<<<ggrid, 128, 0, st>>>((const __nv_bfloat16 *)X, offsets, o.counts, order,
-                                                         plan->d, maxN, total, (__nv_bfloat16 *)(ws + L.xp));
-                if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+                if (!c.ok(launch_pdl(gather_prop_kernel, ggrid, dim3(128), 0, st, 1u,
+                                     (const __nv_bfloat16 *)X, offsets, o.counts, order, plan->d, maxN, total,
+                                     (__nv_bfloat16 *)(ws + L.xp))))
+                    return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "gather");
             }
             // scores: one CTA per (128 consecutive tokens, image)
@@ -296,9 +327,10 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                 (uint64_t)plan->d * 2, kScBK, kScBBoxRows))
                 return RTPRUNE_ERR_CUDA;
             dim3 grid((maxN + kScTileM - 1) / kScTileM, batch);
-            scores_umma_kernel<<<grid, kScThreads, kScSmemBytes, st>>>(
-                tmapX, tmapXp, offsets, plan->d, o.counts, order, (const int32_t *)(ws + L.kpos), norms,
-                kmat, L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header));
+            if (!c.ok(launch_pdl(scores_umma_kernel, grid, dim3(kScThreads), kScSmemBytes, st, 1u, tmapX, tmapXp,
+                                 offsets, plan->d, o.counts, order, (const int32_t *)(ws + L.kpos), norms, kmat,
+                                 L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header))))
+                return RTPRUNE_ERR_CUDA;
         } else {
             const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
             dim3 grid(mtiles * btiles, batch);
@@ -324,22 +356,10 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             all_fast = maxB <= 32 * kSfMaxNc;
             for (int b = 1; b <= maxB && all_fast; ++b)
                 all_fast = sinkhorn_cluster_fits(std::max(maxN - b, 1), b, fast_c, fast_floats);
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)(batch * fast_c));
-            cfg.blockDim = dim3(kSfThreads);
-            cfg.dynamicSmemBytes = (size_t)plan->fast_smem_bytes;
-            cfg.stream = st;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = (unsigned)fast_c;
-            attr[0].val.clusterDim.y = 1;
-            attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            if (!c.ok(cudaLaunchKernelEx(&cfg, sinkhorn_cluster_kernel, offsets, (const int32_t *)o.counts,
-                                         (const int32_t *)o.out_offsets, (const int32_t *)order, kmat,
-                                         L.kmat_stride, maxN, total, op, fast_floats, pbuf, pbuf_pitch,
-                                         o.merged_idx, o.merge_partner, o.merge_weight, o.stats)))
+            if (!c.ok(launch_pdl(sinkhorn_cluster_kernel, dim3((unsigned)(batch * fast_c)), dim3(kSfThreads),
+                                 (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets, o.counts,
+                                 o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op, fast_floats, pbuf,
+                                 pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats)))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_cluster");
         }
@@ -371,10 +391,11 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         const int nct = (plan->d + kMgTileN - 1) / kMgTileN;
         const long long nunits = (long long)batch * mtiles_m * nct;
         const int grid = (int)std::min<long long>(nunits, plan->sm_count);
-        merge_umma_kernel<<<grid, kMgThreads, kMgSmemBytes, st>>>(
-            tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
-            (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
-            (WsHeader *)(ws + L.header));
+        if (!c.ok(launch_pdl(merge_umma_kernel, dim3((unsigned)grid), dim3(kMgThreads), kMgSmemBytes, st, 1u,
+                             tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
+                             (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
+                             (WsHeader *)(ws + L.header))))
+            return RTPRUNE_ERR_CUDA;
     } else {
         const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
         dim3 grid(mtiles * dtiles, batch);

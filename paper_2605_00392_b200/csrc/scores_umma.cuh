@@ -49,6 +49,8 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
 {
     extern __shared__ uint8_t smem_raw[];
     const int img = blockIdx.y, mt = blockIdx.x;
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();     // counts, order, norms and the compact copy come from the kernels ahead
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;

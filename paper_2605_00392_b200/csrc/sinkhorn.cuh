@@ -26,7 +26,7 @@ __host__ __device__ inline long long sinkhorn_cluster_floats(int M, int B, int C
 {
     const long long ldk = (B + 31) & ~31;
     const long long rows_per = (M + C - 1) / C;
-    return rows_per * ldk + 2 * kSfWarps * ldk + 2 * C * ldk + (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
+    return rows_per * ldk + 2 * kSfWarps * ldk + 2 * C * ldk + 2 * (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
 }
 __host__ __device__ inline bool sinkhorn_cluster_fits(int M, int B, int C, int smem_floats)
 {

@@ -68,6 +68,7 @@ struct ScSmem {
     float *vs;      // [ldk + 4]            final V_j, V_d at [ldk]
     float *wsum;    // [16]                 per-warp sums of U
     float *xusum;   // [2][8]               per-CTA sums of U, double-buffered
+    int *toks;      // [rows_per]           token position of each of this CTA's rows (for the plan write)
 };
 
 // The iterations, for tiles of at most 32 * NC columns; Ml = this CTA's rows.  A warp takes
@@ -207,6 +208,8 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     const uint32_t C = ptx::cluster_nctarank(), rank = ptx::cluster_ctarank();
     const int img = blockIdx.x / C, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();     // the scores come from the kernel ahead
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;
@@ -227,6 +230,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     m.vs = m.us + ((rows_per + 8) & ~3);
     m.wsum = m.vs + (ldk + 4);
     m.xusum = m.wsum + kSfWarps;
+    m.toks = reinterpret_cast<int *>(m.xusum + 16);
 
     float *Sg = kmat + kmat_offset(kmat_stride, t_begin, img);
     const int ldS = score_pitch(B);
@@ -265,7 +269,10 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         }
     }
     const float v_init = expf(shift * inv_eps);       // v = 0
-    for (int i = tid; i < Ml; i += kSfThreads) m.us[i] = 1.f;     // u = 0
+    for (int i = tid; i < Ml; i += kSfThreads) {
+        m.us[i] = 1.f;                                            // u = 0
+        m.toks[i] = __ldg(order + t_begin + row_lo + i);
+    }
     // every CTA of the cluster is running and has its shared memory laid out before anyone writes into it
     ptx::cluster_sync_all();
 
@@ -374,7 +381,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         __nv_bfloat16 *Pimg = pbuf + (size_t)t_begin * pbuf_pitch;
         for (int idx = tid; idx < Ml * vpr; idx += kSfThreads) {
             const int i = idx / vpr, j0 = (idx - i * vpr) << 3;
-            const int tok = __ldg(order + t_begin + row_lo + i);
+            const int tok = m.toks[i];
             const float ui = m.us[i];
             __align__(16) float kk[8];
             __align__(16) float vv[8];

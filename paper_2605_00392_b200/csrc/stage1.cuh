@@ -243,6 +243,8 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
     __shared__ uint64_t s_full[kS1MaxStages], s_empty[kS1MaxStages];
     const int img = blockIdx.y, chunk = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();     // the workspace may still be in use by the run ahead in the stream
     int t_begin, n_img;
     const bool valid = image_range(offsets, img, max_tokens, total, t_begin, n_img);
     if (!valid) {
@@ -424,6 +426,8 @@ gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restri
                    int max_tokens, int total, __nv_bfloat16 *__restrict__ xp)
 {
     const int img = blockIdx.y;
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();     // counts and order come from the kernel ahead
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M, Bpad = (B + 63) & ~63;
