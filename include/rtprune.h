@@ -73,9 +73,11 @@ typedef struct {
     float eps;            /* entropic regularisation: Z = S-bar / eps; > 0 (1 uses S-bar itself)     */
     int32_t iters;        /* Sinkhorn iterations T, >= 0 (paper: 100)                                */
     int32_t form;         /* rtprune_sinkhorn_form_t                                                 */
-    int32_t stop_at_fixed_point; /* 1: leave the loop once an iteration returns v bit-identical to
-                             its input -- every later iteration would reproduce it, so the result is
-                             that of all `iters` iterations.  0: always run `iters` iterations.     */
+    int32_t stop_at_fixed_point; /* 1: leave the loop once an iteration reproduces its input: the duals
+                             of the scaling form all within one unit in the last place of their
+                             previous values (bit-identical log-domain duals in the LOG form) -- later
+                             iterations could only move them within rounding, so the result is that
+                             of all `iters` iterations to fp32 accuracy.  0: always run `iters`.     */
     float tol;            /* > 0: also stop once no dual moved by more than tol (log units) in an
                              iteration.  0 (default): never stop on a tolerance.                    */
 } rtprune_params_t;

@@ -22,15 +22,27 @@ constexpr int kSfMaxNc = 8;            // the one-pass kernel takes tiles of at 
 // Shared-memory floats one CTA of the cluster kernel (sinkhorn_cluster.cuh) needs for an M x B tile
 // split over C CTAs: its rows of K padded to 32-column multiples, per-warp and per-CTA partials of the
 // column sums (the same space serves the pairing), duals, scratch.
+// Row pitch (floats) of K in the cluster kernel: the widths its lane layouts cover.
+__host__ __device__ inline int sinkhorn_ldk(int B)
+{
+    return B <= 32 ? 32 : (B <= 64 ? 64 : (B <= 128 ? 128 : (B <= 192 ? 192 : 256)));
+}
 __host__ __device__ inline long long sinkhorn_cluster_floats(int M, int B, int C)
 {
-    const long long ldk = (B + 31) & ~31;
+    const long long ldk = sinkhorn_ldk(B);
     const long long rows_per = (M + C - 1) / C;
     return rows_per * ldk + 2 * kSfWarps * ldk + 2 * C * ldk + 2 * (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
 }
 __host__ __device__ inline bool sinkhorn_cluster_fits(int M, int B, int C, int smem_floats)
 {
     return B >= 1 && B <= 32 * kSfMaxNc && sinkhorn_cluster_floats(M, B, C) <= (long long)smem_floats;
+}
+
+// True if two positive floats differ by more than one unit in the last place.
+__device__ inline bool ulp_far(float a, float b)
+{
+    const int d = (int)__float_as_uint(a) - (int)__float_as_uint(b);
+    return d > 1 || d < -1;
 }
 
 __device__ inline void lse_merge(float &m, float &s, float m2, float s2)
@@ -188,7 +200,7 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
                 const float move = LOG ? fabsf(nv - ov) : fabsf(nv - ov) / fabsf(ov);
                 last_move = fmaxf(last_move, move);
                 if (p.tol > 0.f) cont |= (move > p.tol) ? 1 : 0;
-                else cont |= p.stop_fp ? (__float_as_uint(nv) != __float_as_uint(ov)) : 1;
+                else cont |= p.stop_fp ? (LOG ? (__float_as_uint(nv) != __float_as_uint(ov)) : ulp_far(nv, ov)) : 1;
                 v[j] = nv;
             }
             if (passes > 1 && G > 1) __syncthreads();

@@ -8,41 +8,18 @@
 // kappa = exp((z - c)/eps), mu = [1_M, B], nu = [1_B, M],
 //     U_i = 1 / (sum_j K_ij V_j + kappa V_d)          U_d = B / (kappa (sum_j V_j + V_d))
 //     V_j = 1 / (sum_i K_ij U_i + kappa U_d)          V_d = M / (kappa (sum_i U_i + U_d))
-// One iteration is ONE pass over K in shared memory: a warp owns a few rows at a time, its lanes own
-// the columns lane, lane + 32, ...; the row sums are reduced together across the warp, the new U_i
-// multiply the same K values (still in registers) into per-lane column accumulators; the column sums
-// are completed across the 16 warps through shared memory and across the CTAs through distributed
-// shared memory: every CTA stores its partial column sums into every CTA of the cluster, one cluster
-// barrier, and every warp of every CTA adds the C partials in the same order, so all of them hold
-// bit-identical V and take the same decision to stop.
+// One iteration is ONE pass over K in shared memory: 8 or 16 lanes share a row, the row sum is an
+// all-reduce over them, the new U_i multiplies the same K values (still in registers) into per-lane
+// column accumulators; the column sums are completed across the 16 warps through shared memory and
+// across the CTAs through distributed shared memory: every CTA stores its partial column sums into
+// every CTA of the cluster, one cluster barrier, and every CTA adds the C partials in the same order,
+// so all of them hold bit-identical V and take the same decision to stop.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
 #include "sinkhorn.cuh"
 
 namespace rtp {
-
-// Sums of R per-lane values over the warp, all R at once: afterwards lanes q*(32/R) .. (q+1)*(32/R)-1
-// hold the total of value q.  R - 1 + log2(32 / R) shuffles instead of 5 R.
-template <int R>
-__device__ inline float warp_sum_scatter(float (&p)[R], int lane)
-{
-    int off = 16;
-#pragma unroll
-    for (int n = R; n > 1; n >>= 1, off >>= 1) {
-        const bool hi = (lane & off) != 0;
-#pragma unroll
-        for (int q = 0; q < n / 2; ++q) {
-            const float keep = hi ? p[q + n / 2] : p[q];
-            const float give = hi ? p[q] : p[q + n / 2];
-            p[q] = keep + __shfl_xor_sync(0xffffffffu, give, off);
-        }
-    }
-    float r = p[0];
-#pragma unroll
-    for (; off > 0; off >>= 1) r += __shfl_xor_sync(0xffffffffu, r, off);
-    return r;
-}
 
 __device__ inline float rcp_fast(float x)
 {
@@ -71,126 +48,159 @@ struct ScSmem {
     int *toks;      // [rows_per]           token position of each of this CTA's rows (for the plan write)
 };
 
-// The iterations, for tiles of at most 32 * NC columns; Ml = this CTA's rows.  A warp takes
-// RPC = 32 / NC rows per step, so that the K values it holds in registers stay at 32 whatever the
-// tile's width.  On return every warp of every CTA holds the final V (lane's columns lane + 32 c),
-// V_d and U_d; U of this CTA's rows is in us[].
-template <int NC>
-__device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int M, int B, int nc, int ldk,
-                                                   uint32_t C, uint32_t rank, const OtParams &p, float kappa,
-                                                   float v_init, float (&V)[NC], float &Vd, float &Ud)
+// The iterations for a tile whose rows are ldk = LR * CPL floats wide; Ml = this CTA's rows.
+// Lane layout of the row pass: LR consecutive lanes share a row, a warp takes 32 / LR rows per step;
+// lane `sub` of a row owns the 16-byte column chunks sub, sub + LR, ... (CPL columns in all), so a
+// row's lanes read consecutive chunks.  The row sum is an all-reduce over the LR lanes (every lane of
+// the row then has U_i, no broadcast), the products K_ij U_i go to per-lane column accumulators, which
+// are reduced over the warp's rows at the end of the pass, over the 16 warps through shared memory,
+// and over the CTAs through distributed shared memory (one cluster barrier).  Threads 0 .. ldk-1 then
+// compute one V_j each, the same in every CTA.  On return vs[] holds the final V (V_d at [ldk]) and
+// us[] the U of this CTA's rows.
+template <int LR, int CPL>
+__device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int M, int B, uint32_t C,
+                                                   uint32_t rank, const OtParams &p, float kappa, float v_init)
 {
-    constexpr int RPC = 32 / NC;          // rows per step
-    constexpr int LPR = 32 / RPC;         // lanes that end up holding one row's total
+    constexpr int ldk = LR * CPL;
+    constexpr int RPS = 32 / LR;          // rows per step of a warp
+    constexpr int NQ = CPL / 4;           // 16-byte chunks per lane
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LR, slot = lane / LR;
     const float Bf = (float)B, Mf = (float)M;
-#pragma unroll
-    for (int c = 0; c < NC; ++c) V[c] = (c < nc && lane + 32 * c < B) ? v_init : 0.f;
-    Vd = v_init;
-    float sumV = Bf * v_init;
-    Ud = 1.f;
-    const int ngroups = (Ml + RPC - 1) / RPC;
+    __shared__ float s_vsum[kSfWarps];    // per-warp sums of V (warps 0 .. ldk/32-1)
+
+    for (int j = tid; j <= ldk; j += kSfThreads) m.vs[j] = (j < B || j == ldk) ? v_init : 0.f;
+    if (tid < kSfWarps) s_vsum[tid] = (tid == 0) ? Bf * v_init : 0.f;
+    __syncthreads();
+    const int nsteps = (Ml + RPS - 1) / RPS;
     const uint32_t xpart_u32 = ptx::smem_u32(m.xpart), xusum_u32 = ptx::smem_u32(m.xusum);
     ScState st{0, 0.f};
 
     for (int it = 0; it < p.iters; ++it) {
-        Ud = Bf * rcp_fast(kappa * (sumV + Vd));
-        const float kVd = kappa * Vd;
-        float colacc[NC];
+        // this lane's V, the dustbin terms
+        float4 V[NQ];
 #pragma unroll
-        for (int c = 0; c < NC; ++c) colacc[c] = 0.f;
+        for (int q = 0; q < NQ; ++q) V[q] = *reinterpret_cast<const float4 *>(m.vs + 4 * (q * LR + sub));
+        float sumV = 0.f;
+#pragma unroll
+        for (int w = 0; w < ldk / 32; ++w) sumV += s_vsum[w];
+        const float Vd = m.vs[ldk];
+        const float Ud = Bf * rcp_fast(kappa * (sumV + Vd));
+        const float kVd = kappa * Vd;
+        float4 colacc[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         float usum = 0.f;
 
-        for (int g = warp; g < ngroups; g += kSfWarps) {
-            const int i0 = g * RPC;
-            float k[RPC][NC];
-            float ps[RPC];
+#pragma unroll 2
+        for (int g = warp; g < nsteps; g += kSfWarps) {
+            const int i = g * RPS + slot;
+            const bool valid = i < Ml;
+            // rows past Ml repeat the last row: their values are computed and dropped
+            const float *row = m.Ks + (size_t)min(i, Ml - 1) * ldk + 4 * sub;
+            float4 k[NQ];
+            float s = 0.f;
 #pragma unroll
-            for (int r = 0; r < RPC; ++r) {
-                // rows past Ml repeat the last row: their values are computed and dropped
-                const float *row = m.Ks + (size_t)min(i0 + r, Ml - 1) * ldk + lane;
-                float s = 0.f;
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    k[r][c] = (c < nc) ? row[32 * c] : 0.f;
-                    s = fmaf(k[r][c], V[c], s);
-                }
-                ps[r] = s;
+            for (int q = 0; q < NQ; ++q) {
+                k[q] = *reinterpret_cast<const float4 *>(row + 4 * q * LR);
+                s = fmaf(k[q].x, V[q].x, s);
+                s = fmaf(k[q].y, V[q].y, s);
+                s = fmaf(k[q].z, V[q].z, s);
+                s = fmaf(k[q].w, V[q].w, s);
             }
-            const float tot = warp_sum_scatter<RPC>(ps, lane);
-            const float Unew = rcp_fast(tot + kVd);         // lanes q LPR .. : row i0 + q
-            if ((lane % LPR) == 0 && i0 + lane / LPR < Ml) m.us[i0 + lane / LPR] = Unew;
 #pragma unroll
-            for (int r = 0; r < RPC; ++r) {
-                float Ur = __shfl_sync(0xffffffffu, Unew, LPR * r);
-                Ur = (i0 + r < Ml) ? Ur : 0.f;
-                usum += Ur;
+            for (int o = 1; o < LR; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const float U = valid ? rcp_fast(s + kVd) : 0.f;
+            if (sub == 0 && valid) {
+                m.us[i] = U;
+                usum += U;
+            }
 #pragma unroll
-                for (int c = 0; c < NC; ++c) colacc[c] = fmaf(k[r][c], Ur, colacc[c]);
+            for (int q = 0; q < NQ; ++q) {
+                colacc[q].x = fmaf(k[q].x, U, colacc[q].x);
+                colacc[q].y = fmaf(k[q].y, U, colacc[q].y);
+                colacc[q].z = fmaf(k[q].z, U, colacc[q].z);
+                colacc[q].w = fmaf(k[q].w, U, colacc[q].w);
             }
         }
+        // column partials over the warp's row slots, then to shared memory (lanes of slot 0)
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
-            if (c < nc) m.part[warp * ldk + lane + 32 * c] = colacc[c];
+        for (int o = LR; o < 32; o <<= 1) {
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                colacc[q].x += __shfl_xor_sync(0xffffffffu, colacc[q].x, o);
+                colacc[q].y += __shfl_xor_sync(0xffffffffu, colacc[q].y, o);
+                colacc[q].z += __shfl_xor_sync(0xffffffffu, colacc[q].z, o);
+                colacc[q].w += __shfl_xor_sync(0xffffffffu, colacc[q].w, o);
+            }
+        }
+        if (slot == 0) {
+#pragma unroll
+            for (int q = 0; q < NQ; ++q)
+                *reinterpret_cast<float4 *>(m.part + warp * ldk + 4 * (q * LR + sub)) = colacc[q];
+        }
+        usum = warp_sum(usum);
         if (lane == 0) m.wsum[warp] = usum;
         __syncthreads();
 
         // this CTA's column sums and sum of U go to every CTA of the cluster (this one included)
-        const uint32_t slot = (uint32_t)(it & 1) * C + rank;
+        const uint32_t slot_x = (uint32_t)(it & 1) * C + rank;
         if (tid < ldk) {
             float cs = 0.f;
 #pragma unroll
             for (int w = 0; w < kSfWarps; ++w) cs += m.part[w * ldk + tid];
-            const uint32_t a = xpart_u32 + (slot * (uint32_t)ldk + (uint32_t)tid) * 4u;
+            const uint32_t a = xpart_u32 + (slot_x * (uint32_t)ldk + (uint32_t)tid) * 4u;
             for (uint32_t r = 0; r < C; ++r) ptx::st_cluster_f32(ptx::map_to_rank(a, r), cs);
         }
         if (tid == kSfThreads - 1) {
             float su = 0.f;
 #pragma unroll
             for (int w = 0; w < kSfWarps; ++w) su += m.wsum[w];
-            const uint32_t a = xusum_u32 + slot * 4u;
+            const uint32_t a = xusum_u32 + slot_x * 4u;
             for (uint32_t r = 0; r < C; ++r) ptx::st_cluster_f32(ptx::map_to_rank(a, r), su);
         }
         ptx::cluster_sync_all();
 
-        // ---- V from the completed column sums, in every warp of every CTA alike ----------------------
+        // ---- V from the completed column sums: one thread per column, the same in every CTA ----------
         const float *xb = m.xpart + (size_t)(it & 1) * C * ldk;
         const float *ub = m.xusum + (it & 1) * C;
-        float cs[NC];
-#pragma unroll
-        for (int c = 0; c < NC; ++c) cs[c] = 0.f;
-        float su = 0.f;
-        for (uint32_t r = 0; r < C; ++r) {
-#pragma unroll
-            for (int c = 0; c < NC; ++c)
-                if (c < nc) cs[c] += xb[r * ldk + lane + 32 * c];
-            su += ub[r];
+        int cont = 0;
+        float move = 0.f;
+        if (tid < ldk) {
+            float nv = 0.f;
+            if (tid < B) {
+                float cs = 0.f;
+                for (uint32_t r = 0; r < C; ++r) cs += xb[r * ldk + tid];
+                nv = rcp_fast(cs + kappa * Ud);
+                const float ov = m.vs[tid];
+                move = fabsf(nv - ov) * rcp_fast(ov);
+                cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
+                m.vs[tid] = nv;
+            }
+            const float wv = warp_sum(nv);            // warps 0 .. ldk/32-1 lie entirely inside tid < ldk
+            if (lane == 0) s_vsum[warp] = wv;
         }
-        const float kUd = kappa * Ud;
-        bool changed = false;
-        float move = 0.f, sv = 0.f;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            const bool real = c < nc && lane + 32 * c < B;
-            const float nv = real ? rcp_fast(cs[c] + kUd) : 0.f;
-            changed |= __float_as_uint(nv) != __float_as_uint(V[c]);
-            if (real) move = fmaxf(move, fabsf(nv - V[c]) * rcp_fast(V[c]));
-            V[c] = nv;
-            sv += nv;
+        if (tid == kSfThreads - 1) {                  // the dustbin column
+            float su = 0.f;
+            for (uint32_t r = 0; r < C; ++r) su += ub[r];
+            const float nVd = Mf * rcp_fast(kappa * (su + Ud));
+            move = fabsf(nVd - Vd) * rcp_fast(Vd);
+            cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : 1);
+            m.vs[ldk] = nVd;
         }
-        const float nVd = Mf * rcp_fast(kappa * (su + Ud));
-        changed |= __float_as_uint(nVd) != __float_as_uint(Vd);
-        move = fmaxf(move, fabsf(nVd - Vd) * rcp_fast(Vd));
-        Vd = nVd;
-        sumV = warp_sum(sv);
         st.last_move = move;
         ++st.done;
-        bool cont;
-        if (p.tol > 0.f) cont = __any_sync(0xffffffffu, move > p.tol);
-        else cont = p.stop_fp ? __any_sync(0xffffffffu, changed) : true;
-        if (!cont) break;
+        if (!__syncthreads_or(cont)) break;
     }
-    st.last_move = warp_max(st.last_move);
+    // largest relative dual move of the last executed iteration, over the CTA
+    float mv = warp_max(st.last_move);
+    __syncthreads();
+    if (lane == 0) s_vsum[warp] = mv;
+    __syncthreads();
+    mv = 0.f;
+#pragma unroll
+    for (int w = 0; w < kSfWarps; ++w) mv = fmaxf(mv, s_vsum[w]);
+    st.last_move = mv;
     return st;
 }
 
@@ -217,8 +227,8 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     const int out0 = out_offsets[img];
     const int my_prop = (rank == 0 && tid < B) ? order[t_begin + M + tid] : 0;   // needed at the end
 
-    const int nc = (B + 31) >> 5;
-    const int ldk = nc << 5;
+    const int ldk = sinkhorn_ldk(B);
+    const int nc = ldk >> 5;
     const int rows_per = (M + (int)C - 1) / (int)C;
     const int row_lo = min(M, (int)rank * rows_per);
     const int Ml = min(M, row_lo + rows_per) - row_lo;       // this CTA's rows (may be 0)
@@ -237,6 +247,8 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     const float inv_eps = 1.f / p.eps;
     const float shift = fmaxf(1.f, p.z);
     const float kappa = expf((p.z - shift) * inv_eps);
+
+    for (int i = tid; i < Ml; i += kSfThreads) m.toks[i] = __ldg(order + t_begin + row_lo + i);
 
     // ---- K = exp((S - c)/eps) of this CTA's rows, zero beyond column B ------------------------------
     {
@@ -269,46 +281,21 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         }
     }
     const float v_init = expf(shift * inv_eps);       // v = 0
-    for (int i = tid; i < Ml; i += kSfThreads) {
-        m.us[i] = 1.f;                                            // u = 0
-        m.toks[i] = __ldg(order + t_begin + row_lo + i);
-    }
+    for (int i = tid; i < Ml; i += kSfThreads) m.us[i] = 1.f;     // u = 0
     // every CTA of the cluster is running and has its shared memory laid out before anyone writes into it
     ptx::cluster_sync_all();
 
     // ---- the iterations --------------------------------------------------------------------------------
     ScState st;
-    float Vd, Ud;
-    if (nc <= 2) {
-        float V[2];
-        st = sinkhorn_cluster_iterate<2>(m, Ml, M, B, nc, ldk, C, rank, p, kappa, v_init, V, Vd, Ud);
-        if (warp == 0) {
-#pragma unroll
-            for (int c = 0; c < 2; ++c) if (c < nc) m.vs[lane + 32 * c] = V[c];
-        }
-    } else if (nc <= 4) {
-        float V[4];
-        st = sinkhorn_cluster_iterate<4>(m, Ml, M, B, nc, ldk, C, rank, p, kappa, v_init, V, Vd, Ud);
-        if (warp == 0) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) if (c < nc) m.vs[lane + 32 * c] = V[c];
-        }
-    } else {
-        float V[8];
-        st = sinkhorn_cluster_iterate<8>(m, Ml, M, B, nc, ldk, C, rank, p, kappa, v_init, V, Vd, Ud);
-        if (warp == 0) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) if (c < nc) m.vs[lane + 32 * c] = V[c];
-        }
+    if (ldk == 32) st = sinkhorn_cluster_iterate<8, 4>(m, Ml, M, B, C, rank, p, kappa, v_init);
+    else if (ldk == 64) st = sinkhorn_cluster_iterate<8, 8>(m, Ml, M, B, C, rank, p, kappa, v_init);
+    else if (ldk == 128) st = sinkhorn_cluster_iterate<8, 16>(m, Ml, M, B, C, rank, p, kappa, v_init);
+    else if (ldk == 192) st = sinkhorn_cluster_iterate<16, 12>(m, Ml, M, B, C, rank, p, kappa, v_init);
+    else st = sinkhorn_cluster_iterate<16, 16>(m, Ml, M, B, C, rank, p, kappa, v_init);
+    if (tid == 0 && rank == 0) {
+        stats[(size_t)img * kStats + 5] = (float)st.done;
+        stats[(size_t)img * kStats + 6] = st.last_move;
     }
-    if (tid == 0) {
-        m.vs[ldk] = Vd;
-        if (rank == 0) {
-            stats[(size_t)img * kStats + 5] = (float)st.done;
-            stats[(size_t)img * kStats + 6] = st.last_move;
-        }
-    }
-    (void)Ud;
     // nobody reads xpart any more (it is reused below), and vs is visible to the CTA
     ptx::cluster_sync_all();
 

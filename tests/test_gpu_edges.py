@@ -73,12 +73,20 @@ def test_ot_parameter_ranges(parity, over):
 
 
 def test_fixed_point_stop_equals_all_iterations(parity):
+    # leaving the loop at the fixed point (duals within one unit in the last place) must give what all
+    # 100 iterations give, to fp32 accuracy: same pairs, weights and features equal to a few ulps
     w = synth.make("base", batch=6)
     a = parity.run_gpu(w, overrides=dict(stop_at_fixed_point=1)).out
     b = parity.run_gpu(w, overrides=dict(stop_at_fixed_point=0)).out
-    assert torch.equal(a.Y, b.Y) and torch.equal(a.merge_partner, b.merge_partner)
-    assert torch.equal(a.merge_weight, b.merge_weight)
-    assert float(b.stats[:6, 5].min()) == 100.0 and float(a.stats[:6, 5].max()) <= 100.0
+    assert torch.equal(a.kept_idx, b.kept_idx) and torch.equal(a.merged_idx, b.merged_idx)
+    n = int(a.out_offsets[6])
+    nb = int(w.offsets[6]) - n
+    assert torch.equal(a.merge_partner[:nb], b.merge_partner[:nb])
+    torch.testing.assert_close(a.merge_weight[:nb], b.merge_weight[:nb], rtol=2e-6, atol=0)
+    ya, yb = a.Y[:n].float(), b.Y[:n].float()
+    assert (ya - yb).abs().max() <= 2.0 ** -8 * yb.abs().max()      # at most one bf16 rounding apart
+    assert (ya != yb).float().mean() < 1e-3
+    assert float(b.stats[:6, 5].min()) == 100.0 and float(a.stats[:6, 5].max()) < 40.0
 
 
 def test_tolerance_stop_runs_fewer_iterations(parity):
