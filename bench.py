@@ -211,6 +211,7 @@ def main() -> None:
     # ---- timed region: K steps back to back, CUDA events on the launching stream ------------------
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    torch.cuda._sleep(2000000)     # about 1 ms: the host is ahead of the device when the timed region starts
     e0.record(stream)
     for i in range(args.steps):
         step(i)
@@ -224,6 +225,7 @@ def main() -> None:
     per_kernel = {}
     nprof = min(args.steps, 50)
     for i in range(nprof):
+        torch.cuda._sleep(300000)      # the host gets ahead: no launch gaps inside the measured kernels
         step(i)
         for name, ms in plan.profile_read():
             per_kernel.setdefault(name, []).append(ms)
@@ -272,12 +274,14 @@ def main() -> None:
         dominant = max(avg, key=avg.get)
         x_bytes = total * d * esz
         y_bytes = sumM * d * esz
+        sink_flops = float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))
+        xp_bytes = int(B.sum()) * d * esz
         algo = {   # algorithmic bytes / flops per launch, by kernel
-            "norm_stats": ("hbm", x_bytes + total * 4),
-            "select": ("hbm", total * 4 * 2 + batch * 48),
-            "scores": ("alu", 2.0 * sumMB * d),
-            "sinkhorn": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
-            "sinkhorn_cluster": ("alu", float(np.sum(iters_run * 2 * 2 * (M + 1) * (B + 1)))),
+            "stage1": ("hbm", x_bytes + total * 4 * 3 + batch * 48),
+            "gather": ("hbm", 2 * xp_bytes),
+            "scores": ("hbm", x_bytes + xp_bytes + 4 * sumMB),
+            "sinkhorn_cluster": ("alu", sink_flops),
+            "sinkhorn": ("alu", sink_flops),
             "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
         }
         bound, units = algo[dominant]
@@ -294,7 +298,7 @@ def main() -> None:
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "tokens_per_s": images_s * total / batch,
             "config": {"workload": WORKLOAD_DESC, "global_batch": world * batch,
-                       "accumulate": "fp32", "sinkhorn": "T=100 with exit at the bitwise fixed point",
+                       "accumulate": "fp32", "sinkhorn": "T=100 with exit at the fixed point (no dual moves by more than 1 ulp)",
                        "mean_iterations_run": float(iters_run.mean()),
                        "mean_retention": float(sumM) / total,
                        "l2": "inputs and outputs rotate over %d buffer sets (%.0f MB > L2)"
