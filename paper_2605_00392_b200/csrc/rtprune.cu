@@ -350,12 +350,21 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
         bool all_fast = false;
         if (!use_log_form(params)) {
-            // CTAs per image: as many as keep the whole batch on the chip at once, 8 at most
+            // CTAs per image: as many as keep the whole batch on the chip at once, and at least as many
+            // as the largest possible tile needs to fit their shared memory; 8 at most
             fast_c = 1;
             while (fast_c < 8 && (long long)batch * fast_c * 2 <= plan->sm_count) fast_c *= 2;
-            all_fast = maxB <= 32 * kSfMaxNc;
-            for (int b = 1; b <= maxB && all_fast; ++b)
-                all_fast = sinkhorn_cluster_fits(std::max(maxN - b, 1), b, fast_c, fast_floats);
+            auto fits_all = [&](int cc) {
+                bool ok = maxB <= 32 * kSfMaxNc;
+                for (int b = 1; b <= maxB && ok; ++b)
+                    ok = sinkhorn_cluster_fits(std::max(maxN - b, 1), b, cc, fast_floats);
+                return ok;
+            };
+            all_fast = fits_all(fast_c);
+            while (!all_fast && fast_c < 8 && maxB <= 32 * kSfMaxNc) {
+                fast_c *= 2;
+                all_fast = fits_all(fast_c);
+            }
             if (!c.ok(launch_pdl(sinkhorn_cluster_kernel, dim3((unsigned)(batch * fast_c)), dim3(kSfThreads),
                                  (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets, o.counts,
                                  o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op, fast_floats, pbuf,
