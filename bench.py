@@ -282,6 +282,7 @@ def main() -> None:
             "gather": ("hbm", 2 * xp_bytes),
             "scores": ("hbm", x_bytes + xp_bytes + 4 * sumMB),
             "sinkhorn_cluster": ("alu", sink_flops),
+            "sinkhorn_wide": ("alu", sink_flops),
             "sinkhorn": ("alu", sink_flops),
             "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
         }

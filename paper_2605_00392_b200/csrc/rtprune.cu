@@ -344,33 +344,45 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         OtParams op{params->z, params->alpha, params->eps, params->iters,
                     params->stop_at_fixed_point, params->tol};
         const int smem_floats = plan->sink_smem_bytes / (int)sizeof(float);
-        // Scaling form: tiles that fit one CTA's shared memory go to the one-pass kernel; the general
+        // Scaling form: the cluster kernel takes every tile of up to 32 * kSfMaxNc columns; the general
         // kernel then takes what is left (it skips the images already solved).
         int fast_c = 0;
         const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
         bool all_fast = false;
         if (!use_log_form(params)) {
             // CTAs per image: as many as keep the whole batch on the chip at once, and at least as many
-            // as the largest possible tile needs to fit their shared memory; 8 at most
+            // as the largest possible tile needs to keep K in their shared memory; 8 at most (tiles
+            // larger than that iterate on K in the workspace)
             fast_c = 1;
             while (fast_c < 8 && (long long)batch * fast_c * 2 <= plan->sm_count) fast_c *= 2;
-            auto fits_all = [&](int cc) {
+            auto all_tiles = [&](int cc, bool in_smem) {
                 bool ok = maxB <= 32 * kSfMaxNc;
-                for (int b = 1; b <= maxB && ok; ++b)
-                    ok = sinkhorn_cluster_fits(std::max(maxN - b, 1), b, cc, fast_floats);
+                for (int b = 1; b <= maxB && ok; ++b) {
+                    const int m = std::max(maxN - b, 1);
+                    ok = in_smem ? sinkhorn_cluster_fits(m, b, cc, fast_floats)
+                                 : sinkhorn_cluster_handles(m, b, cc, fast_floats);
+                }
                 return ok;
             };
-            all_fast = fits_all(fast_c);
-            while (!all_fast && fast_c < 8 && maxB <= 32 * kSfMaxNc) {
-                fast_c *= 2;
-                all_fast = fits_all(fast_c);
-            }
-            if (!c.ok(launch_pdl(sinkhorn_cluster_kernel, dim3((unsigned)(batch * fast_c)), dim3(kSfThreads),
-                                 (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets, o.counts,
-                                 o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op, fast_floats, pbuf,
-                                 pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats)))
+            while (fast_c < 8 && !all_tiles(fast_c, true)) fast_c *= 2;
+            all_fast = all_tiles(fast_c, false);
+            if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<false>, dim3((unsigned)(batch * fast_c)),
+                                 dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets,
+                                 o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
+                                 fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
+                                 o.stats)))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_cluster");
+            // tiles wider than 256 columns, or too tall for the cluster's shared memory
+            if (maxB > 256 || !all_tiles(fast_c, true)) {
+                if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<true>, dim3((unsigned)(batch * fast_c)),
+                                     dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c,
+                                     offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total,
+                                     op, fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
+                                     o.merge_weight, o.stats)))
+                    return RTPRUNE_ERR_CUDA;
+                launched(plan, st, "sinkhorn_wide");
+            }
         }
         if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
@@ -548,7 +560,9 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         return RTPRUNE_ERR_CUDA;
     }
     p->fast_smem_bytes = (int)(cap / 16 * 16);
-    if (!c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (!c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   p->fast_smem_bytes)) ||
+        !c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    p->fast_smem_bytes))) {
         delete p;
         return RTPRUNE_ERR_CUDA;

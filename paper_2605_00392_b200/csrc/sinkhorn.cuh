@@ -17,25 +17,39 @@ constexpr int kSinkThreads = 512;
 
 constexpr int kSfThreads = 512;
 constexpr int kSfWarps = kSfThreads / 32;
-constexpr int kSfMaxNc = 8;            // the one-pass kernel takes tiles of at most 32 * 8 columns
+constexpr int kSfMaxNc = 20;           // the cluster kernel takes tiles of at most 32 * 20 columns
 
-// Shared-memory floats one CTA of the cluster kernel (sinkhorn_cluster.cuh) needs for an M x B tile
-// split over C CTAs: its rows of K padded to 32-column multiples, per-warp and per-CTA partials of the
-// column sums (the same space serves the pairing), duals, scratch.
-// Row pitch (floats) of K in the cluster kernel: the widths its lane layouts cover.
+// Row pitch (floats) of K in the cluster kernel (sinkhorn_cluster.cuh): the widths its lane layouts cover.
 __host__ __device__ inline int sinkhorn_ldk(int B)
 {
-    return B <= 32 ? 32 : (B <= 64 ? 64 : (B <= 128 ? 128 : (B <= 192 ? 192 : 256)));
+    if (B <= 128) return B <= 32 ? 32 : (B <= 64 ? 64 : 128);
+    if (B <= 256) return B <= 192 ? 192 : 256;
+    return B <= 384 ? 384 : (B <= 512 ? 512 : 640);
 }
-__host__ __device__ inline long long sinkhorn_cluster_floats(int M, int B, int C)
+// Shared-memory floats one CTA of the cluster kernel needs for an M x B tile split over C CTAs, K
+// aside: per-warp and per-CTA partials of the column sums (the same space serves the pairing), duals,
+// token positions, scratch.
+__host__ __device__ inline long long sinkhorn_cluster_aux_floats(int M, int B, int C)
 {
     const long long ldk = sinkhorn_ldk(B);
     const long long rows_per = (M + C - 1) / C;
-    return rows_per * ldk + 2 * kSfWarps * ldk + 2 * C * ldk + 2 * (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
+    return 2 * kSfWarps * ldk + 2 * C * ldk + 2 * (rows_per + 8) + (ldk + 4) + kSfWarps + 16 + 16;
 }
+// The same with the CTA's rows of K (padded to the pitch) in shared memory too.
+__host__ __device__ inline long long sinkhorn_cluster_floats(int M, int B, int C)
+{
+    const long long rows_per = (M + C - 1) / C;
+    return rows_per * sinkhorn_ldk(B) + sinkhorn_cluster_aux_floats(M, B, C);
+}
+// K fits the cluster's shared memory.
 __host__ __device__ inline bool sinkhorn_cluster_fits(int M, int B, int C, int smem_floats)
 {
     return B >= 1 && B <= 32 * kSfMaxNc && sinkhorn_cluster_floats(M, B, C) <= (long long)smem_floats;
+}
+// The cluster kernel solves the tile: with K in shared memory if it fits, else in the workspace tile.
+__host__ __device__ inline bool sinkhorn_cluster_handles(int M, int B, int C, int smem_floats)
+{
+    return B >= 1 && B <= 32 * kSfMaxNc && sinkhorn_cluster_aux_floats(M, B, C) <= (long long)smem_floats;
 }
 
 // True if two positive floats differ by more than one unit in the last place.
@@ -84,8 +98,8 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;
     if (B == 0) return;
-    // images whose tile fits the cluster kernel launched before this one were solved there
-    if (fast_cluster > 0 && sinkhorn_cluster_fits(M, B, fast_cluster, fast_smem_floats)) return;
+    // images the cluster kernel launched before this one takes were solved there
+    if (fast_cluster > 0 && sinkhorn_cluster_handles(M, B, fast_cluster, fast_smem_floats)) return;
     const int R = M + 1, Cc = B + 1;
 
     float *u = sm;

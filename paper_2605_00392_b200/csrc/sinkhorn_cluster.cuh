@@ -1,6 +1,8 @@
-// Dustbin-augmented optimal transport by Sinkhorn iterations (Eq. 5, Appendix C) in scaling form, for
-// score tiles that fit the shared memory of one thread-block cluster: the rows (kept tokens) of an
-// image's tile are split over the C CTAs of a cluster, C = 1, 2, 4 or 8.
+// Dustbin-augmented optimal transport by Sinkhorn iterations (Eq. 5, Appendix C) in scaling form, one
+// thread-block cluster per image: the rows (kept tokens) of an image's score tile are split over the
+// C CTAs of a cluster, C = 1, 2, 4 or 8.  Tiles of up to 640 pruned tokens are taken; K stays in the
+// cluster's shared memory when it fits there, else it is built in place in the image's workspace
+// tile and read through L2 in every iteration.
 //
 // The duals are carried as U = e^u, V = e^{v + c/eps} against K_ij = exp((S_ij - c)/eps), c = max(1, z),
 // so that U_i K_ij V_j = exp(Z_ij + u_i + v_j) (Appendix C) after any number of iterations.  The
@@ -8,7 +10,7 @@
 // kappa = exp((z - c)/eps), mu = [1_M, B], nu = [1_B, M],
 //     U_i = 1 / (sum_j K_ij V_j + kappa V_d)          U_d = B / (kappa (sum_j V_j + V_d))
 //     V_j = 1 / (sum_i K_ij U_i + kappa U_d)          V_d = M / (kappa (sum_i U_i + U_d))
-// One iteration is ONE pass over K in shared memory: 8 or 16 lanes share a row, the row sum is an
+// One iteration is ONE pass over K: 8, 16 or 32 lanes share a row, the row sum is an
 // all-reduce over them, the new U_i multiplies the same K values (still in registers) into per-lane
 // column accumulators; the column sums are completed across the 16 warps through shared memory and
 // across the CTAs through distributed shared memory: every CTA stores its partial column sums into
@@ -38,7 +40,8 @@ struct ScState {
 
 // Shared-memory regions of one CTA of the cluster kernel.
 struct ScSmem {
-    float *Ks;      // [rows_per][ldk]      this CTA's rows of K
+    int ldr;        // pitch of K's rows: ldk in shared memory, the tile's pitch in the workspace
+    float *Ks;      // [rows_per][ldr]      this CTA's rows of K (shared memory, or the workspace tile)
     float *part;    // [2][16][ldk]         per-warp column partials; pairing values and indices
     float *xpart;   // [2][C][ldk]          per-CTA column partials, double-buffered by iteration parity
     float *us;      // [rows_per + 1]       U of this CTA's rows
@@ -54,16 +57,23 @@ struct ScSmem {
 // row's lanes read consecutive chunks.  The row sum is an all-reduce over the LR lanes (every lane of
 // the row then has U_i, no broadcast), the products K_ij U_i go to per-lane column accumulators, which
 // are reduced over the warp's rows at the end of the pass, over the 16 warps through shared memory,
-// and over the CTAs through distributed shared memory (one cluster barrier).  Threads 0 .. ldk-1 then
-// compute one V_j each, the same in every CTA.  On return vs[] holds the final V (V_d at [ldk]) and
+// and over the CTAs through distributed shared memory (one cluster barrier).  The threads then
+// compute one V_j each (two for B > 512), the same in every CTA.  On return vs[] holds the final V (V_d at [ldk]) and
 // us[] the U of this CTA's rows.
-template <int LR, int CPL>
+template <int LR, int CPL, bool KGLOBAL>
 __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int M, int B, uint32_t C,
                                                    uint32_t rank, const OtParams &p, float kappa, float v_init)
 {
     constexpr int ldk = LR * CPL;
+    // K's rows: in shared memory (pitch ldk, zero from column B on) or, KGLOBAL, for tiles too large
+    // for it, in the image's workspace tile (pitch m.ldr, which is also how many columns exist there;
+    // zero from column B on)
+    const float *Kbase = m.Ks;
+    const int ldr = KGLOBAL ? m.ldr : ldk;
     constexpr int RPS = 32 / LR;          // rows per step of a warp
     constexpr int NQ = CPL / 4;           // 16-byte chunks per lane
+    constexpr bool kOneColumn = ldk <= kSfThreads;                 // a thread per column is enough
+    constexpr int kVWarps = kOneColumn ? ldk / 32 : kSfWarps;      // warps that hold sums of V
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LR, slot = lane / LR;
     const float Bf = (float)B, Mf = (float)M;
@@ -83,7 +93,7 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
         for (int q = 0; q < NQ; ++q) V[q] = *reinterpret_cast<const float4 *>(m.vs + 4 * (q * LR + sub));
         float sumV = 0.f;
 #pragma unroll
-        for (int w = 0; w < ldk / 32; ++w) sumV += s_vsum[w];
+        for (int w = 0; w < kVWarps; ++w) sumV += s_vsum[w];
         const float Vd = m.vs[ldk];
         const float Ud = Bf * rcp_fast(kappa * (sumV + Vd));
         const float kVd = kappa * Vd;
@@ -97,12 +107,16 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
             const int i = g * RPS + slot;
             const bool valid = i < Ml;
             // rows past Ml repeat the last row: their values are computed and dropped
-            const float *row = m.Ks + (size_t)min(i, Ml - 1) * ldk + 4 * sub;
+            const float *row = Kbase + (size_t)min(i, Ml - 1) * ldr + 4 * sub;
             float4 k[NQ];
             float s = 0.f;
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
-                k[q] = *reinterpret_cast<const float4 *>(row + 4 * q * LR);
+                if constexpr (KGLOBAL)
+                    k[q] = (4 * (q * LR + sub) < ldr) ? __ldcg(reinterpret_cast<const float4 *>(row + 4 * q * LR))
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                else
+                    k[q] = *reinterpret_cast<const float4 *>(row + 4 * q * LR);
                 s = fmaf(k[q].x, V[q].x, s);
                 s = fmaf(k[q].y, V[q].y, s);
                 s = fmaf(k[q].z, V[q].z, s);
@@ -145,11 +159,11 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
 
         // this CTA's column sums and sum of U go to every CTA of the cluster (this one included)
         const uint32_t slot_x = (uint32_t)(it & 1) * C + rank;
-        if (tid < ldk) {
+        for (int j = tid; j < ldk; j += kSfThreads) {       // one trip when ldk <= the thread count
             float cs = 0.f;
 #pragma unroll
-            for (int w = 0; w < kSfWarps; ++w) cs += m.part[w * ldk + tid];
-            const uint32_t a = xpart_u32 + (slot_x * (uint32_t)ldk + (uint32_t)tid) * 4u;
+            for (int w = 0; w < kSfWarps; ++w) cs += m.part[w * ldk + j];
+            const uint32_t a = xpart_u32 + (slot_x * (uint32_t)ldk + (uint32_t)j) * 4u;
             for (uint32_t r = 0; r < C; ++r) ptx::st_cluster_f32(ptx::map_to_rank(a, r), cs);
         }
         if (tid == kSfThreads - 1) {
@@ -166,26 +180,44 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
         const float *ub = m.xusum + (it & 1) * C;
         int cont = 0;
         float move = 0.f;
-        if (tid < ldk) {
-            float nv = 0.f;
-            if (tid < B) {
-                float cs = 0.f;
-                for (uint32_t r = 0; r < C; ++r) cs += xb[r * ldk + tid];
-                nv = rcp_fast(cs + kappa * Ud);
-                const float ov = m.vs[tid];
-                move = fabsf(nv - ov) * rcp_fast(ov);
-                cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
-                m.vs[tid] = nv;
+        if constexpr (kOneColumn) {
+            if (tid < ldk) {
+                float nv = 0.f;
+                if (tid < B) {
+                    float cs = 0.f;
+                    for (uint32_t r = 0; r < C; ++r) cs += xb[r * ldk + tid];
+                    nv = rcp_fast(cs + kappa * Ud);
+                    const float ov = m.vs[tid];
+                    move = fabsf(nv - ov) * rcp_fast(ov);
+                    cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
+                    m.vs[tid] = nv;
+                }
+                const float wv = warp_sum(nv);        // warps 0 .. ldk/32-1 lie entirely inside tid < ldk
+                if (lane == 0) s_vsum[warp] = wv;
             }
-            const float wv = warp_sum(nv);            // warps 0 .. ldk/32-1 lie entirely inside tid < ldk
-            if (lane == 0) s_vsum[warp] = wv;
+        } else {
+            float sv = 0.f;
+            for (int j = tid; j < B; j += kSfThreads) {
+                float cs = 0.f;
+                for (uint32_t r = 0; r < C; ++r) cs += xb[r * ldk + j];
+                const float nv = rcp_fast(cs + kappa * Ud);
+                const float ov = m.vs[j];
+                const float mj = fabsf(nv - ov) * rcp_fast(ov);
+                move = fmaxf(move, mj);
+                cont |= p.tol > 0.f ? (mj > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
+                m.vs[j] = nv;
+                sv += nv;
+            }
+            sv = warp_sum(sv);
+            if (lane == 0) s_vsum[warp] = sv;
         }
         if (tid == kSfThreads - 1) {                  // the dustbin column
             float su = 0.f;
             for (uint32_t r = 0; r < C; ++r) su += ub[r];
             const float nVd = Mf * rcp_fast(kappa * (su + Ud));
-            move = fabsf(nVd - Vd) * rcp_fast(Vd);
-            cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : 1);
+            const float mj = fabsf(nVd - Vd) * rcp_fast(Vd);
+            move = fmaxf(move, mj);
+            cont |= p.tol > 0.f ? (mj > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : 1);
             m.vs[ldk] = nVd;
         }
         st.last_move = move;
@@ -206,6 +238,9 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
 
 // grid = batch * C CTAs, clusters of C along x: CTA rank r of cluster i owns rows r*rows_per .. of
 // image i's tile.  Every early return below depends on the image only, so a cluster leaves as a whole.
+// Two instances share the work: WIDE = false takes the tiles of up to 256 columns that fit shared
+// memory (the common case, kept free of everything the others need), WIDE = true the rest.
+template <bool WIDE>
 __global__ void __launch_bounds__(kSfThreads, 1)
 sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__ counts,
                         const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ order,
@@ -223,18 +258,23 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;
-    if (B == 0 || !sinkhorn_cluster_fits(M, B, (int)C, smem_floats)) return;   // the general kernel takes it
-    const int out0 = out_offsets[img];
-    const int my_prop = (rank == 0 && tid < B) ? order[t_begin + M + tid] : 0;   // needed at the end
-
+    if (B == 0 || !sinkhorn_cluster_handles(M, B, (int)C, smem_floats)) return;   // the general kernel takes it
+    const bool in_smem = sinkhorn_cluster_fits(M, B, (int)C, smem_floats);
     const int ldk = sinkhorn_ldk(B);
+    if ((in_smem && ldk <= 256) == WIDE) return;             // the other instance's tile
+    const int out0 = out_offsets[img];
     const int nc = ldk >> 5;
     const int rows_per = (M + (int)C - 1) / (int)C;
     const int row_lo = min(M, (int)rank * rows_per);
     const int Ml = min(M, row_lo + rows_per) - row_lo;       // this CTA's rows (may be 0)
+    float *Sg = kmat + kmat_offset(kmat_stride, t_begin, img);
+    const int ldS = score_pitch(B);
+    // K of this CTA's rows: in shared memory when the tile fits the cluster, else in place in the
+    // workspace tile (read through L2 every iteration)
     ScSmem m;
-    m.Ks = sm;
-    m.part = m.Ks + (size_t)rows_per * ldk;
+    m.Ks = (!WIDE || in_smem) ? sm : Sg + (size_t)row_lo * ldS;
+    m.ldr = (!WIDE || in_smem) ? ldk : ldS;
+    m.part = (!WIDE || in_smem) ? sm + (size_t)rows_per * ldk : sm;
     m.xpart = m.part + 2 * kSfWarps * ldk;
     m.us = m.xpart + 2 * C * ldk;
     m.vs = m.us + ((rows_per + 8) & ~3);
@@ -242,8 +282,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     m.xusum = m.wsum + kSfWarps;
     m.toks = reinterpret_cast<int *>(m.xusum + 16);
 
-    float *Sg = kmat + kmat_offset(kmat_stride, t_begin, img);
-    const int ldS = score_pitch(B);
+    const int ldr = m.ldr;
     const float inv_eps = 1.f / p.eps;
     const float shift = fmaxf(1.f, p.z);
     const float kappa = expf((p.z - shift) * inv_eps);
@@ -252,7 +291,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
 
     // ---- K = exp((S - c)/eps) of this CTA's rows, zero beyond column B ------------------------------
     {
-        const int qpr = ldk >> 2;                     // float4 per row of Ks
+        const int qpr = ldr >> 2;                     // float4 per row of K
         const int total_q = Ml * qpr;
         for (int q0 = tid; q0 < total_q; q0 += kSfThreads * 4) {
             float4 s[4];
@@ -275,7 +314,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                     k.y = (jj[a] + 1 < B) ? exp_fast((s[a].y - shift) * inv_eps) : 0.f;
                     k.z = (jj[a] + 2 < B) ? exp_fast((s[a].z - shift) * inv_eps) : 0.f;
                     k.w = (jj[a] + 3 < B) ? exp_fast((s[a].w - shift) * inv_eps) : 0.f;
-                    *reinterpret_cast<float4 *>(m.Ks + (size_t)ii[a] * ldk + jj[a]) = k;
+                    *reinterpret_cast<float4 *>(m.Ks + (size_t)ii[a] * ldr + jj[a]) = k;
                 }
             }
         }
@@ -287,11 +326,32 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
 
     // ---- the iterations --------------------------------------------------------------------------------
     ScState st;
-    if (ldk == 32) st = sinkhorn_cluster_iterate<8, 4>(m, Ml, M, B, C, rank, p, kappa, v_init);
-    else if (ldk == 64) st = sinkhorn_cluster_iterate<8, 8>(m, Ml, M, B, C, rank, p, kappa, v_init);
-    else if (ldk == 128) st = sinkhorn_cluster_iterate<8, 16>(m, Ml, M, B, C, rank, p, kappa, v_init);
-    else if (ldk == 192) st = sinkhorn_cluster_iterate<16, 12>(m, Ml, M, B, C, rank, p, kappa, v_init);
-    else st = sinkhorn_cluster_iterate<16, 16>(m, Ml, M, B, C, rank, p, kappa, v_init);
+#define RTP_SC_SMEM(LR, CPL) st = sinkhorn_cluster_iterate<LR, CPL, false>(m, Ml, M, B, C, rank, p, kappa, v_init)
+#define RTP_SC_GLOBAL(LR, CPL) st = sinkhorn_cluster_iterate<LR, CPL, true>(m, Ml, M, B, C, rank, p, kappa, v_init)
+#define RTP_SC_EITHER(LR, CPL)                                                                            \
+    if (in_smem) RTP_SC_SMEM(LR, CPL);                                                                    \
+    else RTP_SC_GLOBAL(LR, CPL)
+    if constexpr (!WIDE) {
+        if (ldk == 32) RTP_SC_SMEM(8, 4);
+        else if (ldk == 64) RTP_SC_SMEM(8, 8);
+        else if (ldk == 128) RTP_SC_SMEM(8, 16);
+        else if (ldk == 192) RTP_SC_SMEM(16, 12);
+        else RTP_SC_SMEM(16, 16);
+    } else {
+        switch (ldk) {
+        case 32: RTP_SC_GLOBAL(8, 4); break;
+        case 64: RTP_SC_GLOBAL(8, 8); break;
+        case 128: RTP_SC_GLOBAL(8, 16); break;
+        case 192: RTP_SC_GLOBAL(16, 12); break;
+        case 256: RTP_SC_GLOBAL(16, 16); break;
+        case 384: RTP_SC_EITHER(32, 12); break;
+        case 512: RTP_SC_EITHER(32, 16); break;
+        default: RTP_SC_EITHER(32, 20); break;
+        }
+    }
+#undef RTP_SC_SMEM
+#undef RTP_SC_GLOBAL
+#undef RTP_SC_EITHER
     if (tid == 0 && rank == 0) {
         stats[(size_t)img * kStats + 5] = (float)st.done;
         stats[(size_t)img * kStats + 6] = st.last_move;
@@ -309,9 +369,11 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
             const bool two = cb + 1 < nc;
             for (int i = warp; i < Ml; i += kSfWarps) {
                 const float ui = m.us[i];
-                const float *row = m.Ks + (size_t)i * ldk + lane + 32 * cb;
-                const float k0 = row[0] * ui;
-                const float k1 = two ? row[32] * ui : -INFINITY;
+                // columns past the row's end (workspace tile narrower than ldk) are past B: never read back
+                const int c0 = lane + 32 * cb;
+                const float *row = m.Ks + (size_t)i * ldr + c0;
+                const float k0 = (c0 < ldr) ? row[0] * ui : 0.f;
+                const float k1 = two ? ((c0 + 32 < ldr) ? row[32] * ui : 0.f) : -INFINITY;
                 if (k0 > best0) { best0 = k0; bi0 = row_lo + i; }    // i ascends: strict > keeps the lower index
                 if (k1 > best1) { best1 = k1; bi1 = row_lo + i; }
             }
@@ -324,38 +386,40 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         }
         __syncthreads();
         // this CTA's best per column goes to rank 0: values in xpart[0][rank][.], indices in xpart[1][rank][.]
-        if (tid < B) {
-            float b = pv[tid];
-            int ib = pi[tid];
+        for (int j = tid; j < B; j += kSfThreads) {
+            float b = pv[j];
+            int ib = pi[j];
 #pragma unroll
             for (int w = 1; w < kSfWarps; ++w) {
-                const float ob = pv[w * ldk + tid];
-                const int oi = pi[w * ldk + tid];
+                const float ob = pv[w * ldk + j];
+                const int oi = pi[w * ldk + j];
                 if (ob > b || (ob == b && oi < ib)) {
                     b = ob;
                     ib = oi;
                 }
             }
             const uint32_t base = ptx::map_to_rank(ptx::smem_u32(m.xpart), 0);
-            ptx::st_cluster_f32(base + ((rank * (uint32_t)ldk) + (uint32_t)tid) * 4u, b);
-            ptx::st_cluster_u32(base + (((C + rank) * (uint32_t)ldk) + (uint32_t)tid) * 4u, (uint32_t)ib);
+            ptx::st_cluster_f32(base + ((rank * (uint32_t)ldk) + (uint32_t)j) * 4u, b);
+            ptx::st_cluster_u32(base + (((C + rank) * (uint32_t)ldk) + (uint32_t)j) * 4u, (uint32_t)ib);
         }
         ptx::cluster_sync_all();      // after this barrier nothing is written into another CTA any more
-        if (rank == 0 && tid < B) {
+        if (rank == 0) {
             const int *xi = reinterpret_cast<const int *>(m.xpart + (size_t)C * ldk);
-            float b = m.xpart[tid];
-            int ib = xi[tid];
-            for (uint32_t r = 1; r < C; ++r) {     // ranks hold ascending row ranges: strict > keeps the lower index
-                const float ob = m.xpart[r * ldk + tid];
-                if (ob > b) {
-                    b = ob;
-                    ib = xi[r * ldk + tid];
-                }
-            }
             const int seg = t_begin - out0;
-            merged_idx[seg + tid] = my_prop;
-            merge_partner[seg + tid] = ib;
-            merge_weight[seg + tid] = b * m.vs[tid];    // (K U) V, the product the plan stores
+            for (int j = tid; j < B; j += kSfThreads) {
+                float b = m.xpart[j];
+                int ib = xi[j];
+                for (uint32_t r = 1; r < C; ++r) {     // ranks hold ascending row ranges: strict > keeps the lower index
+                    const float ob = m.xpart[r * ldk + j];
+                    if (ob > b) {
+                        b = ob;
+                        ib = xi[r * ldk + j];
+                    }
+                }
+                merged_idx[seg + j] = __ldg(order + t_begin + M + j);
+                merge_partner[seg + j] = ib;
+                merge_weight[seg + j] = b * m.vs[j];    // (K U) V, the product the plan stores
+            }
         }
     }
 
@@ -372,14 +436,13 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
             const float ui = m.us[i];
             __align__(16) float kk[8];
             __align__(16) float vv[8];
-            if (j0 < ldk) {
-                *reinterpret_cast<float4 *>(kk) = *reinterpret_cast<const float4 *>(m.Ks + (size_t)i * ldk + j0);
-                *reinterpret_cast<float4 *>(kk + 4) = *reinterpret_cast<const float4 *>(m.Ks + (size_t)i * ldk + j0 + 4);
-                *reinterpret_cast<float4 *>(vv) = *reinterpret_cast<const float4 *>(m.vs + j0);
-                *reinterpret_cast<float4 *>(vv + 4) = *reinterpret_cast<const float4 *>(m.vs + j0 + 4);
-            } else {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) kk[e] = vv[e] = 0.f;
+            for (int h = 0; h < 8; h += 4) {
+                const bool have = j0 + h < ldk && j0 + h < ldr;      // beyond: columns past B, zero
+                *reinterpret_cast<float4 *>(kk + h) =
+                    have ? *reinterpret_cast<const float4 *>(m.Ks + (size_t)i * ldr + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
+                *reinterpret_cast<float4 *>(vv + h) =
+                    have ? *reinterpret_cast<const float4 *>(m.vs + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             __nv_bfloat162 o[4];
 #pragma unroll
@@ -395,7 +458,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         // fp32, in place in the workspace tile (row pitch score_pitch(B))
         for (int idx = tid; idx < Ml * B; idx += kSfThreads) {
             const int i = idx / B, j = idx - i * B;
-            Sg[(size_t)(row_lo + i) * ldS + j] = (m.Ks[(size_t)i * ldk + j] * m.us[i]) * m.vs[j];
+            Sg[(size_t)(row_lo + i) * ldS + j] = (m.Ks[(size_t)i * ldr + j] * m.us[i]) * m.vs[j];
         }
     }
 }
