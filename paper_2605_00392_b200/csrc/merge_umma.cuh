@@ -13,9 +13,16 @@
 //     whose zero rows pad B to a multiple of 64.
 //   * D: two 128-lane x 256-column fp32 accumulators in TMEM, so that the epilogue of one unit
 //     overlaps the loads and UMMAs of the next.
-// The kernel is persistent: CTA c takes units c, c + gridDim.x, ...  Warp roles (192 threads):
+// The kernel is persistent: CTA c takes units c, c + gridDim.x, ...  When the Sinkhorn kernel ahead
+// publishes a list of finished images, the units follow that list (its s-th entry takes the place of
+// image s), the CTAs draw them from a counter, and the scheduler waits, bounded, for the entry it
+// needs: the kernel is launched as a programmatic dependent and merges the first images on whatever
+// SMs are free while the last ones still iterate.  Warp roles (224 threads):
 // warps 0-3 epilogue (TMEM -> registers -> bf16 -> own row of a padded staging tile -> one bulk store
-// per kept row); warp 4 lane 0 issues the TMA loads; warp 5 owns TMEM and lane 0 issues the UMMAs.
+// per kept row); warp 4 lane 0 issues the TMA loads; warp 5 owns TMEM and lane 0 issues the UMMAs;
+// warp 6 lane 0 is the scheduler: it draws the units, looks up what the other roles need to know about
+// them (a chain of dependent loads from L2) a few units ahead and hands them over through a small queue
+// in shared memory.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -27,7 +34,8 @@ constexpr int kMgTileN = 256;        // output columns per unit
 constexpr int kMgBK = 64;            // contraction rows per k-block
 constexpr int kMgBStages = 3;        // ring of B tiles (every k-block)
 constexpr int kMgAStages = 2;        // ring of plan tiles (k-blocks after the identity ones)
-constexpr int kMgThreads = 192;
+constexpr int kMgThreads = 224;
+constexpr int kMgLookahead = 1;       // units the scheduler may be ahead of the producer
 constexpr int kMgABytes = kMgTileM * 128;            // A tile: 128 rows x 64 bf16
 constexpr int kMgBBytes = kMgBK * kMgTileN * 2;      // B tile: 64 rows x 256 bf16 = 32 KB
 constexpr int kMgBBoxBytes = kMgBK * 128;            // one 64-column slab of it
@@ -38,7 +46,9 @@ constexpr int kMgIdentKb = 2;                        // k-blocks that carry the 
 constexpr int kMgStagePitch = kMgTileN * 2 + 16;     // bytes per staging row: padded, conflict-free
 constexpr int kMgStagingBytes = kMgTileM * kMgStagePitch;
 constexpr int kMgSmemBytes = kMgBStages * kMgBBytes + kMgAStages * kMgABytes + kMgIdentBytes +
-                             kMgStagingBytes + 1024 + 256;
+                             kMgStagingBytes + 1024 /*alignment*/ + 1024 /*barriers, unit queue*/;
+
+constexpr int kMgQueue = 16;         // ring of units between the producer and the other roles (about 6 in flight)
 
 struct MergeBarriers {
     uint64_t full[kMgBStages];       // B tile (and, for plan k-blocks, the A tile) of a k-block has landed
@@ -49,26 +59,70 @@ struct MergeBarriers {
     volatile int abort_flag;
 };
 
-// What every role needs to know about a unit; all roles compute it alike.
+// What every role needs to know about a unit.  img = -1 ends the queue.
 struct MergeUnit {
     int img, mt, ct;
     int t_begin, N, M, B, out0;
     bool valid;
+    bool timed_out;   // the image's list entry never came
 };
+
+struct MergeQueue {
+    volatile uint32_t head;          // units pushed by the scheduler
+    volatile uint32_t prod;          // units the producer has taken
+    volatile uint32_t tail;          // units every role is done with
+    MergeUnit e[kMgQueue];
+};
+
+// Bounded wait for the n-th unit of the queue.  false = gave up, or the kernel is being abandoned.
+__device__ inline bool merge_pop(MergeQueue *mq, const MergeBarriers *bars, uint32_t n, MergeUnit &q)
+{
+    for (uint32_t i = 0; i < ptx::kSpinLimit && !bars->abort_flag; ++i) {
+        if (mq->head > n) {
+            __threadfence_block();
+            q = mq->e[n % kMgQueue];
+            return true;
+        }
+        __nanosleep(40);
+    }
+    return false;
+}
+
+// Image in slot `slot` of the list of finished plans (bounded wait), -1 if it never shows up.
+__device__ inline int merge_wait_image(const int32_t *ready_list, int slot)
+{
+    for (uint32_t i = 0; i < ptx::kSpinLimit; ++i) {
+        const int v = ptx::ld_acquire_gpu(ready_list + slot);
+        if (v != 0) return v - 1;
+        __nanosleep(200);
+    }
+    return -1;
+}
 
 __device__ inline MergeUnit merge_unit(int u, int mtiles, int nct, const int32_t *__restrict__ offsets,
                                        const int32_t *__restrict__ counts,
-                                       const int32_t *__restrict__ out_offsets, int max_tokens, int total)
+                                       const int32_t *__restrict__ out_offsets, int max_tokens, int total,
+                                       const int32_t *ready_list)
 {
     MergeUnit q;
     q.ct = u % nct;
     const int v = u / nct;
     q.mt = v % mtiles;
     q.img = v / mtiles;
+    q.timed_out = false;
+    if (ready_list) {
+        q.img = merge_wait_image(ready_list, q.img);
+        if (q.img < 0) {
+            q.valid = false;
+            q.timed_out = true;
+            return q;
+        }
+    }
+    // L2 loads: with a ready list this kernel may have started before the selection wrote these
     q.valid = image_range(offsets, q.img, max_tokens, total, q.t_begin, q.N) && q.mt * kMgTileM < q.N;
-    q.M = q.valid ? __ldg(counts + q.img) : 0;
+    q.M = q.valid ? __ldcg(counts + q.img) : 0;
     q.B = q.N - q.M;
-    q.out0 = q.valid ? __ldg(out_offsets + q.img) : 0;
+    q.out0 = q.valid ? __ldcg(out_offsets + q.img) : 0;
     return q;
 }
 
@@ -78,7 +132,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                   int batch, int mtiles, const int32_t *__restrict__ counts,
                   const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ kpos,
                   int max_tokens, int total, __nv_bfloat16 *__restrict__ Y, int32_t *__restrict__ kept_idx,
-                  WsHeader *__restrict__ hdr)
+                  WsHeader *__restrict__ hdr, const int32_t *ready_list)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -86,6 +140,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
     uint8_t *ident = a_ring + kMgAStages * kMgABytes;
     uint8_t *staging = ident + kMgIdentBytes;
     MergeBarriers *bars = reinterpret_cast<MergeBarriers *>(staging + kMgStagingBytes);
+    MergeQueue *mq = reinterpret_cast<MergeQueue *>(staging + kMgStagingBytes + 256);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nct = (d + kMgTileN - 1) / kMgTileN;
     const int nunits = batch * mtiles * nct;
@@ -111,6 +166,9 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
             ptx::mbar_init(&bars->accum_empty[b], 128);
         }
         bars->abort_flag = 0;
+        mq->head = 0;
+        mq->prod = 0;
+        mq->tail = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 5) {
@@ -123,9 +181,10 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
     const uint32_t tmem_base = bars->tmem_base;
     const uint32_t smem_base = ptx::smem_u32(smem);
     // everything above is local set-up; the plan, the selection and the compact copy come from the
-    // kernels ahead in the stream
+    // kernels ahead in the stream: wait for them to end, or, with a list of finished images, for each
+    // image's entry (which is published after everything the image needs has been written)
     ptx::grid_dep_launch();
-    ptx::grid_dep_wait();
+    if (!ready_list) ptx::grid_dep_wait();
 
     if (warp == 4) {
         // ---------------- producer: tiled TMA for every operand -------------------------------------
@@ -138,9 +197,16 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
             uint32_t it = 0, ia = 0;
             uint32_t a_user[kMgAStages];
             for (int s = 0; s < kMgAStages; ++s) a_user[s] = 0xffffffffu;
-            for (int u = blockIdx.x; u < nunits && !bars->abort_flag; u += gridDim.x) {
-                const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total);
-                if (!q.valid) continue;
+            for (uint32_t n = 0; !bars->abort_flag; ++n) {
+                MergeUnit q;
+                if (!merge_pop(mq, bars, n, q)) {
+                    bars->abort_flag = 1;
+                    atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                    break;
+                }
+                if (q.img < 0) break;
+                mq->prod = n + 1;
+                if (ready_list) ptx::fence_proxy_async_all();   // the plan was written with ordinary stores
                 const int nkb = kMgIdentKb + (q.B + kMgBK - 1) / kMgBK;
                 const int row0 = q.t_begin + q.mt * kMgTileM;
                 const int xp0 = xp_row0(q.t_begin, q.img);
@@ -180,14 +246,55 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                 }
             }
         }
+    } else if (warp == 6) {
+        // ---------------- scheduler -------------------------------------------------------------------
+        if (lane == 0) {
+            uint32_t pushed = 0, drawn = 0;
+            auto push = [&](const MergeUnit &q) {
+                // stay a few units ahead of the producer, no more: a unit drawn is a unit no other CTA
+                // can take.  (The queue itself cannot fill up: fewer units are in flight than it holds.)
+                for (uint32_t i = 0; pushed - mq->prod >= (uint32_t)kMgLookahead ||
+                                     pushed - mq->tail >= (uint32_t)kMgQueue; ++i) {
+                    if (i >= ptx::kSpinLimit || bars->abort_flag) return false;
+                    __nanosleep(100);
+                }
+                mq->e[pushed % kMgQueue] = q;
+                __threadfence_block();
+                mq->head = ++pushed;
+                return true;
+            };
+            bool ok = true;
+            while (ok && !bars->abort_flag) {
+                // next unit: from the shared counter when the units follow the list of finished images
+                const int u = ready_list ? (int)atomicAdd(&hdr->merge_next, 1u)
+                                         : (int)(blockIdx.x + drawn++ * gridDim.x);
+                if (u >= nunits) break;
+                const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total,
+                                               ready_list);
+                if (q.timed_out) ok = false;
+                else if (q.valid) ok = push(q);
+            }
+            MergeUnit end{};
+            end.img = -1;
+            if (ok) ok = push(end);
+            if (!ok && !bars->abort_flag) {
+                bars->abort_flag = 1;
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+            }
+        }
     } else if (warp == 5) {
         // ---------------- UMMA issuer -----------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = ptx::idesc_bf16(kMgTileM, kMgTileN, false, true);
             uint32_t it = 0, ia = 0, acc = 0;
-            for (int u = blockIdx.x; u < nunits && !bars->abort_flag; u += gridDim.x) {
-                const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total);
-                if (!q.valid) continue;
+            for (uint32_t n = 0; !bars->abort_flag; ++n) {
+                MergeUnit q;
+                if (!merge_pop(mq, bars, n, q)) {
+                    bars->abort_flag = 1;
+                    atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                    break;
+                }
+                if (q.img < 0) break;
                 const int nkb = kMgIdentKb + (q.B + kMgBK - 1) / kMgBK;
                 const int buf = acc & 1;
                 if (acc >= 2) {
@@ -242,11 +349,17 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
         uint8_t *srow = staging + row * kMgStagePitch;        // this thread's staging row, nobody else's
         const uint32_t srow_u32 = ptx::smem_u32(srow);
         uint32_t acc = 0;
-        for (int u = blockIdx.x; u < nunits; u += gridDim.x) {
-            const MergeUnit q = merge_unit(u, mtiles, nct, offsets, counts, out_offsets, max_tokens, total);
-            if (!q.valid) continue;
+        for (uint32_t n = 0;; ++n) {
+            MergeUnit q;
+            const bool got = merge_pop(mq, bars, n, q);
+            if (!__all_sync(0xffffffffu, got)) {
+                bars->abort_flag = 1;
+                if (lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                break;
+            }
+            if (q.img < 0) break;
             const int tok = q.mt * kMgTileM + row;            // image-local token of this row
-            const int p = (tok < q.N) ? __ldg(kpos + q.t_begin + tok) : -1;   // >= 0: position among kept
+            const int p = (tok < q.N) ? __ldcg(kpos + q.t_begin + tok) : -1;   // >= 0: position among kept
             const int buf = acc & 1;
             // the TMEM loads below are warp-collective: take the go / no-go decision per warp
             bool ok = !bars->abort_flag && ptx::mbar_wait(&bars->accum_full[buf], (acc >> 1) & 1);
@@ -256,6 +369,9 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                 break;
             }
             ptx::tc_fence_after();
+            // unit n's accumulator is complete, so every epilogue thread is done with unit n - 2 (its
+            // accumulator buffer was handed back) and the UMMA issuer is past it: those entries are free
+            if (tid == 0 && n >= 1) mq->tail = n - 1;
             ptx::bulk_wait_read<0>();                         // the previous unit's store has read this row
             const int col0 = q.ct * kMgTileN;
             const int ncols = min(kMgTileN, d - col0);
@@ -292,6 +408,8 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, 512);
     }
+    // keep the stream's order: this grid does not end before the ones ahead of it have
+    if (ready_list) ptx::grid_dep_wait();
 }
 
 }  // namespace rtp

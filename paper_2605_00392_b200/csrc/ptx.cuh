@@ -61,6 +61,19 @@ __device__ inline void fence_proxy_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// The same for every state space: generic-proxy writes to global memory (made visible to the GPU by a
+// release / acquire pair around it) before TMA reads of them.
+__device__ inline void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ inline int ld_acquire_gpu(const int *p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ inline void st_release_gpu(int *p, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 // 16-byte global -> shared copy; src_bytes = 0 writes 16 zero bytes without reading.
 __device__ inline void cp_async_16(uint32_t dst_smem, const void *src, uint32_t src_bytes)
 {

@@ -64,6 +64,10 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(WsHeader), 256);
     L.img_done = off;
     off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
+    L.sink_done = off;
+    off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
+    L.ready_list = off;
+    off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
     L.clear_bytes = off;
     L.norms = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
@@ -306,6 +310,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     constexpr bool kTensor = std::is_same<T, __nv_bfloat16>::value;
     __nv_bfloat16 *pbuf = kTensor ? (__nv_bfloat16 *)(ws + L.pbuf) : nullptr;
     const int pbuf_pitch = (std::max(maxB, 1) + 63) / 64 * 64;   // <= L.pbuf_pitch_max
+    int32_t *ready_list = nullptr;   // images in the order their plans are finished, when the merge follows it
 
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
@@ -315,7 +320,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 dim3 ggrid((rows_max + kGpRows - 1) / kGpRows, batch);
                 if (!c.ok(launch_pdl(gather_prop_kernel, ggrid, dim3(128), 0, st, 1u,
                                      (const __nv_bfloat16 *)X, offsets, o.counts, order, plan->d, maxN, total,
-                                     (__nv_bfloat16 *)(ws + L.xp))))
+                                     (__nv_bfloat16 *)(ws + L.xp), (uint32_t *)(ws + L.sink_done),
+                                     (int32_t *)(ws + L.ready_list), (WsHeader *)(ws + L.header))))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "gather");
             }
@@ -366,20 +372,25 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             };
             while (fast_c < 8 && !all_tiles(fast_c, true)) fast_c *= 2;
             all_fast = all_tiles(fast_c, false);
+            // tiles wider than 256 columns, or too tall for the cluster's shared memory, are possible
+            const bool wide = maxB > 256 || !all_tiles(fast_c, true);
+            // When the first instance solves every image, it hands them to the merge kernel one by one
+            ready_list = (kTensor && !wide) ? (int32_t *)(ws + L.ready_list) : nullptr;
             if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<false>, dim3((unsigned)(batch * fast_c)),
                                  dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets,
                                  o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                                  fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                                 o.stats)))
+                                 o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
+                                 (WsHeader *)(ws + L.header))))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_cluster");
-            // tiles wider than 256 columns, or too tall for the cluster's shared memory
-            if (maxB > 256 || !all_tiles(fast_c, true)) {
+            if (wide) {
                 if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<true>, dim3((unsigned)(batch * fast_c)),
                                      dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c,
                                      offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total,
                                      op, fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
-                                     o.merge_weight, o.stats)))
+                                     o.merge_weight, o.stats, (uint32_t *)nullptr, (int32_t *)nullptr,
+                                     (WsHeader *)nullptr)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "sinkhorn_wide");
             }
@@ -415,7 +426,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         if (!c.ok(launch_pdl(merge_umma_kernel, dim3((unsigned)grid), dim3(kMgThreads), kMgSmemBytes, st, 1u,
                              tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
                              (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
-                             (WsHeader *)(ws + L.header))))
+                             (WsHeader *)(ws + L.header), (const int32_t *)ready_list)))
             return RTPRUNE_ERR_CUDA;
     } else {
         const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;

@@ -236,6 +236,26 @@ __device__ inline ScState sinkhorn_cluster_iterate(const ScSmem &m, int Ml, int 
     return st;
 }
 
+// This CTA has written everything it contributes to image `img`; the last CTA of the cluster to say so
+// appends the image to the list that the merge kernel consumes in order of completion (it may already
+// be running: it was launched as a programmatic dependent).  Called by every thread of the CTA.
+__device__ inline void sinkhorn_publish(int img, uint32_t C, uint32_t *__restrict__ sink_done,
+                                        int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr)
+{
+    if (!ready_list) return;
+    ptx::fence_proxy_async_all();     // the plan rows are read by TMA over there
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t prev = atomicAdd(&sink_done[img], 1u);
+        if (prev == C - 1u) {
+            __threadfence();
+            const uint32_t slot = atomicAdd(&hdr->n_ready, 1u);
+            ptx::st_release_gpu(ready_list + slot, img + 1);
+        }
+    }
+}
+
 // grid = batch * C CTAs, clusters of C along x: CTA rank r of cluster i owns rows r*rows_per .. of
 // image i's tile.  Every early return below depends on the image only, so a cluster leaves as a whole.
 // Two instances share the work: WIDE = false takes the tiles of up to 256 columns that fit shared
@@ -247,7 +267,9 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                         float *__restrict__ kmat, int kmat_stride, int max_tokens, int total, OtParams p,
                         int smem_floats, __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch,
                         int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
-                        float *__restrict__ merge_weight, float *__restrict__ stats)
+                        float *__restrict__ merge_weight, float *__restrict__ stats,
+                        uint32_t *__restrict__ sink_done, int32_t *__restrict__ ready_list,
+                        WsHeader *__restrict__ hdr)
 {
     extern __shared__ __align__(16) float sm[];
     const uint32_t C = ptx::cluster_nctarank(), rank = ptx::cluster_ctarank();
@@ -256,9 +278,17 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();     // the scores come from the kernel ahead
     int t_begin, N;
-    if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
+    // (a ready list is only passed when this instance is the only Sinkhorn kernel of the run, so an
+    // image that leaves here needs no plan)
+    if (!image_range(offsets, img, max_tokens, total, t_begin, N)) {
+        sinkhorn_publish(img, C, sink_done, ready_list, hdr);
+        return;
+    }
     const int M = counts[img], B = N - M;
-    if (B == 0 || !sinkhorn_cluster_handles(M, B, (int)C, smem_floats)) return;   // the general kernel takes it
+    if (B == 0 || !sinkhorn_cluster_handles(M, B, (int)C, smem_floats)) {   // the general kernel takes it
+        sinkhorn_publish(img, C, sink_done, ready_list, hdr);
+        return;
+    }
     const bool in_smem = sinkhorn_cluster_fits(M, B, (int)C, smem_floats);
     const int ldk = sinkhorn_ldk(B);
     if ((in_smem && ldk <= 256) == WIDE) return;             // the other instance's tile
@@ -356,6 +386,42 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         stats[(size_t)img * kStats + 5] = (float)st.done;
         stats[(size_t)img * kStats + 6] = st.last_move;
     }
+    // ---- plan P = U K V (non-dustbin block), this CTA's rows --------------------------------------------
+    // (needs this CTA's K and U and the V every CTA holds: no cluster barrier before it)
+    if (pbuf) {
+        // alpha P in bf16 for the tensor-core merge: row = the kept token's position in X; columns up to
+        // the next multiple of 64 are written (zeros past B), 8 columns = 16 bytes per store
+        const int kpad = (B + 63) & ~63;
+        const int vpr = kpad >> 3;
+        __nv_bfloat16 *Pimg = pbuf + (size_t)t_begin * pbuf_pitch;
+        for (int idx = tid; idx < Ml * vpr; idx += kSfThreads) {
+            const int i = idx / vpr, j0 = (idx - i * vpr) << 3;
+            const int tok = m.toks[i];
+            const float ui = m.us[i];
+            __align__(16) float kk[8];
+            __align__(16) float vv[8];
+#pragma unroll
+            for (int h = 0; h < 8; h += 4) {
+                const bool have = j0 + h < ldk && j0 + h < ldr;      // beyond: columns past B, zero
+                *reinterpret_cast<float4 *>(kk + h) =
+                    have ? *reinterpret_cast<const float4 *>(m.Ks + (size_t)i * ldr + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
+                *reinterpret_cast<float4 *>(vv + h) =
+                    have ? *reinterpret_cast<const float4 *>(m.vs + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            __nv_bfloat162 o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                // K is zero past column B, so those products are zero
+                const float a = (kk[2 * e] * ui) * vv[2 * e];
+                const float b = (kk[2 * e + 1] * ui) * vv[2 * e + 1];
+                o[e] = __floats2bfloat162_rn(p.alpha * a, p.alpha * b);
+            }
+            *reinterpret_cast<uint4 *>(Pimg + (size_t)tok * pbuf_pitch + j0) = *reinterpret_cast<uint4 *>(o);
+        }
+    }
+    // the merge kernel may take the image from here: the pairs below are outputs of their own
+    sinkhorn_publish(img, C, sink_done, ready_list, hdr);
+
     // nobody reads xpart any more (it is reused below), and vs is visible to the CTA
     ptx::cluster_sync_all();
 
@@ -423,39 +489,9 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         }
     }
 
-    // ---- plan P = U K V (non-dustbin block), this CTA's rows --------------------------------------------
-    if (pbuf) {
-        // alpha P in bf16 for the tensor-core merge: row = the kept token's position in X; columns up to
-        // the next multiple of 64 are written (zeros past B), 8 columns = 16 bytes per store
-        const int kpad = (B + 63) & ~63;
-        const int vpr = kpad >> 3;
-        __nv_bfloat16 *Pimg = pbuf + (size_t)t_begin * pbuf_pitch;
-        for (int idx = tid; idx < Ml * vpr; idx += kSfThreads) {
-            const int i = idx / vpr, j0 = (idx - i * vpr) << 3;
-            const int tok = m.toks[i];
-            const float ui = m.us[i];
-            __align__(16) float kk[8];
-            __align__(16) float vv[8];
-#pragma unroll
-            for (int h = 0; h < 8; h += 4) {
-                const bool have = j0 + h < ldk && j0 + h < ldr;      // beyond: columns past B, zero
-                *reinterpret_cast<float4 *>(kk + h) =
-                    have ? *reinterpret_cast<const float4 *>(m.Ks + (size_t)i * ldr + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
-                *reinterpret_cast<float4 *>(vv + h) =
-                    have ? *reinterpret_cast<const float4 *>(m.vs + j0 + h) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            __nv_bfloat162 o[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                // K is zero past column B, so those products are zero
-                const float a = (kk[2 * e] * ui) * vv[2 * e];
-                const float b = (kk[2 * e + 1] * ui) * vv[2 * e + 1];
-                o[e] = __floats2bfloat162_rn(p.alpha * a, p.alpha * b);
-            }
-            *reinterpret_cast<uint4 *>(Pimg + (size_t)tok * pbuf_pitch + j0) = *reinterpret_cast<uint4 *>(o);
-        }
-    } else {
-        // fp32, in place in the workspace tile (row pitch score_pitch(B))
+    // fp32 storage: the plan in place in the workspace tile (row pitch score_pitch(B)), after the pairing
+    // because the tile may be where K lives
+    if (!pbuf) {
         for (int idx = tid; idx < Ml * B; idx += kSfThreads) {
             const int i = idx / B, j = idx - i * B;
             Sg[(size_t)(row_lo + i) * ldS + j] = (m.Ks[(size_t)i * ldr + j] * m.us[i]) * m.vs[j];

@@ -423,11 +423,22 @@ constexpr int kGpRows = 8;     // rows per CTA: four warps, two rows each
 __global__ void __launch_bounds__(128)
 gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restrict__ offsets,
                    const int32_t *__restrict__ counts, const int32_t *__restrict__ order, int d,
-                   int max_tokens, int total, __nv_bfloat16 *__restrict__ xp)
+                   int max_tokens, int total, __nv_bfloat16 *__restrict__ xp, uint32_t *__restrict__ sink_done,
+                   int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr)
 {
     const int img = blockIdx.y;
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();     // counts and order come from the kernel ahead
+    // The list of finished transport plans starts empty: the merge kernel of the run before has ended
+    // (it is ahead of stage 1 in the stream), this run's Sinkhorn kernel starts after this kernel ends.
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        sink_done[img] = 0;
+        ready_list[img] = 0;
+        if (img == 0) {
+            hdr->n_ready = 0;
+            hdr->merge_next = 0;
+        }
+    }
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M, Bpad = (B + 63) & ~63;
