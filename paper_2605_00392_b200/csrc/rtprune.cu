@@ -213,7 +213,7 @@ template <typename T>
 cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, const void *X,
                                  const int32_t *offsets, int batch, int total, const RatioParams &rp,
                                  const float *rho, char *ws, int32_t *out_offsets, int32_t *counts,
-                                 float *stats, float *norms_out, int32_t *order_out)
+                                 float *stats, float *norms_out, int32_t *order_out, int scan_here)
 {
     constexpr int EPV = Elem<T>::kPerVec;
     const WsLayout &L = pl->ws;
@@ -240,7 +240,7 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
             (const T *)X, offsets, batch, d, L.chunks, chunk_tokens, pl->max_tokens, total, rp, rho, \
             (float *)(ws + L.norms), (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),     \
             (int32_t *)(ws + L.order), (int32_t *)(ws + L.kpos), counts, out_offsets, stats,     \
-            norms_out, order_out, (WsHeader *)(ws + L.header));                                  \
+            norms_out, order_out, (WsHeader *)(ws + L.header), scan_here);                       \
         if (e != cudaSuccess) return e;                                                          \
         break;                                                                                   \
     }
@@ -280,15 +280,17 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
                                const int32_t *offsets, int32_t batch, int total,
                                const rtprune_params_t *params, char *ws, int32_t *out_offsets,
                                int32_t *counts, float *stats, float *norms_out,
-                               int32_t *order_out)
+                               int32_t *order_out, bool scan_here)
 {
     Checked c{plan};
     RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
     cudaError_t e = (plan->dtype == RTPRUNE_BF16)
                         ? launch_stage1_kernel<__nv_bfloat16>(plan, st, X, offsets, batch, total, rp, params->rho,
-                                                              ws, out_offsets, counts, stats, norms_out, order_out)
+                                                              ws, out_offsets, counts, stats, norms_out, order_out,
+                                                              scan_here ? 1 : 0)
                         : launch_stage1_kernel<float>(plan, st, X, offsets, batch, total, rp, params->rho, ws,
-                                                      out_offsets, counts, stats, norms_out, order_out);
+                                                      out_offsets, counts, stats, norms_out, order_out,
+                                                      scan_here ? 1 : 0);
     if (!c.ok(e)) return RTPRUNE_ERR_CUDA;
     launched(plan, st, "stage1");
     return RTPRUNE_OK;
@@ -321,7 +323,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 if (!c.ok(launch_pdl(gather_prop_kernel, ggrid, dim3(128), 0, st, 1u,
                                      (const __nv_bfloat16 *)X, offsets, o.counts, order, plan->d, maxN, total,
                                      (__nv_bfloat16 *)(ws + L.xp), (uint32_t *)(ws + L.sink_done),
-                                     (int32_t *)(ws + L.ready_list), (WsHeader *)(ws + L.header))))
+                                     (int32_t *)(ws + L.ready_list), (WsHeader *)(ws + L.header), batch,
+                                     o.out_offsets)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "gather");
             }
@@ -450,8 +453,11 @@ rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X
         return RTPRUNE_OK;
     }
     prof_begin(plan, st);
+    // with bf16 storage and anything to prune, the kernel that copies the pruned rows also turns the counts
+    // into out_offsets, so that stage 1 ends with the last image's selection
+    const bool scan_later = plan->dtype == RTPRUNE_BF16 && max_pruned(params, plan->max_tokens) > 0;
     rtprune_status_t s = launch_stage1(plan, st, X, offsets, batch, total, params, ws, o.out_offsets,
-                                       o.counts, o.stats, nullptr, nullptr);
+                                       o.counts, o.stats, nullptr, nullptr, !scan_later);
     if (s != RTPRUNE_OK) return s;
     return (plan->dtype == RTPRUNE_BF16)
                ? launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o)
@@ -656,7 +662,7 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
     }
     prof_begin(plan, (cudaStream_t)cuda_stream);
     return launch_stage1(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
-                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out);
+                         (char *)workspace, out_offsets, counts, stats, norms_out, order_out, true);
 }
 
 rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
@@ -703,7 +709,7 @@ rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, 
         return RTPRUNE_ERR_CUDA;
     prof_begin(plan, st);
     return launch_stage1(plan, st, X, offsets, batch, (int)total_tokens, params, scratch, out_offsets,
-                         counts, stats, norms_out, order_out);
+                         counts, stats, norms_out, order_out, true);
 }
 
 rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)

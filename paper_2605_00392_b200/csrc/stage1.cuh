@@ -87,23 +87,68 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int nth = kS1Threads;
 
-    // every global read is issued up front: rho, the norms (keys of the ranking), the chunk partials
+    // Every global read is issued before the first use of any of them (one trip to L2, not one per
+    // loop iteration): rho, the norms (keys of the ranking), the chunk partials.
     const float rho_i = (tid == 0 && rho) ? __ldg(rho + img) : 0.f;
+    constexpr int kKeysAhead = 4;      // norms per thread held in registers (N <= 1024), the rest in a loop
+    float key_r[kKeysAhead];
+#pragma unroll
+    for (int q = 0; q < kKeysAhead; ++q) {
+        const int k = tid + q * nth;
+        key_r[q] = (k < N) ? __ldcg(norms + t_begin + k) : 0.f;
+    }
+    // phi (Eq. 8) via |sum of unit tokens|^2; the partials were written by other CTAs: read them from L2.
+    // A thread owns groups of 4 columns (tid, tid + 256, ...) and adds them over the chunks, four chunks
+    // and four groups to a batch of loads.
+    const int nchunk = (N + chunk_tokens - 1) / chunk_tokens;
+    const float4 *sp4 = reinterpret_cast<const float4 *>(spart + (size_t)img * chunks * d);
+    const int ngroups = d >> 2, d4 = d >> 2;
+    float local = 0.f;
+    for (int g0 = tid; g0 < ngroups; g0 += 4 * nth) {
+        float4 a4[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) a4[a] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k0 = 0; k0 < nchunk; k0 += 4) {
+            float4 v[4][4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int g = g0 + a * nth;
+                    v[a][u] = (g < ngroups && k0 + u < nchunk) ? __ldcg(sp4 + (size_t)(k0 + u) * d4 + g)
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    a4[a].x += v[a][u].x;
+                    a4[a].y += v[a][u].y;
+                    a4[a].z += v[a][u].z;
+                    a4[a].w += v[a][u].w;
+                }
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            local = fmaf(a4[a].x, a4[a].x, local);
+            local = fmaf(a4[a].y, a4[a].y, local);
+            local = fmaf(a4[a].z, a4[a].z, local);
+            local = fmaf(a4[a].w, a4[a].w, local);
+        }
+    }
     // norm bits: for non-negative floats the unsigned order is the float order, and a NaN still ranks
-    for (int k = tid; k < N; k += nth) {
+#pragma unroll
+    for (int q = 0; q < kKeysAhead; ++q) {
+        const int k = tid + q * nth;
+        if (k < N) {
+            s_keys[k] = __float_as_uint(key_r[q]) & 0x7fffffffu;
+            if (norms_out) norms_out[t_begin + k] = key_r[q];
+        }
+    }
+    for (int k = tid + kKeysAhead * nth; k < N; k += nth) {
         const float key = __ldcg(norms + t_begin + k);
         s_keys[k] = __float_as_uint(key) & 0x7fffffffu;
         if (norms_out) norms_out[t_begin + k] = key;
-    }
-    // phi (Eq. 8) via |sum of unit tokens|^2; the partials were written by other CTAs: read them from L2
-    const int nchunk = (N + chunk_tokens - 1) / chunk_tokens;
-    const float *sp = spart + (size_t)img * chunks * d;
-    float local = 0.f;
-    for (int c = tid; c < d; c += nth) {
-        float s = 0.f;
-#pragma unroll 8
-        for (int k = 0; k < nchunk; ++k) s += __ldcg(sp + (size_t)k * d + c);
-        local = fmaf(s, s, local);
     }
     const float ssum = block_sum(local, s_redf);
     if (tid == 0) {
@@ -214,6 +259,44 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
     __syncthreads();
 }
 
+// out_offsets = exclusive prefix sum of counts (and the total at [batch]), by one CTA of NTH threads;
+// `scratch` holds 32 ints.
+template <int NTH>
+__device__ inline void scan_counts(const int32_t *counts, int32_t *__restrict__ out_offsets, int batch,
+                                   int *scratch)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ipt2 = (batch + NTH - 1) / NTH;
+    const int b0 = min(tid * ipt2, batch), b1 = min(b0 + ipt2, batch);
+    int sum = 0;
+    for (int b = b0; b < b1; ++b) sum += __ldcg(counts + b);
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < (NTH >> 5)) ? scratch[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        scratch[lane] = wi - w;
+    }
+    __syncthreads();
+    int run = scratch[warp] + incl - sum;
+    for (int b = b0; b < b1; ++b) {
+        out_offsets[b] = run;
+        run += __ldcg(counts + b);
+    }
+    if (tid == NTH - 1) out_offsets[batch] = run;  // the last thread's running sum is the total
+}
+
 // ---------------------------------------------------------------------------------------------
 // grid = (chunks of this run, batch), 256 threads; CTA (c, i) owns chunk_tokens consecutive tokens of
 // image i (a multiple of 8, at least kChunkTokens, chosen by the host so that the grid is about one wave).
@@ -234,7 +317,7 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
               float *norms, float *spart, uint32_t *img_done, int32_t *__restrict__ order,
               int32_t *__restrict__ kpos, int32_t *counts, int32_t *__restrict__ out_offsets,
               float *__restrict__ stats, float *__restrict__ norms_out, int32_t *__restrict__ order_out,
-              WsHeader *hdr)
+              WsHeader *hdr, int scan_here)
 {
     constexpr int EPV = Elem<T>::kPerVec;
     extern __shared__ __align__(16) float s_dyn[];
@@ -370,7 +453,9 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
                      norms_out, order_out, reinterpret_cast<uint32_t *>(s_dyn));
     }
 
-    // the CTA that completes the batch: out_offsets = exclusive prefix sum of counts
+    // the CTA that completes the batch: out_offsets = exclusive prefix sum of counts (unless a kernel
+    // that follows does it, off the path of the last image's selection)
+    if (!scan_here) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -381,36 +466,7 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    constexpr int nth = kS1Threads;
-    const int ipt2 = (batch + nth - 1) / nth;
-    const int b0 = min(tid * ipt2, batch), b1 = min(b0 + ipt2, batch);
-    int sum = 0;
-    for (int b = b0; b < b1; ++b) sum += __ldcg(counts + b);
-    int incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) s_scan[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int w = (lane < (nth >> 5)) ? s_scan[lane] : 0;
-        int wi = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, wi, o);
-            if (lane >= o) wi += t;
-        }
-        s_scan[lane] = wi - w;
-    }
-    __syncthreads();
-    int run = s_scan[warp] + incl - sum;
-    for (int b = b0; b < b1; ++b) {
-        out_offsets[b] = run;
-        run += __ldcg(counts + b);
-    }
-    if (tid == nth - 1) out_offsets[batch] = run;  // the last thread's running sum is the total
+    scan_counts<kS1Threads>(counts, out_offsets, batch, s_scan);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -424,11 +480,15 @@ __global__ void __launch_bounds__(128)
 gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restrict__ offsets,
                    const int32_t *__restrict__ counts, const int32_t *__restrict__ order, int d,
                    int max_tokens, int total, __nv_bfloat16 *__restrict__ xp, uint32_t *__restrict__ sink_done,
-                   int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr)
+                   int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr, int batch,
+                   int32_t *__restrict__ out_offsets)
 {
+    __shared__ int s_scan[32];
     const int img = blockIdx.y;
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();     // counts and order come from the kernel ahead
+    // one CTA turns the counts into out_offsets while the others copy
+    if (blockIdx.x == 0 && img == 0) scan_counts<128>(counts, out_offsets, batch, s_scan);
     // The list of finished transport plans starts empty: the merge kernel of the run before has ended
     // (it is ahead of stage 1 in the stream), this run's Sinkhorn kernel starts after this kernel ends.
     if (blockIdx.x == 0 && threadIdx.x == 0) {
