@@ -221,3 +221,45 @@ def test_host_side_argument_errors(binding):
                        "rtprune_run")
     assert e.value.status == 3
     plan.close()
+
+
+def test_runs_back_to_back_on_one_plan_leave_no_state(parity, binding):
+    # Three workloads alternate on ONE plan and workspace without a synchronisation between the runs:
+    # a batch whose images all take the fast Sinkhorn kernel (the merge kernel then follows the list of
+    # finished images), a ragged one with images that prune nothing, and one at retention 1 (no stage
+    # 2 at all).  Counters, the list and the unit counter in the workspace must be left as a fresh run
+    # expects them: the second round must reproduce the first bit for bit, and match the oracle.
+    dev = torch.device("cuda", 0)
+    wa = synth.make("large", batch=6)
+    wb = synth.ragged([1, 400, 2, 77, 300], params=dict(dynamic=1, phi_lo=0.0, phi_hi=0.6, r_max=0.5))
+    wb.rho[3] = 1.0                                   # image 3 keeps every token
+    wc = synth.ragged([64, 200, 9], params=dict(r_fixed=0.0))
+    ws = [wa, wb, wc]
+    plan = binding.Plan(1280, torch.bfloat16, 6, max(w.total_tokens for w in ws), 400, device=dev)
+    try:
+        ins, outs = [], []
+        for w in ws:
+            rho = torch.from_numpy(w.rho.copy()).to(dev)
+            fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w.params.items()}
+            ins.append((w.X.to(dev), torch.from_numpy(w.offsets.copy()).to(dev),
+                        binding.make_params(rho, **fields), rho))
+        for rnd in range(2):
+            for w, (X, offs, params, _) in zip(ws, ins):
+                out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, dev)
+                plan.run(X, offs, params, out)
+                outs.append(out)
+        torch.cuda.synchronize()
+        assert plan.query_status() == 0
+        for k, w in enumerate(ws):
+            a, b = outs[k], outs[k + 3]
+            n = int(a.out_offsets[w.batch])
+            nb = w.total_tokens - n
+            assert torch.equal(a.out_offsets, b.out_offsets) and torch.equal(a.counts, b.counts)
+            assert torch.equal(a.kept_idx[:n], b.kept_idx[:n]) and torch.equal(a.Y[:n], b.Y[:n])
+            assert torch.equal(a.merged_idx[:nb], b.merged_idx[:nb])
+            assert torch.equal(a.merge_partner[:nb], b.merge_partner[:nb])
+            assert torch.equal(a.merge_weight[:nb], b.merge_weight[:nb])
+    finally:
+        plan.close()
+    for w in ws:                                      # and each of them is what the oracle computes
+        parity.check_workload(w)
