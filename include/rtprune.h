@@ -227,6 +227,27 @@ rtprune_status_t rtprune_profile_enable(rtprune_plan_t *plan, int32_t enable);
 rtprune_status_t rtprune_profile_read(rtprune_plan_t *plan, int32_t *n, float *ms,
                                       const char **names);
 
+/*
+ * Textual density rho of page images (Eq. 9; Appendix B), the input `rho` of the dynamic ratio
+ * (Eq. 10): BT.601 grayscale of the 8-bit channels on the [0, 1] scale, the two 3 x 3 Sobel kernels,
+ * E = [sqrt(Gx^2 + Gy^2) >= tau], rho_k = mean of E over the patch x patch pixels of token patch k,
+ * rho = mean of rho_k.  Pixels outside the image take the value of the nearest pixel inside (the paper
+ * does not say).  The decision G >= tau is taken in exact integer arithmetic.  No plan is needed.
+ *
+ *   images       DEVICE [batch][height][width][3] uint8, R, G, B interleaved, 16-byte aligned; read only
+ *   patch        16, 32 or 64; height and width are multiples of it (else RTPRUNE_ERR_UNSUPPORTED)
+ *   tau          threshold on the gradient magnitude, >= 0 (Algorithm 1: 0.2)
+ *   rho          DEVICE [batch] float, written
+ *   image_counts DEVICE [batch] uint32 scratch of the caller, written: edge pixels of each image
+ *   edge_counts  DEVICE [batch][height/patch][width/patch] int32, written: edge pixels of each patch
+ *                (rho_k = edge_counts / patch^2); may be NULL
+ * Asynchronous on the stream (one memset, two kernels), allocates nothing.  Host-detectable errors
+ * are returned before any launch.
+ */
+rtprune_status_t rtprune_density(void *cuda_stream, const uint8_t *images, int32_t batch, int32_t height,
+                                 int32_t width, int32_t patch, float tau, float *rho,
+                                 uint32_t *image_counts, int32_t *edge_counts);
+
 /* Kernels launched by the most recent run / select / run_host call on this plan. */
 int32_t rtprune_last_launch_count(const rtprune_plan_t *plan);
 

@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
                                    vp, vp, vp, vp, vp, vp, vp, vp]
     L.rtprune_host_arena_bytes.argtypes = [vp, ctypes.POINTER(sz)]
     L.rtprune_query_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.rtprune_density.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp]
     L.rtprune_profile_enable.argtypes = [vp, i32]
     L.rtprune_profile_read.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float),
                                        ctypes.POINTER(ctypes.c_char_p)]
@@ -269,6 +270,27 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+def density(images: torch.Tensor, patch: int = 64, tau: float = 0.2, *, want_patch_counts: bool = False,
+            stream: Optional[torch.cuda.Stream] = None):
+    """rtprune_density: textual density rho [batch] (float32, on the images' device) of a batch of page
+    images [batch, H, W, 3] uint8 (Eq. 9).  Returns (rho, image_counts, edge_counts or None)."""
+    if images.dtype != torch.uint8 or images.dim() != 4 or images.shape[3] != 3 or not images.is_contiguous():
+        raise ValueError("images must be a contiguous [batch, H, W, 3] uint8 tensor")
+    if not images.is_cuda:
+        raise ValueError("images must live on a CUDA device")
+    batch, H, W, _ = images.shape
+    dev = images.device
+    rho = torch.empty(batch, dtype=torch.float32, device=dev)
+    counts = torch.empty(batch, dtype=torch.int32, device=dev)          # uint32 in the library
+    per_patch = None
+    if want_patch_counts and patch > 0:
+        per_patch = torch.empty((batch, H // patch, W // patch), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().rtprune_density(_stream_handle(stream), images.data_ptr(), batch, H, W, patch, float(tau),
+                                     rho.data_ptr(), counts.data_ptr(), _ptr(per_patch)), "rtprune_density")
+    return rho, counts, per_patch
 
 
 def shard_images(batch: int, world_size: int, rank: int):

@@ -1,4 +1,4 @@
-"""Seeded synthetic token batches with the shapes of the paper's workloads.
+"""Seeded synthetic token batches (and page images) with the shapes of the paper's workloads.
 
 This module is the ONLY code shared by the CUDA path's tests/benchmark and the CPU oracle.  It
 draws random inputs and nothing else: none of the pruning method's arithmetic lives here.  (The one
@@ -216,3 +216,46 @@ def ragged(lengths: List[int], *, seed: int = 7, d: int = D_MODEL,
     if params:
         p.update(params)
     return _assemble("ragged", ims, np.full(len(lengths), text_density), p)
+
+
+# ---------------------------------------------------------------------------------------------
+# Page images for the textual-density step (Eq. 9): 8-bit RGB, [batch, H, W, 3].
+# ---------------------------------------------------------------------------------------------
+PAGE_PATCH = 64          # pixels per token patch side: 1280 x 1280 pixels <-> 20 x 20 = 400 tokens
+
+
+def page_image(rng: np.random.Generator, height: int, width: int, text_fraction: float) -> np.ndarray:
+    """One synthetic document page: a near-white, slightly tinted background with faint sensor noise,
+    and text in a `text_fraction` share of the 64 x 64 patches: lines 16 pixels high whose glyph
+    cells (8 pixels wide) are inked at random with dark, sharp-edged dots.  Blank patches stay
+    uniform up to the noise, whose amplitude (+-2 levels) is far below the edge threshold."""
+    ph, pw = height // PAGE_PATCH, width // PAGE_PATCH
+    r = rng.integers(0, 256, size=(height, width), dtype=np.uint8)      # one draw serves noise and ink
+    text_patch = rng.random((ph, pw)) < text_fraction
+    inked_cell = rng.random((height // 16, width // 8)) < 0.55
+    rows = np.arange(height) % 16
+    line_rows = (rows >= 3) & (rows <= 12)
+    mask = np.repeat(np.repeat(text_patch, PAGE_PATCH, axis=0), PAGE_PATCH, axis=1)
+    mask &= np.repeat(np.repeat(inked_cell, 16, axis=0), 8, axis=1)
+    mask &= line_rows[:, None]
+    mask &= (r >> 2) < 22                                               # about a third of the cell's pixels
+    base = np.array([rng.integers(244, 253), rng.integers(242, 251), rng.integers(236, 249)], dtype=np.int16)
+    ink = np.array([rng.integers(10, 60), rng.integers(10, 60), rng.integers(20, 90)], dtype=np.int16)
+    noise = (r & 3).astype(np.int16) - 2                                # -2 .. 1
+    img = np.empty((height, width, 3), dtype=np.uint8)
+    for ch in range(3):
+        plane = np.where(mask, ink[ch], base[ch]) + noise
+        img[..., ch] = np.clip(plane, 0, 255).astype(np.uint8)
+    return img
+
+
+def pages(batch: int, height: int = 1280, width: int = 1280, *, seed: int = 11,
+          text_fraction: Optional[np.ndarray] = None) -> torch.Tensor:
+    """[batch, H, W, 3] uint8 pages; image i's share of text patches is text_fraction[i] (default
+    U[0.2, 0.9], the range of the token batches' textual density)."""
+    out = np.empty((batch, height, width, 3), dtype=np.uint8)
+    for i in range(batch):
+        rng = _rng(SEED_BASE + 0x200 + seed, i)
+        tf = float(rng.uniform(0.2, 0.9)) if text_fraction is None else float(text_fraction[i])
+        out[i] = page_image(rng, height, width, tf)
+    return torch.from_numpy(out)
