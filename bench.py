@@ -144,8 +144,73 @@ def run_reference(args, rank: int) -> None:
     print(json.dumps(line), flush=True)
 
 
+def run_density(args) -> None:
+    """`--step density`: the textual-density kernel (Eq. 9) alone, on the pages of one Large batch (64
+    pages of 1280 x 1280 RGB, 8 bits per channel).  One GPU; prints one JSON line of its own."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    from paper_2605_00392_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    batch, H, W, patch, tau = 64, 1280, 1280, synth.PAGE_PATCH, 0.2
+    host = synth.pages(8, H, W, seed=1)
+    sets = [torch.roll(host, k, 0).repeat(batch // 8, 1, 1, 1).contiguous().to(dev) for k in range(2)]   # 2 x 315 MB > L2
+    warm = max(args.warmup, 3)
+    sampler = ClockSampler(0)       # a step is 0.15 ms: the sampler runs over the warm-up and both legs
+    sampler.start()
+    for i in range(warm):
+        binding.density(sets[i % 2], patch, tau)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(2000000)
+    e0.record()
+    for i in range(args.steps):
+        binding.density(sets[i % 2], patch, tau)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    # end to end from pinned host pages: copy in, kernel, rho back
+    pinned = sets[0].cpu().pin_memory()
+    stage = torch.empty_like(sets[0])
+    rho_host = torch.empty(batch, dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(e2e_steps):
+        stage.copy_(pinned, non_blocking=True)
+        rho, _, _ = binding.density(stage, patch, tau)
+        rho_host.copy_(rho, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    clocks = sampler.stop()
+    hbm_peak, _, src = measured_peaks()
+    nbytes = batch * H * W * 3
+    line = {"metric": "pages/sec (textual density)", "value": batch / ms * 1e3, "unit": "images/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u8 -> int64 (exact)", "data": "synthetic",
+            "config": {"workload": "density: 64 pages x 1280 x 1280 x RGB8, patch 64, tau 0.2",
+                       "l2": "pages rotate over 2 buffer sets (629 MB > L2)"},
+            "roofline": {"kernel": "density_tile", "bound": "hbm", "achieved": nbytes / ms / 1e6, "peak": hbm_peak,
+                         "unit": "GB/s", "frac": nbytes / ms / 1e6 / hbm_peak, "peak_source": src, "traffic": None},
+            "e2e": {"value": batch / e2e_ms * 1e3, "unit": "images/s", "h2d_bytes_per_step": nbytes,
+                    "d2h_bytes_per_step": 4 * batch, "ms_per_step": e2e_ms},
+            "gpu_launches": 2 * args.steps, "clocks": clocks}
+    if not args.no_cpu_baseline:
+        from oracle import density as od
+        sample = host[:4].numpy()
+        t0 = time.perf_counter()
+        od.density_batch(sample, patch, float(np.float32(tau)))
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": len(sample) / dt, "unit": "images/s", "cores": 1, "kind": "oracle",
+                                "sample": "4 pages of the batch, numpy fp64, one thread"}
+    print(json.dumps(line))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
+    ap.add_argument("--step", default="prune", choices=["prune", "density"],
+                    help="prune: the pruning path (the headline); density: the textual-density kernel alone")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
@@ -160,6 +225,10 @@ def main() -> None:
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.step == "density":
+        if rank == 0:
+            run_density(args)
         return
 
     if not torch.cuda.is_available():

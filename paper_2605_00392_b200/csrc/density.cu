@@ -8,15 +8,23 @@
 // therefore the one exact arithmetic takes, and the counts do not depend on the order of anything.
 // Pixels outside the image take the value of the nearest pixel inside.
 //
-// One CTA of 256 threads per token patch (p x p pixels, p = 16, 32 or 64):
-//   1. the patch's rows are 3p contiguous bytes, 16-byte aligned (p and the image width are multiples
-//      of 16): a thread fetches 48 bytes = 16 pixels with three 16-byte loads, turns them into 16
-//      integer gray values and stores those into a (p+2) x (p+2) tile in shared memory; the one-pixel
-//      ring around the patch is fetched pixel by pixel;
-//   2. a thread walks down a column of the patch over p*p/256 rows with the horizontal sums of three
-//      rows in registers: three shared-memory loads and about a dozen integer operations per pixel.
-// The CTA writes its patch's count and adds it to the image's count (integer atomics: the result does
-// not depend on the order); a second small kernel turns the image counts into rho.
+// One CTA of 288 threads per 64 x 64 tile of pixels (one token patch of 64 x 64, or 4 / 16 patches of
+// 32 x 32 / 16 x 16):
+//   1. a tile row is up to 192 contiguous bytes, 16-byte aligned (the image width is a multiple of
+//      16): a thread fetches 48 bytes = 16 pixels with three 16-byte loads, and the one-pixel ring left
+//      and right of the tile pixel by pixel; every load of the CTA is issued before the first use (one
+//      trip to memory); the pixels become integer gray values in a 66-row tile in shared memory.  The
+//      gray value of a pixel is two dp2a instructions on the words as loaded (16-bit weights against
+//      the bytes of a word, whichever of the four alignments the 3-byte pixel has), no byte is
+//      extracted;
+//   2. 128 threads each walk down 16 rows of two adjacent columns with the horizontal sums of three
+//      rows in registers: 1.5 shared-memory loads and about a dozen integer operations per pixel; the
+//      rows and columns of a thread lie in one patch, so the counts are reduced over the lanes that
+//      share a patch and added to the patch's counter in shared memory.
+// The kernel is bound by instruction issue, not by memory, which is why the instruction count per
+// pixel is what the layout above is about.
+// The CTA writes its patches' counts and adds their sum to the image's count (integer atomics: the
+// result does not depend on the order); a second small kernel turns the image counts into rho.
 #include <cstdint>
 #include <cmath>
 
@@ -26,30 +34,55 @@
 
 namespace rtp {
 
-constexpr int kDnThreads = 256;
-constexpr int kDnMaxPatch = 64;
-constexpr int kDnPitch = kDnMaxPatch + 2 + 1;      // odd pitch of the gray tile: conflict-free column walks
+constexpr int kDnTile = 64;                        // tile side in pixels
+constexpr int kDnThreads = 288;                    // 66 rows x 4 groups of 16 pixels = 264 fetch tasks
+constexpr int kDnPitch = 72;                       // gray tile row: ring at [3], pixels at [4 .. 67], ring at [68]
 
 __device__ inline int gray_of(uint32_t r, uint32_t g, uint32_t b) { return (int)(299u * r + 587u * g + 114u * b); }
 
-__global__ void __launch_bounds__(kDnThreads)
-density_patch_kernel(const uint8_t *__restrict__ images, int H, int W, int p, unsigned long long thr2,
-                     int32_t *__restrict__ edge_counts, uint32_t *__restrict__ image_counts)
-{
-    __shared__ int s_gray[(kDnMaxPatch + 2) * kDnPitch];
-    __shared__ int s_cnt[kDnThreads / 32];
-    const int tid = threadIdx.x;
-    const int px = blockIdx.x, py = blockIdx.y, img = blockIdx.z;
-    const uint8_t *im = images + (size_t)img * H * W * 3;
-    const int x0 = px * p, y0 = py * p;
+// 16-bit weight pairs (low half | high half << 16) for dp2a: low half times the lower byte of the
+// selected byte pair of the data word, high half times the upper one.
+constexpr uint32_t kW_RG = 299u | (587u << 16);
+constexpr uint32_t kW_B0 = 114u;
+constexpr uint32_t kW_0R = 299u << 16;
+constexpr uint32_t kW_GB = 587u | (114u << 16);
 
-    // ---- gray tile: rows y0-1 .. y0+p, columns x0-1 .. x0+p (tile coordinates 0 .. p+1) -------------
-    const int groups = p >> 4;                       // 16-pixel groups per patch row
-    for (int t = tid; t < (p + 2) * groups; t += kDnThreads) {
-        const int ty = t / groups, gx = t - ty * groups;
-        const int y = min(max(y0 + ty - 1, 0), H - 1);
-        const uint4 *src = reinterpret_cast<const uint4 *>(im + ((size_t)y * W + x0 + 16 * gx) * 3);
-        uint32_t w[12];
+// Gray values of the 4 pixels whose 12 bytes are the words a, b, c (R G B R | G B R G | B R G B).
+__device__ inline int4 gray4(uint32_t a, uint32_t b, uint32_t c)
+{
+    int4 o;
+    o.x = (int)__dp2a_lo(kW_RG, a, __dp2a_hi(kW_B0, a, 0u));     // R, G = a[0], a[1]; B = a[2]
+    o.y = (int)__dp2a_hi(kW_0R, a, __dp2a_lo(kW_GB, b, 0u));     // R = a[3]; G, B = b[0], b[1]
+    o.z = (int)__dp2a_hi(kW_RG, b, __dp2a_lo(kW_B0, c, 0u));     // R, G = b[2], b[3]; B = c[0]
+    o.w = (int)__dp2a_lo(kW_0R, c, __dp2a_hi(kW_GB, c, 0u));     // R = c[1]; G, B = c[2], c[3]
+    return o;
+}
+
+__global__ void __launch_bounds__(kDnThreads, 7)
+density_tile_kernel(const uint8_t *__restrict__ images, int H, int W, int p, unsigned long long thr2,
+                    int32_t *__restrict__ edge_counts, uint32_t *__restrict__ image_counts)
+{
+    __shared__ __align__(16) int s_gray[(kDnTile + 2) * kDnPitch];
+    __shared__ int s_cnt[16];                        // up to 4 x 4 patches in a tile
+    const int tid = threadIdx.x;
+    const int img = blockIdx.z;
+    const uint8_t *im = images + (size_t)img * H * W * 3;
+    const int x0 = blockIdx.x * kDnTile, y0 = blockIdx.y * kDnTile;
+    const int tw = min(kDnTile, W - x0), th = min(kDnTile, H - y0);   // multiples of p (and of 16)
+    if (tid < 16) s_cnt[tid] = 0;
+
+    // ---- gray tile: rows y0-1 .. y0+th, columns x0-1 .. x0+tw -------------------------------------------
+    const int groups = tw >> 4;                      // 16-pixel groups per tile row
+    const bool has_group = tid < (th + 2) * groups;
+    const bool has_ring = tid < 2 * (th + 2);
+    uint32_t w[12];
+    uint32_t rc[3];
+    int g_ty = 0, g_gx = 0;
+    if (has_group) {
+        g_ty = tid / groups;
+        g_gx = tid - g_ty * groups;
+        const int y = min(max(y0 + g_ty - 1, 0), H - 1);
+        const uint4 *src = reinterpret_cast<const uint4 *>(im + ((size_t)y * W + x0 + 16 * g_gx) * 3);
 #pragma unroll
         for (int q = 0; q < 3; ++q) {
             const uint4 v = __ldg(src + q);
@@ -58,62 +91,75 @@ density_patch_kernel(const uint8_t *__restrict__ images, int H, int W, int p, un
             w[4 * q + 2] = v.z;
             w[4 * q + 3] = v.w;
         }
-        int *dst = s_gray + ty * kDnPitch + 1 + 16 * gx;
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {               // pixel k = bytes 3k .. 3k+2 of the 48
-            uint32_t c[3];
-#pragma unroll
-            for (int e = 0; e < 3; ++e) {
-                const int byte = 3 * k + e;
-                c[e] = (w[byte >> 2] >> (8 * (byte & 3))) & 0xffu;
-            }
-            dst[k] = gray_of(c[0], c[1], c[2]);
-        }
     }
-    for (int t = tid; t < 2 * (p + 2); t += kDnThreads) {    // left and right ring columns
-        const int ty = t >> 1, right = t & 1;
+    if (has_ring) {
+        const int ty = tid >> 1, right = tid & 1;
         const int y = min(max(y0 + ty - 1, 0), H - 1);
-        const int x = right ? min(x0 + p, W - 1) : max(x0 - 1, 0);
+        const int x = right ? min(x0 + tw, W - 1) : max(x0 - 1, 0);
         const uint8_t *q = im + ((size_t)y * W + x) * 3;
-        s_gray[ty * kDnPitch + (right ? p + 1 : 0)] = gray_of(__ldg(q), __ldg(q + 1), __ldg(q + 2));
+        rc[0] = __ldg(q);
+        rc[1] = __ldg(q + 1);
+        rc[2] = __ldg(q + 2);
     }
+    if (has_group) {
+        int4 *dst = reinterpret_cast<int4 *>(s_gray + g_ty * kDnPitch + 4 + 16 * g_gx);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) dst[k4] = gray4(w[3 * k4], w[3 * k4 + 1], w[3 * k4 + 2]);
+    }
+    if (has_ring) s_gray[(tid >> 1) * kDnPitch + ((tid & 1) ? 4 + tw : 3)] = gray_of(rc[0], rc[1], rc[2]);
     __syncthreads();
 
-    // ---- Sobel, threshold, count: thread = (column c, block of rows) -----------------------------------
-    const int ngroups = kDnThreads / p;              // 4, 8 or 16 row blocks
-    const int rows_per = p / ngroups;                // 16, 4 or 1
-    const int c = tid % p, r0 = (tid / p) * rows_per;
-    // horizontal sums of a tile row at this column: smooth s = l + 2 m + r, difference d = r - l
-    auto hrow = [&](int trow, int &s, int &d) {
-        const int *g = s_gray + trow * kDnPitch + c;          // tile columns c, c+1, c+2 = image x-1, x, x+1
-        const int l = g[0], m = g[1], r = g[2];
-        s = l + 2 * m + r;
-        d = r - l;
-    };
-    int s_up, d_up, s_mid, d_mid, s_dn, d_dn;
-    hrow(r0, s_up, d_up);                            // tile row r0 = image row y0 + r0 - 1
-    hrow(r0 + 1, s_mid, d_mid);
+    // ---- Sobel, threshold, count: thread = (columns 2 cp and 2 cp + 1, block of 16 rows) ------------------
+    const int cp = tid & 31, r0 = (tid >> 5) * 16;
+    const bool active = tid < 128 && 2 * cp < tw && r0 < th;
     int cnt = 0;
-    for (int r = 0; r < rows_per; ++r) {
-        hrow(r0 + r + 2, s_dn, d_dn);
-        const int gx = d_up + 2 * d_mid + d_dn;
-        const int gy = s_up - s_dn;
-        const unsigned long long g2 = (unsigned long long)((long long)gx * gx) + (unsigned long long)((long long)gy * gy);
-        cnt += (g2 >= thr2) ? 1 : 0;
-        s_up = s_mid;
-        d_up = d_mid;
-        s_mid = s_dn;
-        d_mid = d_dn;
+    if (active) {
+        // horizontal sums of a tile row at the two columns: smooth s = l + 2 m + r, difference d = r - l
+        auto hrow = [&](int trow, int &s0, int &d0, int &s1, int &d1) {
+            const int *g = s_gray + trow * kDnPitch + 3 + 2 * cp;    // image columns x-1 .. x+2, x = 2 cp
+            const int g0 = g[0];
+            const int2 g12 = *reinterpret_cast<const int2 *>(g + 1);
+            const int g3 = g[3];
+            s0 = g0 + 2 * g12.x + g12.y;
+            d0 = g12.y - g0;
+            s1 = g12.x + 2 * g12.y + g3;
+            d1 = g3 - g12.x;
+        };
+        auto edge = [&](int gx, int gy) {
+            const unsigned long long g2 =
+                (unsigned long long)((long long)gx * gx) + (unsigned long long)((long long)gy * gy);
+            return g2 >= thr2 ? 1 : 0;
+        };
+        int su0, du0, su1, du1, sm0, dm0, sm1, dm1, sd0, dd0, sd1, dd1;
+        hrow(r0, su0, du0, su1, du1);                // tile row r0 = image row y0 + r0 - 1
+        hrow(r0 + 1, sm0, dm0, sm1, dm1);
+#pragma unroll 4
+        for (int r = 0; r < 16; ++r) {               // th is a multiple of 16: the block is whole
+            hrow(r0 + r + 2, sd0, dd0, sd1, dd1);
+            cnt += edge(du0 + 2 * dm0 + dd0, su0 - sd0);
+            cnt += edge(du1 + 2 * dm1 + dd1, su1 - sd1);
+            su0 = sm0; du0 = dm0; su1 = sm1; du1 = dm1;
+            sm0 = sd0; dm0 = dd0; sm1 = sd1; dm1 = dd1;
+        }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    if ((tid & 31) == 0) s_cnt[tid >> 5] = cnt;
+    // the lanes that share a patch: p / 2 of them (a warp holds the 64 columns of one block of rows)
+    if (tid < 128) {
+        const int width = p >> 1;
+        for (int o = width >> 1; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if ((cp & (width - 1)) == 0 && active) atomicAdd(&s_cnt[(r0 / p) * (kDnTile / p) + (2 * cp) / p], cnt);
+    }
     __syncthreads();
+    const int npt = kDnTile / p;                     // patches per tile side
+    if (tid < npt * npt) {
+        const int pi = tid / npt, pj = tid - pi * npt;
+        if (pi * p < th && pj * p < tw && edge_counts) {
+            const int gy = y0 / p + pi, gx = x0 / p + pj;
+            edge_counts[((size_t)img * (H / p) + gy) * (W / p) + gx] = s_cnt[tid];
+        }
+    }
     if (tid == 0) {
         int total = 0;
-#pragma unroll
-        for (int w = 0; w < kDnThreads / 32; ++w) total += s_cnt[w];
-        if (edge_counts) edge_counts[((size_t)img * gridDim.y + py) * gridDim.x + px] = total;
+        for (int q = 0; q < npt * npt; ++q) total += s_cnt[q];
         atomicAdd(image_counts + img, (uint32_t)total);
     }
 }
@@ -140,15 +186,15 @@ extern "C" rtprune_status_t rtprune_density(void *cuda_stream, const uint8_t *im
     if (!(tau >= 0.f) || !std::isfinite(tau)) return RTPRUNE_ERR_INVALID_ARG;
     if (batch == 0) return RTPRUNE_OK;
     if (!images || !rho || !image_counts || ((uintptr_t)images & 15u)) return RTPRUNE_ERR_INVALID_ARG;
-    if (batch > 65535 || height / patch > 65535) return RTPRUNE_ERR_UNSUPPORTED;
+    if (batch > 65535 || height / kDnTile > 65535) return RTPRUNE_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     // G >= tau  <=>  Gx_int^2 + Gy_int^2 >= (255000 tau)^2; the left side is an integer
     const double t = (double)tau * 255000.0;
     const double t2 = std::ceil(t * t);
     const unsigned long long thr2 = t2 >= 1.8e19 ? ~0ull : (unsigned long long)t2;
     if (cudaMemsetAsync(image_counts, 0, sizeof(uint32_t) * (size_t)batch, st) != cudaSuccess) return RTPRUNE_ERR_CUDA;
-    dim3 grid((unsigned)(width / patch), (unsigned)(height / patch), (unsigned)batch);
-    density_patch_kernel<<<grid, kDnThreads, 0, st>>>(images, height, width, patch, thr2, edge_counts, image_counts);
+    dim3 grid((unsigned)((width + kDnTile - 1) / kDnTile), (unsigned)((height + kDnTile - 1) / kDnTile), (unsigned)batch);
+    density_tile_kernel<<<grid, kDnThreads, 0, st>>>(images, height, width, patch, thr2, edge_counts, image_counts);
     density_finish_kernel<<<(batch + 255) / 256, 256, 0, st>>>(image_counts, batch,
                                                              1.f / ((float)height * (float)width), rho);
     return cudaGetLastError() == cudaSuccess ? RTPRUNE_OK : RTPRUNE_ERR_CUDA;
