@@ -35,7 +35,7 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 f
 REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
 NCU_TRAFFIC_BYTES = {"stage1": 65893632, "gather": 10351616, "scores": 86195968,
-                     "sinkhorn_cluster": 4833280, "merge": 123877888}
+                     "sinkhorn_cluster": 4833280, "merge": 123877888, "density_tile": 318444544}
 
 
 def cpu_threads() -> int:
@@ -192,7 +192,8 @@ def run_density(args) -> None:
             "config": {"workload": "density: 64 pages x 1280 x 1280 x RGB8, patch 64, tau 0.2",
                        "l2": "pages rotate over 2 buffer sets (629 MB > L2)"},
             "roofline": {"kernel": "density_tile", "bound": "hbm", "achieved": nbytes / ms / 1e6, "peak": hbm_peak,
-                         "unit": "GB/s", "frac": nbytes / ms / 1e6 / hbm_peak, "peak_source": src, "traffic": None},
+                         "unit": "GB/s", "frac": nbytes / ms / 1e6 / hbm_peak, "peak_source": src,
+                         "traffic": NCU_TRAFFIC_BYTES["density_tile"]},
             "e2e": {"value": batch / e2e_ms * 1e3, "unit": "images/s", "h2d_bytes_per_step": nbytes,
                     "d2h_bytes_per_step": 4 * batch, "ms_per_step": e2e_ms},
             "gpu_launches": 2 * args.steps, "clocks": clocks}
