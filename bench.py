@@ -363,6 +363,16 @@ def main() -> None:
         else:
             achieved, peak, unit = units / dur_s / 1e12, FP32_FMA_PEAK_TFLOPS, "TFLOP/s"
         path_bytes = x_bytes + y_bytes + 12 * total
+        # the same figures for every kernel of the step (the per-kernel times come from events between the
+        # kernels, which serialise them: in the timed steps above they overlap)
+        per_kernel_roofline = {}
+        for name, t_ms in avg.items():
+            kb, ku = algo[name]
+            ach = ku / (t_ms / 1e3) / (1e9 if kb == "hbm" else 1e12)
+            pk = hbm_peak if kb == "hbm" else FP32_FMA_PEAK_TFLOPS
+            per_kernel_roofline[name] = {"bound": kb, "achieved": ach, "unit": "GB/s" if kb == "hbm" else "TFLOP/s",
+                                         "frac": ach / pk, "avg_launch_ms": t_ms,
+                                         "traffic": NCU_TRAFFIC_BYTES.get(name)}
         line = {
             "metric": "pruned images/sec", "value": images_s, "unit": "images/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -385,6 +395,7 @@ def main() -> None:
                               "unit": "GB/s", "frac": path_bytes / (ms_step / 1e3) / 1e9 / hbm_peak,
                               "peak_source": peak_kind},
             "kernel_ms": avg,
+            "kernel_rooflines": per_kernel_roofline,
             "e2e": {"value": e2e_images_s, "unit": "images/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "kept_rows": kept_total},
             "gpu_launches": launches,
