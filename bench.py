@@ -35,7 +35,7 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 f
 REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
 NCU_TRAFFIC_BYTES = {"stage1": 65893632, "gather": 10351616, "scores": 86195968,
-                     "sinkhorn_cluster": 4833280, "merge": 123877888, "density_tile": 318444544}
+                     "sinkhorn_cluster": 4833280, "merge": 123877888, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
