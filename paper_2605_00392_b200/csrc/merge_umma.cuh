@@ -42,7 +42,8 @@ constexpr int kMgBBoxBytes = kMgBK * 128;            // one 64-column slab of it
 // I_128 as two 128 x 64 K-major views of [64 zero rows][I_64][64 zero rows]: the view that starts at
 // the I_64 block has its ones in rows 0-63, the view that starts 64 rows earlier in rows 64-127.
 constexpr int kMgIdentBytes = 3 * (kMgABytes / 2);
-constexpr int kMgIdentKb = 2;                        // k-blocks that carry the token tile's own rows
+constexpr int kMgIdentKb = 2;                        // k-blocks that carry the token tile's own rows (one, if
+                                                     // the image ends within the tile's first 64 rows)
 constexpr int kMgStagePitch = kMgTileN * 2 + 16;     // bytes per staging row: padded, conflict-free
 constexpr int kMgStagingBytes = kMgTileM * kMgStagePitch;
 constexpr int kMgSmemBytes = kMgBStages * kMgBBytes + kMgAStages * kMgABytes + kMgIdentBytes +
@@ -63,6 +64,7 @@ struct MergeBarriers {
 struct MergeUnit {
     int img, mt, ct;
     int t_begin, N, M, B, out0;
+    int nident;       // identity k-blocks: 64-row blocks of the tile that hold tokens of the image
     bool valid;
     bool timed_out;   // the image's list entry never came
 };
@@ -123,6 +125,7 @@ __device__ inline MergeUnit merge_unit(int u, int mtiles, int nct, const int32_t
     q.M = q.valid ? __ldcg(counts + q.img) : 0;
     q.B = q.N - q.M;
     q.out0 = q.valid ? __ldcg(out_offsets + q.img) : 0;
+    q.nident = (q.N - q.mt * kMgTileM <= kMgBK) ? 1 : kMgIdentKb;
     return q;
 }
 
@@ -207,7 +210,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                 if (q.img < 0) break;
                 mq->prod = n + 1;
                 if (ready_list) ptx::fence_proxy_async_all();   // the plan was written with ordinary stores
-                const int nkb = kMgIdentKb + (q.B + kMgBK - 1) / kMgBK;
+                const int nkb = q.nident + (q.B + kMgBK - 1) / kMgBK;
                 const int row0 = q.t_begin + q.mt * kMgTileM;
                 const int xp0 = xp_row0(q.t_begin, q.img);
                 const int col0 = q.ct * kMgTileN;
@@ -221,7 +224,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                         break;
                     }
                     const uint32_t b_dst = smem_base + s * kMgBBytes;
-                    const bool own = kb < kMgIdentKb;       // the token tile's own rows: A is the identity
+                    const bool own = kb < q.nident;         // the token tile's own rows: A is the identity
                     ptx::mbar_arrive_expect_tx(&bars->full[s], (own ? 0 : kMgABytes) + nslab * kMgBBoxBytes);
                     if (!own) {
                         const int sa = ia % kMgAStages;
@@ -236,11 +239,11 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                         }
                         a_user[sa] = it;
                         ptx::tma_load_2d(ptx::smem_u32(a_ring) + sa * kMgABytes, &tmapP, &bars->full[s],
-                                         (kb - kMgIdentKb) * kMgBK, row0);
+                                         (kb - q.nident) * kMgBK, row0);
                         ++ia;
                     }
                     const CUtensorMap *bm = own ? &tmapX : &tmapXp;
-                    const int brow = own ? row0 + kb * kMgBK : xp0 + (kb - kMgIdentKb) * kMgBK;
+                    const int brow = own ? row0 + kb * kMgBK : xp0 + (kb - q.nident) * kMgBK;
                     for (int sl = 0; sl < nslab; ++sl)
                         ptx::tma_load_2d(b_dst + sl * kMgBBoxBytes, bm, &bars->full[s], col0 + sl * 64, brow);
                 }
@@ -295,7 +298,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                     break;
                 }
                 if (q.img < 0) break;
-                const int nkb = kMgIdentKb + (q.B + kMgBK - 1) / kMgBK;
+                const int nkb = q.nident + (q.B + kMgBK - 1) / kMgBK;
                 const int buf = acc & 1;
                 if (acc >= 2) {
                     if (!ptx::mbar_wait(&bars->accum_empty[buf], ((acc >> 1) - 1) & 1)) {
@@ -316,7 +319,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                     ptx::tc_fence_after();
                     // identity k-block 0: the view whose rows 0-63 are I_64; k-block 1: rows 64-127
                     uint32_t a_base;
-                    if (kb < kMgIdentKb) {
+                    if (kb < q.nident) {
                         a_base = ptx::smem_u32(ident) + (1 - kb) * (kMgABytes / 2);
                     } else {
                         a_base = ptx::smem_u32(a_ring) + (ia % kMgAStages) * kMgABytes;
@@ -375,7 +378,9 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
             ptx::bulk_wait_read<0>();                         // the previous unit's store has read this row
             const int col0 = q.ct * kMgTileN;
             const int ncols = min(kMgTileN, d - col0);
-            for (int c0 = 0; c0 < ncols; c0 += 32) {
+            // a warp whose 32 rows all lie past the image's end has nothing to convert or store
+            const bool warp_has_rows = q.mt * kMgTileM + warp * 32 < q.N;
+            for (int c0 = 0; c0 < (warp_has_rows ? ncols : 0); c0 += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kMgTileN + c0), r);
                 ptx::tmem_ld_wait();
