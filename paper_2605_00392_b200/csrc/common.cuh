@@ -18,7 +18,8 @@ struct WsHeader {
     uint32_t select_done;  // images whose selection has been published
     uint32_t n_ready;      // images whose transport plan has been published (entries of ready_list)
     uint32_t merge_next;   // next unit of the merge kernel when its CTAs draw units from a counter
-    uint32_t pad[60];
+    int32_t run_tag;       // number of the run whose counters and lists below are in place (see wait_run_tag)
+    uint32_t pad[59];
 };
 
 // Byte offsets of the workspace regions; computed on the host from the plan's maxima.
@@ -27,6 +28,7 @@ struct WsLayout {
     size_t img_done;   // uint32 [batch]           chunks of each image that have finished their pass
     size_t sink_done;  // uint32 [batch]           CTAs of each image's cluster that have written their plan rows
     size_t ready_list; // int32 [batch]            1 + image, in the order the plans were finished
+    size_t scores_done; // uint32 [batch]          score tiles of each image that are complete
     size_t clear_bytes;  // the workspace's first clear_bytes bytes (header, counters) start at zero
     size_t norms;      // float [total]            C_k
     size_t spart;      // float [batch][chunks][d] partial sums of the unit tokens

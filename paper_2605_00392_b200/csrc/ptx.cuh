@@ -74,6 +74,15 @@ __device__ inline void st_release_gpu(int *p, int v)
 {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+// Bounded wait until *p == want (acquire).  false = gave up.
+__device__ inline bool wait_equal_gpu(const int *p, int want)
+{
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (ld_acquire_gpu(p) == want) return true;
+        __nanosleep(200);
+    }
+    return false;
+}
 // 16-byte global -> shared copy; src_bytes = 0 writes 16 zero bytes without reading.
 __device__ inline void cp_async_16(uint32_t dst_smem, const void *src, uint32_t src_bytes)
 {

@@ -1,6 +1,7 @@
 // C ABI of the RTPrune pruning path: plan, argument checks, workspace layout and kernel launches.
 // Every step of the path runs in the kernels included below; this file only marshals.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -39,6 +40,8 @@ struct rtprune_plan_s {
     cudaEvent_t ev[RTPRUNE_PROFILE_MAX + 1];
     const char *ev_name[RTPRUNE_PROFILE_MAX];
     int ev_count;  // kernels recorded by the most recent run
+    int run;       // number of the most recent run's second stage, unique in the process: what the kernels
+                   // that share counters through the workspace wait for before they read them
 };
 
 // Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
@@ -47,6 +50,8 @@ struct rtprune_plan_s {
 static __device__ __align__(256) unsigned char g_static_scratch[RTPRUNE_STATIC_SCRATCH_BYTES];
 
 namespace {
+
+std::atomic<int> g_run_count{0};   // second-stage launches of the process, over all plans
 
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
@@ -68,6 +73,8 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
     L.ready_list = off;
     off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
+    L.scores_done = off;
+    off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
     L.clear_bytes = off;
     L.norms = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
@@ -313,6 +320,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     __nv_bfloat16 *pbuf = kTensor ? (__nv_bfloat16 *)(ws + L.pbuf) : nullptr;
     const int pbuf_pitch = (std::max(maxB, 1) + 63) / 64 * 64;   // <= L.pbuf_pitch_max
     int32_t *ready_list = nullptr;   // images in the order their plans are finished, when the merge follows it
+    do plan->run = ++g_run_count; while (plan->run == 0);   // 0 is what a fresh workspace holds
+    uint32_t *scores_done = nullptr; // per-image counts of finished score tiles, when the scores kernel keeps them
 
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
@@ -324,7 +333,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                      (const __nv_bfloat16 *)X, offsets, o.counts, order, plan->d, maxN, total,
                                      (__nv_bfloat16 *)(ws + L.xp), (uint32_t *)(ws + L.sink_done),
                                      (int32_t *)(ws + L.ready_list), (WsHeader *)(ws + L.header), batch,
-                                     o.out_offsets)))
+                                     o.out_offsets, (uint32_t *)(ws + L.scores_done), plan->run)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "gather");
             }
@@ -336,9 +345,14 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                 (uint64_t)plan->d * 2, kScBK, kScBBoxRows))
                 return RTPRUNE_ERR_CUDA;
             dim3 grid((maxN + kScTileM - 1) / kScTileM, batch);
+            // The Sinkhorn kernel can start on an image as soon as that image's score tiles are in.  That
+            // costs each scores CTA a release (its stores made visible before it counts itself), which
+            // pays when the grid is one wave of CTAs and its end is a tail of a few slow CTAs, not when
+            // CTAs queue for the SMs.
+            if ((long long)grid.x * grid.y <= 2LL * plan->sm_count) scores_done = (uint32_t *)(ws + L.scores_done);
             if (!c.ok(launch_pdl(scores_umma_kernel, grid, dim3(kScThreads), kScSmemBytes, st, 1u, tmapX, tmapXp,
                                  offsets, plan->d, o.counts, order, (const int32_t *)(ws + L.kpos), norms, kmat,
-                                 L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header))))
+                                 L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header), scores_done)))
                 return RTPRUNE_ERR_CUDA;
         } else {
             const int btiles = (maxB + kSimtTile - 1) / kSimtTile;
@@ -384,7 +398,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                  o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                                  fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
                                  o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
-                                 (WsHeader *)(ws + L.header))))
+                                 (WsHeader *)(ws + L.header),
+                                 ready_list ? (const uint32_t *)scores_done : (const uint32_t *)nullptr, plan->run)))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_cluster");
             if (wide) {
@@ -393,7 +408,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                      offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total,
                                      op, fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
                                      o.merge_weight, o.stats, (uint32_t *)nullptr, (int32_t *)nullptr,
-                                     (WsHeader *)nullptr)))
+                                     (WsHeader *)nullptr, (const uint32_t *)nullptr, 0)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "sinkhorn_wide");
             }
@@ -429,7 +444,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         if (!c.ok(launch_pdl(merge_umma_kernel, dim3((unsigned)grid), dim3(kMgThreads), kMgSmemBytes, st, 1u,
                              tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
                              (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
-                             (WsHeader *)(ws + L.header), (const int32_t *)ready_list)))
+                             (WsHeader *)(ws + L.header), (const int32_t *)ready_list, plan->run)))
             return RTPRUNE_ERR_CUDA;
     } else {
         const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
@@ -585,6 +600,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         return RTPRUNE_ERR_CUDA;
     }
     p->encode_tiled = nullptr;
+    p->run = 0;
     {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;

@@ -45,7 +45,7 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
                    const int32_t *__restrict__ offsets, int d, const int32_t *__restrict__ counts,
                    const int32_t *__restrict__ order, const int32_t *__restrict__ kpos,
                    const float *__restrict__ norms, float *__restrict__ kmat, int kmat_stride,
-                   int max_tokens, int total, WsHeader *__restrict__ hdr)
+                   int max_tokens, int total, WsHeader *__restrict__ hdr, uint32_t *__restrict__ scores_done)
 {
     extern __shared__ uint8_t smem_raw[];
     const int img = blockIdx.y, mt = blockIdx.x;
@@ -54,7 +54,14 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
     const int M = counts[img], B = N - M;
-    if (B == 0 || mt * kScTileM >= N) return;
+    if (mt * kScTileM >= N) return;
+    // With scores_done, every tile of a valid image is counted when it is complete (at once if nothing is
+    // pruned): the Sinkhorn kernel, launched as a programmatic dependent, starts on an image when its
+    // tiles are in.
+    if (B == 0) {
+        if (scores_done && threadIdx.x == 0) atomicAdd(&scores_done[img], 1u);
+        return;
+    }
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     ScoresBarriers *bars = reinterpret_cast<ScoresBarriers *>(smem + kScRingBytes);
@@ -204,7 +211,12 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
     }
 
     ptx::tc_fence_before();
+    if (scores_done) __threadfence();          // the epilogue's stores, before the count below
     __syncthreads();
+    if (scores_done && tid == 0) {
+        __threadfence();
+        atomicAdd(&scores_done[img], 1u);
+    }
     if (warp == 5) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kScBNMax);

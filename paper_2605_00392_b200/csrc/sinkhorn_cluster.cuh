@@ -269,30 +269,52 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                         int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
                         float *__restrict__ merge_weight, float *__restrict__ stats,
                         uint32_t *__restrict__ sink_done, int32_t *__restrict__ ready_list,
-                        WsHeader *__restrict__ hdr)
+                        WsHeader *__restrict__ hdr, const uint32_t *scores_done, int run)
 {
     extern __shared__ __align__(16) float sm[];
     const uint32_t C = ptx::cluster_nctarank(), rank = ptx::cluster_ctarank();
     const int img = blockIdx.x / C, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     ptx::grid_dep_launch();
-    ptx::grid_dep_wait();     // the scores come from the kernel ahead
+    // The scores come from the kernel ahead: wait for that grid to end, or, with per-image counts of
+    // finished score tiles, only for this image's tiles (and for the grid before leaving, so that this
+    // grid's end still implies that one's).
+    if (!scores_done) ptx::grid_dep_wait();
     int t_begin, N;
     // (a ready list is only passed when this instance is the only Sinkhorn kernel of the run, so an
     // image that leaves here needs no plan)
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) {
         sinkhorn_publish(img, C, sink_done, ready_list, hdr);
+        if (scores_done) ptx::grid_dep_wait();
         return;
     }
-    const int M = counts[img], B = N - M;
+    if (scores_done) {
+        if (tid == 0) {
+            const uint32_t want = (uint32_t)((N + 127) / 128);     // the scores kernel's 128-token tiles
+            // first the run's number: before it is there the counts are what the run before left
+            const bool tagged = ptx::wait_equal_gpu(&hdr->run_tag, run);
+            bool ok = false;
+            for (uint32_t i = 0; tagged && i < ptx::kSpinLimit && !ok; ++i) {
+                ok = (uint32_t)ptx::ld_acquire_gpu(reinterpret_cast<const int *>(scores_done + img)) >= want;
+                if (!ok) __nanosleep(200);
+            }
+            if (!ok) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+        }
+        __syncthreads();
+    }
+    const int M = __ldcg(counts + img), B = N - M;
     if (B == 0 || !sinkhorn_cluster_handles(M, B, (int)C, smem_floats)) {   // the general kernel takes it
         sinkhorn_publish(img, C, sink_done, ready_list, hdr);
+        if (scores_done) ptx::grid_dep_wait();
         return;
     }
     const bool in_smem = sinkhorn_cluster_fits(M, B, (int)C, smem_floats);
     const int ldk = sinkhorn_ldk(B);
-    if ((in_smem && ldk <= 256) == WIDE) return;             // the other instance's tile
-    const int out0 = out_offsets[img];
+    if ((in_smem && ldk <= 256) == WIDE) {                   // the other instance's tile
+        if (scores_done) ptx::grid_dep_wait();
+        return;
+    }
+    const int out0 = __ldcg(out_offsets + img);
     const int nc = ldk >> 5;
     const int rows_per = (M + (int)C - 1) / (int)C;
     const int row_lo = min(M, (int)rank * rows_per);
@@ -317,7 +339,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     const float shift = fmaxf(1.f, p.z);
     const float kappa = expf((p.z - shift) * inv_eps);
 
-    for (int i = tid; i < Ml; i += kSfThreads) m.toks[i] = __ldg(order + t_begin + row_lo + i);
+    for (int i = tid; i < Ml; i += kSfThreads) m.toks[i] = __ldcg(order + t_begin + row_lo + i);
 
     // ---- K = exp((S - c)/eps) of this CTA's rows, zero beyond column B ------------------------------
     {
@@ -482,7 +504,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                         ib = xi[r * ldk + j];
                     }
                 }
-                merged_idx[seg + j] = __ldg(order + t_begin + M + j);
+                merged_idx[seg + j] = __ldcg(order + t_begin + M + j);
                 merge_partner[seg + j] = ib;
                 merge_weight[seg + j] = b * m.vs[j];    // (K U) V, the product the plan stores
             }
@@ -497,6 +519,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
             Sg[(size_t)(row_lo + i) * ldS + j] = (m.Ks[(size_t)i * ldr + j] * m.us[i]) * m.vs[j];
         }
     }
+    if (scores_done) ptx::grid_dep_wait();
 }
 
 }  // namespace rtp

@@ -481,23 +481,31 @@ gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restri
                    const int32_t *__restrict__ counts, const int32_t *__restrict__ order, int d,
                    int max_tokens, int total, __nv_bfloat16 *__restrict__ xp, uint32_t *__restrict__ sink_done,
                    int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr, int batch,
-                   int32_t *__restrict__ out_offsets)
+                   int32_t *__restrict__ out_offsets, uint32_t *__restrict__ scores_done, int run)
 {
     __shared__ int s_scan[32];
     const int img = blockIdx.y;
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();     // counts and order come from the kernel ahead
-    // one CTA turns the counts into out_offsets while the others copy
-    if (blockIdx.x == 0 && img == 0) scan_counts<128>(counts, out_offsets, batch, s_scan);
-    // The list of finished transport plans starts empty: the merge kernel of the run before has ended
-    // (it is ahead of stage 1 in the stream), this run's Sinkhorn kernel starts after this kernel ends.
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        sink_done[img] = 0;
-        ready_list[img] = 0;
-        if (img == 0) {
+    // One CTA prepares what the kernels behind this one share through the workspace, while the others
+    // copy: it empties the per-image counters and the list of finished plans, then publishes the run's
+    // number.  Kernels launched as programmatic dependents may already be resident and must not read
+    // those words before they see that number: until then they hold what the run before left.  (That
+    // run has ended: it is ahead of stage 1 in the stream.)  It also turns the counts into out_offsets.
+    if (blockIdx.x == 0 && img == 0) {
+        for (int i = threadIdx.x; i < batch; i += 128) {
+            sink_done[i] = 0;
+            scores_done[i] = 0;
+            ready_list[i] = 0;
+        }
+        if (threadIdx.x == 0) {
             hdr->n_ready = 0;
             hdr->merge_next = 0;
         }
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) ptx::st_release_gpu(&hdr->run_tag, run);
+        scan_counts<128>(counts, out_offsets, batch, s_scan);
     }
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;

@@ -272,3 +272,44 @@ def test_runs_back_to_back_on_one_plan_leave_no_state(parity, binding):
         plan.close()
     for w in ws:                                      # and each of them is what the oracle computes
         parity.check_workload(w)
+
+
+@pytest.mark.parametrize("name,batch,bursts", [("base", 32, 40), ("large", 64, 12)])
+def test_many_runs_in_bursts_reproduce_bit_for_bit(binding, name, batch, bursts):
+    # The kernels of a run hand images to one another through counters and lists in the workspace while
+    # later kernels of the run (programmatic dependents) may already be resident.  Bursts of runs
+    # without a synchronisation, on inputs that alternate, must each reproduce the first result of
+    # their input bit for bit: a kernel that reads a counter left by the run before shows up here (the
+    # small batch leaves SMs free for dependents to become resident early).
+    dev = torch.device("cuda", 0)
+    sets = [synth.make(name, seed_offset=s, batch=batch) for s in range(3)]
+    w0 = sets[0]
+    fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
+    plan = binding.Plan(w0.d, w0.X.dtype, batch, max(s.total_tokens for s in sets), w0.max_tokens, device=dev)
+    keys = ("out_offsets", "counts", "kept_idx", "Y", "merged_idx", "merge_partner", "merge_weight")
+    try:
+        ins, ref = [], []
+        for w in sets:
+            rho = torch.from_numpy(w.rho.copy()).to(dev)
+            ins.append((w, w.X.to(dev), torch.from_numpy(w.offsets.copy()).to(dev), binding.make_params(rho, **fields), rho))
+            out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, dev)
+            plan.run(ins[-1][1], ins[-1][2], ins[-1][3], out)
+            torch.cuda.synchronize()
+            ref.append(out)
+        outs = [binding.Outputs.allocate(ins[j % 3][0].total_tokens, batch, w0.d, w0.X.dtype, dev) for j in range(6)]
+        for _ in range(bursts):
+            for j in range(6):
+                plan.run(ins[j % 3][1], ins[j % 3][2], ins[j % 3][3], outs[j])
+            torch.cuda.synchronize()
+            for j in range(6):
+                w, rf, o = ins[j % 3][0], ref[j % 3], outs[j]
+                n = int(rf.out_offsets[batch])
+                nb = w.total_tokens - n
+                for k in keys:
+                    m = n if k in ("kept_idx", "Y") else (nb if k.startswith("merge") else None)
+                    a, b = getattr(o, k), getattr(rf, k)
+                    assert torch.equal(a[:m] if m is not None else a, b[:m] if m is not None else b), k
+                o.Y.zero_()
+        assert plan.query_status() == 0
+    finally:
+        plan.close()
