@@ -110,7 +110,10 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan, int32_t d, rtprune_dtype_t 
 
 /*
  * Runs Algorithm 1 on a ragged batch, asynchronously on `cuda_stream`: no allocation, no host
- * synchronisation.  Inputs are not modified.
+ * synchronisation.  Inputs are not modified.  Each call gives its kernels a number that no other
+ * call of the process has had (they hand images to one another through the workspace and tell this
+ * run's entries from the last run's by it): do not capture the call into a CUDA graph that is
+ * replayed; call it again instead.  One workspace serves one run at a time.
  *
  *   X        DEVICE [total_tokens, d] row-major, dtype of the plan, 16-byte aligned
  *   offsets  DEVICE int32 [batch+1]: offsets[0] = 0, offsets[batch] = total_tokens, image i owns
