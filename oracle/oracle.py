@@ -70,6 +70,27 @@ def norms(T) -> np.ndarray:
     return C
 
 
+def variance(T) -> np.ndarray:
+    """Selection-metric ablation: population variance of each token over its D features."""
+    T = _f64(T)
+    C = np.empty(T.shape[0])
+    lib().rtp_oracle_variance(_dp(T), ctypes.c_int(T.shape[0]), ctypes.c_int(T.shape[1]), _dp(C))
+    return C
+
+
+def entropy(T) -> np.ndarray:
+    """Selection-metric ablation: entropy of the softmax of each token's features (a reading: the
+    paper names the metric without a formula)."""
+    T = _f64(T)
+    C = np.empty(T.shape[0])
+    lib().rtp_oracle_entropy(_dp(T), ctypes.c_int(T.shape[0]), ctypes.c_int(T.shape[1]), _dp(C))
+    return C
+
+
+def criterion(T, which: int) -> np.ndarray:
+    return (norms, variance, entropy)[which](T)
+
+
 def phi(T, C=None) -> float:
     """Eq. 8, by the i<j double loop."""
     T = _f64(T)
@@ -166,6 +187,7 @@ class Params:
     alpha: float = 0.1
     eps: float = 1.0
     iters: int = 100
+    criterion: int = 0      # ranking of stage 1: 0 l2 norm (Eq. 1), 1 variance, 2 entropy (selection-metric ablation)
 
 
 @dataclass
@@ -210,7 +232,7 @@ def run_image(T, p: Params, rho: float = 0.0, *, want_plan: bool = False,
         ctypes.c_int(int(p.dynamic)), ctypes.c_double(p.r_fixed), ctypes.c_double(p.phi_lo),
         ctypes.c_double(p.phi_hi), ctypes.c_double(p.r_max), ctypes.c_double(p.z),
         ctypes.c_double(p.alpha), ctypes.c_double(p.eps), ctypes.c_int(p.iters),
-        ctypes.c_int(int(compute_phi)), _dp(C), _dp(stats), _ip(kept), _ip(prop), _ip(partner),
+        ctypes.c_int(int(compute_phi)), ctypes.c_int(int(p.criterion)), _dp(C), _dp(stats), _ip(kept), _ip(prop), _ip(partner),
         _dp(weight), _dp(gap), _dp(Y), _dp(u), _dp(v), _dp(Pbar))
     B = N - M
     res = ImageResult(N=N, M=M, B=B, C=C, phi=float(stats[0]), rho=float(stats[1]),

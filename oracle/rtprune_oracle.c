@@ -35,6 +35,52 @@ void rtp_oracle_norms(const double *T, int N, int D, double *C)
     }
 }
 
+/*
+ * Selection-metric ablation (the table that ranks tokens by "variance" and by "entropy" instead of the
+ * l2 norm): alternative criteria C_k for stage 1; everything after the selection is unchanged
+ * (cosines still divide by the l2 norms).
+ *   variance: C_k = (1/D) sum_c (T_kc - mean_k)^2, mean_k = (1/D) sum_c T_kc  (population variance
+ *             over the D features of token k, the "dispersion" the ablation's discussion speaks of).
+ *   entropy:  the paper gives no formula.  Reading taken: the token's features are turned into a
+ *             distribution over the D channels by a softmax, p_c = exp(T_kc) / sum_c' exp(T_kc'),
+ *             and C_k = - sum_c p_c log p_c (natural logarithm); the M tokens of LARGEST criterion
+ *             are kept, as for the other two.  PARITY UNPINNED against the paper for this reading.
+ */
+void rtp_oracle_variance(const double *T, int N, int D, double *C)
+{
+    for (int k = 0; k < N; ++k) {
+        double mean = 0.0;
+        for (int c = 0; c < D; ++c)
+            mean += T[(size_t)k * D + c];
+        mean /= (double)D;
+        double acc = 0.0;
+        for (int c = 0; c < D; ++c) {
+            double dv = T[(size_t)k * D + c] - mean;
+            acc += dv * dv;
+        }
+        C[k] = acc / (double)D;
+    }
+}
+
+void rtp_oracle_entropy(const double *T, int N, int D, double *C)
+{
+    for (int k = 0; k < N; ++k) {
+        const double *t = T + (size_t)k * D;
+        double mx = t[0];
+        for (int c = 1; c < D; ++c)
+            if (t[c] > mx) mx = t[c];
+        double total = 0.0;
+        for (int c = 0; c < D; ++c)
+            total += exp(t[c] - mx);
+        double h = 0.0;
+        for (int c = 0; c < D; ++c) {
+            double p = exp(t[c] - mx) / total;
+            if (p > 0.0) h -= p * log(p);
+        }
+        C[k] = h;
+    }
+}
+
 static double floor_norm(double n) { return n > RTP_ORACLE_NORM_FLOOR ? n : RTP_ORACLE_NORM_FLOOR; }
 
 /* Eq. 8: phi = 2 / (N (N-1)) * sum_{i<j} (T_i . T_j) / (||T_i|| ||T_j||), by the double loop. */
@@ -239,12 +285,14 @@ void rtp_oracle_partners(const double *Pbar, int M, int B, int32_t *partner, dou
  *   ascending); partner[N], weight[N], gap[N] (first B valid); Y[N x D] (first M rows valid);
  *   optional (may be NULL) u[N+1], v[N+1], Pbar[(M+1)(B+1)] -- Pbar needs (N/2+1)^2 doubles at most.
  * With B == 0 stage 2 is skipped and Y is the input, unchanged.  phi is evaluated in dynamic mode
- * only when compute_phi is zero, else always.
+ * only when compute_phi is zero, else always.  criterion: 0 ranks by the l2 norm (Eq. 1), 1 by
+ * the variance, 2 by the entropy (see rtp_oracle_variance / rtp_oracle_entropy); C always
+ * returns the l2 norms, which the cosines use whatever the ranking.
  * Returns M.
  */
 int rtp_oracle_image(const double *T, int N, int D, double rho, int dynamic, double r_fixed,
                      double phi_lo, double phi_hi, double r_max, double z, double alpha,
-                     double eps, int iters, int compute_phi, double *C, double *stats,
+                     double eps, int iters, int compute_phi, int criterion, double *C, double *stats,
                      int32_t *kept, int32_t *prop, int32_t *partner, double *weight, double *gap,
                      double *Y, double *u_out, double *v_out, double *Pbar_out)
 {
@@ -259,7 +307,15 @@ int rtp_oracle_image(const double *T, int N, int D, double rho, int dynamic, dou
     stats[1] = rho;
     stats[2] = r;
     stats[3] = (double)M;
-    rtp_oracle_select(C, N, M, kept, prop);
+    if (criterion == 0) {
+        rtp_oracle_select(C, N, M, kept, prop);
+    } else {
+        double *Calt = (double *)malloc(sizeof(double) * (size_t)N);
+        if (criterion == 1) rtp_oracle_variance(T, N, D, Calt);
+        else rtp_oracle_entropy(T, N, D, Calt);
+        rtp_oracle_select(Calt, N, M, kept, prop);
+        free(Calt);
+    }
     if (B == 0) {
         for (int i = 0; i < M; ++i)
             memcpy(Y + (size_t)i * D, T + (size_t)kept[i] * D, sizeof(double) * (size_t)D);

@@ -436,3 +436,89 @@ def test_counts_and_partition(oracle):
     res1 = oracle.run_batch(X, offsets, oracle.Params(r_fixed=0.3), threads=1)
     for a, b in zip(res.images, res1.images):
         np.testing.assert_array_equal(a.Y, b.Y)
+
+
+# ------------------------------------------------- selection-metric ablation: variance, entropy
+def test_variance_hand_values_and_library(oracle):
+    T = np.array([[1.0, 1.0, 1.0, 1.0], [0.0, 2.0, 0.0, 2.0], [-3.0, 0.0, 3.0, 0.0], [1.0, 2.0, 3.0, 4.0]])
+    np.testing.assert_allclose(oracle.variance(T), [0.0, 1.0, 4.5, 1.25], rtol=0, atol=1e-15)
+    T = _tokens(31, 29, 47) + 0.3
+    np.testing.assert_allclose(oracle.variance(T), np.var(T, axis=1), rtol=1e-13)
+
+
+def test_variance_ignores_a_common_shift_and_scales_quadratically(oracle):
+    # the paper's remark on this metric: a token whose norm grows by an overall feature shift is not
+    # ranked higher by its variance
+    T = _tokens(32, 11, 40)
+    v = oracle.variance(T)
+    np.testing.assert_allclose(oracle.variance(T + 5.0), v, rtol=1e-12)
+    assert np.all(oracle.norms(T + 5.0) > oracle.norms(T))
+    np.testing.assert_allclose(oracle.variance(-3.0 * T), 9.0 * v, rtol=1e-13)
+    # and it is the mean square minus the squared mean
+    np.testing.assert_allclose(v, (T * T).mean(axis=1) - T.mean(axis=1) ** 2, rtol=1e-12)
+
+
+def test_entropy_closed_forms(oracle):
+    d = 12
+    # equal features: the uniform distribution, log d
+    assert oracle.entropy(np.full((1, d), -2.5))[0] == pytest.approx(np.log(d), abs=1e-14)
+    # one feature far above the rest: a point mass, 0
+    T = np.zeros((1, d))
+    T[0, 3] = 800.0
+    assert oracle.entropy(T)[0] == pytest.approx(0.0, abs=1e-300)
+    # two levels: k features at a, the rest at 0 -> p = e^a / (k e^a + d - k) on the k, 1 / (...) elsewhere
+    a, k = 1.7, 5
+    T = np.zeros((1, d))
+    T[0, :k] = a
+    zsum = k * np.exp(a) + (d - k)
+    p1, p0 = np.exp(a) / zsum, 1.0 / zsum
+    expect = -(k * p1 * np.log(p1) + (d - k) * p0 * np.log(p0))
+    assert oracle.entropy(T)[0] == pytest.approx(expect, abs=1e-14)
+    # large features must not overflow (max-shifted) and a common shift changes nothing
+    T = _tokens(33, 6, 30)
+    np.testing.assert_allclose(oracle.entropy(T + 700.0), oracle.entropy(T), rtol=1e-12)
+
+
+def test_entropy_matches_library(oracle):
+    from scipy.special import softmax
+    from scipy.stats import entropy as scipy_entropy
+    T = 2.0 * _tokens(34, 23, 61)
+    np.testing.assert_allclose(oracle.entropy(T), scipy_entropy(softmax(T, axis=1), axis=1), rtol=1e-12)
+    # a permutation of the features changes nothing; sharpening (scaling up) lowers the entropy
+    np.testing.assert_allclose(oracle.entropy(T[:, ::-1]), oracle.entropy(T), rtol=1e-13)
+    assert np.all(oracle.entropy(3.0 * T) < oracle.entropy(T))
+
+
+@pytest.mark.parametrize("which", [1, 2])
+def test_alternative_criterion_changes_only_the_ranking(oracle, which):
+    # stage 1 keeps the M tokens of largest criterion (ties to the lower index); everything after the
+    # selection is the unchanged pipeline applied to that split
+    T = _tokens(35 + which, 24, 16) + np.linspace(-1.0, 1.0, 24)[:, None]   # shifts separate norm and variance rankings
+    p = oracle.Params(r_fixed=0.375, criterion=which)
+    res = oracle.run_image(T, p, want_plan=True)
+    C = oracle.criterion(T, which)
+    M = 15
+    rank = sorted(range(24), key=lambda k: (-C[k], k))
+    assert res.M == M and res.kept.tolist() == sorted(rank[:M]) and res.prop.tolist() == sorted(rank[M:])
+    assert res.kept.tolist() != oracle.run_image(T, oracle.Params(r_fixed=0.375)).kept.tolist()
+    np.testing.assert_array_equal(res.C, oracle.norms(T))          # cosines still use the l2 norms
+    S = oracle.scores(T, res.C, res.kept, res.prop)
+    _, _, Pbar = oracle.sinkhorn(S)
+    np.testing.assert_allclose(res.Pbar, Pbar, rtol=1e-13)
+    np.testing.assert_allclose(res.Y, oracle.merge(T, res.kept, res.prop, Pbar), rtol=1e-13)
+
+
+def test_criterion_ties_keep_lower_index(oracle):
+    T = _tokens(38, 10, 8)
+    T[7] = T[2]
+    T[9] = T[2] + 4.0              # same variance as tokens 2 and 7, another norm
+    for which in (1, 2):
+        C = oracle.criterion(T, which)
+        assert C[7] == C[2]
+    C = oracle.variance(T)
+    assert C[9] == pytest.approx(C[2], rel=1e-12)
+    order = sorted(range(10), key=lambda k: (-oracle.variance(T)[k], k))
+    M = order.index(7)             # cut between token 2 (kept) and token 7
+    if order.index(2) < M:
+        res = oracle.run_image(T, oracle.Params(r_fixed=(10 - M) / 10.0, criterion=1))
+        assert 2 in res.kept and 7 in res.prop
