@@ -60,6 +60,16 @@ typedef enum { RTPRUNE_BF16 = 0, RTPRUNE_FP32 = 1 } rtprune_dtype_t;
 typedef enum { RTPRUNE_SINKHORN_AUTO = 0, RTPRUNE_SINKHORN_LOG = 1, RTPRUNE_SINKHORN_SCALING = 2 }
     rtprune_sinkhorn_form_t;
 
+/* Criterion C_k by which stage 1 ranks the tokens of an image (the M largest are kept).  The paper's
+ * method uses the l2 norm (Eq. 1); its ablation on the selection metric also ranks by variance and by
+ * entropy.  Only the ranking changes: the cosine scores divide by the l2 norms whatever the criterion.
+ *   L2NORM   C_k = ||T_v^k||_2                                                          (Eq. 1)
+ *   VARIANCE C_k = (1/d) sum_c (T_kc - mean_k)^2, the population variance over the d features
+ *   ENTROPY  C_k = - sum_c p_c log p_c with p = softmax of the token's d features.  The paper names
+ *            this metric without a formula: this is the library's reading of it. */
+typedef enum { RTPRUNE_CRITERION_L2NORM = 0, RTPRUNE_CRITERION_VARIANCE = 1, RTPRUNE_CRITERION_ENTROPY = 2 }
+    rtprune_criterion_t;
+
 /* Parameters of one run (Algorithm 1 inputs; Appendix C for `iters`). */
 typedef struct {
     int32_t dynamic;      /* 0: use r_fixed.  1: r = min(r_max, f_normalize(phi) (1 - rho)), Eq. 10 */
@@ -80,6 +90,7 @@ typedef struct {
                              of all `iters` iterations to fp32 accuracy.  0: always run `iters`.     */
     float tol;            /* > 0: also stop once no dual moved by more than tol (log units) in an
                              iteration.  0 (default): never stop on a tolerance.                    */
+    int32_t criterion;    /* rtprune_criterion_t: what stage 1 ranks by (default L2NORM, Eq. 1)     */
 } rtprune_params_t;
 
 /* Number of floats per image in the `stats` output. */
@@ -93,7 +104,8 @@ typedef struct {
 #define RTPRUNE_DEV_BAD_OFFSETS 4u /* an image had N_i < 1 or N_i > max_tokens_per_image */
 
 /* Fills *params with the paper's defaults: fixed r = 0.25, z = 0.2, alpha = 0.1, eps = 1,
- * iters = 100, identity f_normalize, r_max = 1, form AUTO, stop_at_fixed_point = 1, tol = 0. */
+ * iters = 100, identity f_normalize, r_max = 1, form AUTO, stop_at_fixed_point = 1, tol = 0,
+ * criterion L2NORM. */
 rtprune_status_t rtprune_default_params(rtprune_params_t *params);
 
 /*

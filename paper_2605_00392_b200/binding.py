@@ -37,7 +37,8 @@ class CParams(ctypes.Structure):
                 ("rho", ctypes.c_void_p), ("phi_lo", ctypes.c_float), ("phi_hi", ctypes.c_float),
                 ("r_max", ctypes.c_float), ("z", ctypes.c_float), ("alpha", ctypes.c_float),
                 ("eps", ctypes.c_float), ("iters", ctypes.c_int32), ("form", ctypes.c_int32),
-                ("stop_at_fixed_point", ctypes.c_int32), ("tol", ctypes.c_float)]
+                ("stop_at_fixed_point", ctypes.c_int32), ("tol", ctypes.c_float),
+                ("criterion", ctypes.c_int32)]
 
 
 _lib: Optional[ctypes.CDLL] = None

@@ -30,7 +30,8 @@ struct WsLayout {
     size_t ready_list; // int32 [batch]            1 + image, in the order the plans were finished
     size_t scores_done; // uint32 [batch]          score tiles of each image that are complete
     size_t clear_bytes;  // the workspace's first clear_bytes bytes (header, counters) start at zero
-    size_t norms;      // float [total]            C_k
+    size_t norms;      // float [total]            l2 norms (the criterion C_k of Eq. 1)
+    size_t crit;       // float [total]            C_k of a run that ranks by variance or entropy
     size_t spart;      // float [batch][chunks][d] partial sums of the unit tokens
     size_t order;      // int32 [total]            per image: kept indices then pruned indices
     size_t kpos;       // int32 [total]            per token: position among kept, or -1 - position

@@ -19,7 +19,7 @@
 
 using namespace rtp;
 
-static_assert(sizeof(rtprune_params_t) == 56, "rtprune_params_t layout is part of the ABI");
+static_assert(sizeof(rtprune_params_t) == 64, "rtprune_params_t layout is part of the ABI");
 
 struct rtprune_plan_s {
     int d;
@@ -77,6 +77,8 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
     L.clear_bytes = off;
     L.norms = off;
+    off = align_up(off + sizeof(float) * (size_t)max_total, 256);
+    L.crit = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
     L.spart = off;
     off = align_up(off + sizeof(float) * (size_t)max_batch * L.chunks * d, 256);
@@ -193,6 +195,8 @@ rtprune_status_t check_params(const rtprune_params_t *p)
     if (p->form < RTPRUNE_SINKHORN_AUTO || p->form > RTPRUNE_SINKHORN_SCALING)
         return RTPRUNE_ERR_INVALID_ARG;
     if (!(p->tol >= 0.f)) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->criterion < RTPRUNE_CRITERION_L2NORM || p->criterion > RTPRUNE_CRITERION_ENTROPY)
+        return RTPRUNE_ERR_INVALID_ARG;
     const bool scaling_safe = p->eps >= 0.25f && std::fabs(p->z) <= 4.f;
     if (p->form == RTPRUNE_SINKHORN_SCALING && !scaling_safe) return RTPRUNE_ERR_INVALID_ARG;
     return RTPRUNE_OK;
@@ -245,7 +249,8 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
         }                                                                                        \
         cudaError_t e = launch_pdl(k, grid, dim3(kS1Threads), smem, st, 1u,                      \
             (const T *)X, offsets, batch, d, L.chunks, chunk_tokens, pl->max_tokens, total, rp, rho, \
-            (float *)(ws + L.norms), (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),     \
+            (float *)(ws + L.norms), (float *)(ws + (rp.criterion ? L.crit : L.norms)),          \
+            (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),                              \
             (int32_t *)(ws + L.order), (int32_t *)(ws + L.kpos), counts, out_offsets, stats,     \
             norms_out, order_out, (WsHeader *)(ws + L.header), scan_here);                       \
         if (e != cudaSuccess) return e;                                                          \
@@ -290,7 +295,8 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
                                int32_t *order_out, bool scan_here)
 {
     Checked c{plan};
-    RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max};
+    RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max,
+                   params->criterion};
     cudaError_t e = (plan->dtype == RTPRUNE_BF16)
                         ? launch_stage1_kernel<__nv_bfloat16>(plan, st, X, offsets, batch, total, rp, params->rho,
                                                               ws, out_offsets, counts, stats, norms_out, order_out,
@@ -533,6 +539,7 @@ rtprune_status_t rtprune_default_params(rtprune_params_t *p)
     p->form = RTPRUNE_SINKHORN_AUTO;
     p->stop_at_fixed_point = 1;
     p->tol = 0.f;
+    p->criterion = RTPRUNE_CRITERION_L2NORM;
     return RTPRUNE_OK;
 }
 

@@ -1,0 +1,453 @@
+// Dustbin-augmented optimal transport by Sinkhorn iterations (Eq. 5, Appendix C) in scaling form for
+// score tiles too wide for the kernels of sinkhorn_cluster.cuh: images with many tokens (thousands
+// per image, as the OCR models with large visual token sets produce), up to 4092 pruned tokens.  One
+// cluster of 8 CTAs per image; the tile's rows (kept tokens) are split over the CTAs; K =
+// exp((S - c)/eps) is built in place in the image's workspace tile and read once per iteration
+// through L2.
+//
+// Same recursion and notation as sinkhorn_cluster.cuh (U = e^u, V = e^{v + c/eps}, the dustbin row and
+// column carried as scalars).  What differs is the layout: a thread owns fixed columns (16-byte chunks
+// ct, ct + W, ...) of every row of its row group, so the column sums K^T U live in registers across
+// the whole pass; the row sums K V are completed across the W threads of a row by shuffles and one
+// __syncthreads per block of R rows.  The column sums are reduce-scattered over the cluster: CTA r
+// owns a slice of the columns, receives the other CTAs' partial sums for it through distributed shared
+// memory, adds them in rank order, computes V for the slice and broadcasts it, so every CTA holds
+// bit-identical V and takes the same decision to stop.  Two cluster barriers per iteration.
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+#include "sinkhorn.cuh"
+#include "sinkhorn_cluster.cuh"
+
+namespace rtp {
+
+constexpr int kTallC = 8;             // CTAs per image
+constexpr int kTallThreads = 512;
+constexpr int kTallMaxB = 4092;       // row pitch (B + 4) & ~3 <= 4096 floats = 512 threads x 2 chunks
+
+// Dynamic shared memory (floats) of sinkhorn_tall_kernel for tiles of at most maxB columns and maxM rows.
+__host__ __device__ inline size_t sinkhorn_tall_smem_floats(int maxB, int maxM)
+{
+    const size_t qpr = (size_t)score_pitch(maxB) / 4;
+    const size_t sl = (qpr + kTallC - 1) / kTallC;
+    const size_t rows_cap = ((size_t)maxM + kTallC - 1) / kTallC;
+    return (4 * qpr + 4) + 2 * kTallC * 4 * sl + 2048 + 256 + 64 + 48 + 2 * (rows_cap + 4);
+}
+
+// One image's tile on one CTA of the cluster.  W threads share a row (G = 512 / W row groups), a thread
+// owns NQ 16-byte column chunks, rows are taken R per group at a time.
+template <int W, int NQ, int R>
+__device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int Ml, int row_lo, uint32_t rank,
+                                           const OtParams &p, float *sm, int rows_cap,
+                                           const int32_t *__restrict__ ord, __nv_bfloat16 *__restrict__ Pimg,
+                                           int pbuf_pitch, int32_t *__restrict__ merged_seg,
+                                           int32_t *__restrict__ partner_seg, float *__restrict__ weight_seg,
+                                           float *__restrict__ stats_img)
+{
+    constexpr int C = kTallC;
+    constexpr int G = kTallThreads / W;
+    constexpr int WPG = W / 32;
+    constexpr int kWarps = kTallThreads / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ct = tid % W, g = tid / W;
+    const int qpr = ldS >> 2;                 // 16-byte chunks per row of the tile
+    const int ldc = qpr * 4;
+    const int sl = (qpr + C - 1) / C;         // chunks per owner slice
+    const int slc = 4 * sl;                   // columns per owner slice (<= 512)
+
+    float *vs = sm;                           // [ldc + 4]      V of every column
+    float *xrecv = vs + ldc + 4;              // [2][C][slc]    partial column sums received (pairing: values, indices)
+    float *cpart = xrecv + 2 * C * slc;       // [2][1024]      row group 1's column partials (pairing: values, indices)
+    float *red = cpart + 2048;                // [2][16][8]     per-warp row-sum partials, double-buffered by block
+    float *wred = red + 256;                  // [2][16] + [2]  per-warp sums of V and moves; the groups' sums of U
+    float *xs = wred + 64;                    // [4][C]         per-CTA sums of U, sums of V, continue flags, moves
+    float *us = xs + 48;                      // [rows_cap + 4] U of this CTA's rows
+    int *toks = reinterpret_cast<int *>(us + rows_cap + 4);   // [rows_cap] token position of this CTA's rows
+
+    int cq[NQ];
+    bool cv[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        cq[q] = q * W + ct;
+        cv[q] = cq[q] < qpr;
+    }
+    const float inv_eps = 1.f / p.eps;
+    const float shift = fmaxf(1.f, p.z);
+    const float kappa = expf((p.z - shift) * inv_eps);
+    const float v_init = expf(shift * inv_eps);       // v = 0
+    const float Bf = (float)B, Mf = (float)M;
+
+    for (int i = tid; i < Ml; i += kTallThreads) {
+        toks[i] = __ldcg(ord + row_lo + i);
+        us[i] = 1.f;                                  // u = 0
+    }
+    // ---- K = exp((S - c)/eps) of this CTA's rows, in place, zero from column B on ---------------------
+    {
+        const int total_q = Ml * qpr;
+        for (int q0 = tid; q0 < total_q; q0 += kTallThreads * 4) {
+            float4 s[4];
+            int ii[4], jj[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int q = q0 + a * kTallThreads;
+                ii[a] = q / qpr;
+                jj[a] = (q - ii[a] * qpr) << 2;
+                s[a] = (q < total_q) ? __ldcg(reinterpret_cast<const float4 *>(Kg + (size_t)ii[a] * ldS + jj[a]))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int q = q0 + a * kTallThreads;
+                if (q < total_q) {
+                    float4 k;
+                    k.x = (jj[a] + 0 < B) ? exp_fast((s[a].x - shift) * inv_eps) : 0.f;
+                    k.y = (jj[a] + 1 < B) ? exp_fast((s[a].y - shift) * inv_eps) : 0.f;
+                    k.z = (jj[a] + 2 < B) ? exp_fast((s[a].z - shift) * inv_eps) : 0.f;
+                    k.w = (jj[a] + 3 < B) ? exp_fast((s[a].w - shift) * inv_eps) : 0.f;
+                    *reinterpret_cast<float4 *>(Kg + (size_t)ii[a] * ldS + jj[a]) = k;
+                }
+            }
+        }
+    }
+    for (int j = tid; j < ldc; j += kTallThreads) vs[j] = (j < B) ? v_init : 0.f;
+    __syncthreads();              // K (re-read from L2 below by other threads of this CTA), vs, us, toks
+    // every CTA of the cluster is running and has its shared memory laid out before anyone writes into it
+    ptx::cluster_sync_all();
+
+    // rows of block `blk` for this thread's group: blk * G * R + g * R + r
+    auto load_block = [&](int blk, float4 (&k)[R][NQ]) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int i = (blk * G + g) * R + r;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q)
+                k[r][q] = (i < Ml && cv[q]) ? __ldcg(reinterpret_cast<const float4 *>(Kg + (size_t)i * ldS) + cq[q])
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    const int nblk = (Ml + G * R - 1) / (G * R);
+    const uint32_t xrecv_u32 = ptx::smem_u32(xrecv), xs_u32 = ptx::smem_u32(xs), vs_u32 = ptx::smem_u32(vs);
+
+    // ---- the iterations --------------------------------------------------------------------------------
+    float sumV = Bf * v_init, Vd = v_init;    // the same in every thread of every CTA
+    int done = 0;
+    float last_move = 0.f;
+    for (int it = 0; it < p.iters; ++it) {
+        float4 V[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q)
+            V[q] = cv[q] ? *reinterpret_cast<const float4 *>(vs + 4 * cq[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float Ud = Bf * rcp_fast(kappa * (sumV + Vd));
+        const float kVd = kappa * Vd;
+        float4 colacc[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float usum = 0.f;
+
+        float4 kn[R][NQ];
+        load_block(0, kn);
+        for (int blk = 0; blk < nblk; ++blk) {
+            float4 k[R][NQ];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) k[r][q] = kn[r][q];
+            if (blk + 1 < nblk) load_block(blk + 1, kn);      // in flight during the reduction below
+            float s[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float a = 0.f;
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    a = fmaf(k[r][q].x, V[q].x, a);
+                    a = fmaf(k[r][q].y, V[q].y, a);
+                    a = fmaf(k[r][q].z, V[q].z, a);
+                    a = fmaf(k[r][q].w, V[q].w, a);
+                }
+                s[r] = warp_sum(a);
+            }
+            float *rb = red + (blk & 1) * 128;
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) rb[warp * 8 + r] = s[r];
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < WPG; ++w) t += rb[(g * WPG + w) * 8 + r];
+                const int i = (blk * G + g) * R + r;
+                const bool valid = i < Ml;
+                const float U = valid ? rcp_fast(t + kVd) : 0.f;
+                if (ct == 0 && valid) {
+                    us[i] = U;
+                    usum += U;
+                }
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    colacc[q].x = fmaf(k[r][q].x, U, colacc[q].x);
+                    colacc[q].y = fmaf(k[r][q].y, U, colacc[q].y);
+                    colacc[q].z = fmaf(k[r][q].z, U, colacc[q].z);
+                    colacc[q].w = fmaf(k[r][q].w, U, colacc[q].w);
+                }
+            }
+        }
+        // the row groups' column partials and sums of U meet in group 0
+        if (ct == 0) wred[32 + g] = usum;
+        if constexpr (G == 2) {
+            if (g == 1) {
+#pragma unroll
+                for (int q = 0; q < NQ; ++q)
+                    if (cv[q]) *reinterpret_cast<float4 *>(cpart + 4 * cq[q]) = colacc[q];
+            }
+        }
+        __syncthreads();
+        if (g == 0) {
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                if (!cv[q]) continue;
+                float4 cs = colacc[q];
+                if constexpr (G == 2) {
+                    const float4 o = *reinterpret_cast<const float4 *>(cpart + 4 * cq[q]);
+                    cs.x += o.x;
+                    cs.y += o.y;
+                    cs.z += o.z;
+                    cs.w += o.w;
+                }
+                // to the CTA that owns these columns
+                const int owner = cq[q] / sl, off = cq[q] - owner * sl;
+                const uint32_t a = ptx::map_to_rank(xrecv_u32 + (uint32_t)((rank * slc) + 4 * off) * 4u, (uint32_t)owner);
+                ptx::st_cluster_f32(a, cs.x);
+                ptx::st_cluster_f32(a + 4u, cs.y);
+                ptx::st_cluster_f32(a + 8u, cs.z);
+                ptx::st_cluster_f32(a + 12u, cs.w);
+            }
+        }
+        if (tid == 0) {
+            float su = wred[32];
+            if constexpr (G == 2) su += wred[33];
+            for (uint32_t r = 0; r < (uint32_t)C; ++r)
+                ptx::st_cluster_f32(ptx::map_to_rank(xs_u32 + rank * 4u, r), su);
+        }
+        ptx::cluster_sync_all();
+
+        // ---- this CTA's slice of V from the completed column sums, broadcast to the cluster -----------
+        float su_all = 0.f;
+#pragma unroll
+        for (int r = 0; r < C; ++r) su_all += xs[r];          // read here: the next pass may overwrite it early
+        int cont = 0;
+        float move = 0.f, nv = 0.f;
+        const int j = (int)rank * slc + tid;
+        if (tid < slc && j < B) {
+            float cs = 0.f;
+#pragma unroll
+            for (int r = 0; r < C; ++r) cs += xrecv[r * slc + tid];
+            nv = rcp_fast(cs + kappa * Ud);
+            const float ov = vs[j];
+            move = fabsf(nv - ov) * rcp_fast(ov);
+            cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
+            const uint32_t a = vs_u32 + (uint32_t)j * 4u;
+#pragma unroll
+            for (uint32_t r = 0; r < (uint32_t)C; ++r) ptx::st_cluster_f32(ptx::map_to_rank(a, r), nv);
+        }
+        const float wv = warp_sum(nv), wm = warp_max(move);
+        if (lane == 0) {
+            wred[warp] = wv;
+            wred[16 + warp] = wm;
+        }
+        cont = __syncthreads_or(cont);
+        if (tid == 0) {
+            float sv = 0.f, mv = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                sv += wred[w];
+                mv = fmaxf(mv, wred[16 + w]);
+            }
+            for (uint32_t r = 0; r < (uint32_t)C; ++r) {
+                ptx::st_cluster_f32(ptx::map_to_rank(xs_u32 + (uint32_t)(C + rank) * 4u, r), sv);
+                ptx::st_cluster_f32(ptx::map_to_rank(xs_u32 + (uint32_t)(2 * C + rank) * 4u, r), cont ? 1.f : 0.f);
+                ptx::st_cluster_f32(ptx::map_to_rank(xs_u32 + (uint32_t)(3 * C + rank) * 4u, r), mv);
+            }
+        }
+        ptx::cluster_sync_all();
+
+        // every thread of every CTA: the sums, the dustbin column, the decision to go on
+        const float nVd = Mf * rcp_fast(kappa * (su_all + Ud));
+        const float md = fabsf(nVd - Vd) * rcp_fast(Vd);
+        bool go = p.tol > 0.f ? (md > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : true);
+        float sv_all = 0.f, mv_all = md;
+#pragma unroll
+        for (int r = 0; r < C; ++r) {
+            sv_all += xs[C + r];
+            go = go || (xs[2 * C + r] != 0.f);
+            mv_all = fmaxf(mv_all, xs[3 * C + r]);
+        }
+        sumV = sv_all;
+        Vd = nVd;
+        last_move = mv_all;
+        ++done;
+        if (!go) break;
+    }
+    if (rank == 0 && tid == 0) {
+        stats_img[5] = (float)done;
+        stats_img[6] = last_move;
+    }
+
+    // ---- plan P = U K V of this CTA's rows, and per column the best K_ij U_i over them ------------------
+    const int kpad = (B + 63) & ~63;          // the tensor-core merge reads whole 64-column blocks
+    {
+        float4 V[NQ];
+        float best[NQ][4];
+        int bi[NQ][4];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            V[q] = cv[q] ? *reinterpret_cast<const float4 *>(vs + 4 * cq[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                best[q][e] = -INFINITY;
+                bi[q][e] = 0x7fffffff;
+            }
+        }
+        for (int blk = 0; blk < nblk; ++blk) {
+            float4 k[R][NQ];
+            load_block(blk, k);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = (blk * G + g) * R + r;
+                if (i >= Ml) continue;
+                const float U = us[i];
+                const int tok = toks[i];
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (!cv[q]) continue;
+                    const float ku[4] = {k[r][q].x * U, k[r][q].y * U, k[r][q].z * U, k[r][q].w * U};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (ku[e] > best[q][e]) {        // rows ascend within a thread: strict > keeps the lower index
+                            best[q][e] = ku[e];
+                            bi[q][e] = row_lo + i;
+                        }
+                    }
+                    const float4 P = make_float4(ku[0] * V[q].x, ku[1] * V[q].y, ku[2] * V[q].z, ku[3] * V[q].w);
+                    if (Pimg) {
+                        if (4 * cq[q] < kpad) {          // alpha P in bf16, row = the kept token's position in X
+                            __nv_bfloat162 o[2];
+                            o[0] = __floats2bfloat162_rn(p.alpha * P.x, p.alpha * P.y);
+                            o[1] = __floats2bfloat162_rn(p.alpha * P.z, p.alpha * P.w);
+                            *reinterpret_cast<uint2 *>(Pimg + (size_t)tok * pbuf_pitch + 4 * cq[q]) =
+                                *reinterpret_cast<uint2 *>(o);
+                        }
+                    } else {
+                        *reinterpret_cast<float4 *>(Kg + (size_t)i * ldS + 4 * cq[q]) = P;   // fp32: in place
+                    }
+                }
+            }
+        }
+        if (Pimg && kpad > ldc) {             // zero columns between the tile's pitch and the 64-column block's end
+            const int zq = (kpad - ldc) >> 2;
+            for (int idx = tid; idx < Ml * zq; idx += kTallThreads) {
+                const int i = idx / zq, c = idx - i * zq;
+                *reinterpret_cast<uint2 *>(Pimg + (size_t)toks[i] * pbuf_pitch + ldc + 4 * c) = make_uint2(0u, 0u);
+            }
+        }
+        // pairing: the row groups meet in group 0, the CTAs in the owner of the column
+        int *cparti = reinterpret_cast<int *>(cpart + 1024);
+        if constexpr (G == 2) {
+            if (g == 1) {
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (!cv[q]) continue;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        cpart[4 * cq[q] + e] = best[q][e];
+                        cparti[4 * cq[q] + e] = bi[q][e];
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        if (g == 0) {
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                if (!cv[q]) continue;
+                const int owner = cq[q] / sl, off = cq[q] - owner * sl;
+                const uint32_t a = ptx::map_to_rank(xrecv_u32 + (uint32_t)((rank * slc) + 4 * off) * 4u, (uint32_t)owner);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float b = best[q][e];
+                    int ib = bi[q][e];
+                    if constexpr (G == 2) {
+                        const float ob = cpart[4 * cq[q] + e];
+                        const int oi = cparti[4 * cq[q] + e];
+                        if (ob > b || (ob == b && oi < ib)) {
+                            b = ob;
+                            ib = oi;
+                        }
+                    }
+                    ptx::st_cluster_f32(a + 4u * e, b);
+                    ptx::st_cluster_u32(a + (uint32_t)(C * slc) * 4u + 4u * e, (uint32_t)ib);
+                }
+            }
+        }
+        ptx::cluster_sync_all();      // after this barrier nothing is written into another CTA any more
+        const int j = (int)rank * slc + tid;
+        if (tid < slc && j < B) {
+            const int *xi = reinterpret_cast<const int *>(xrecv + C * slc);
+            float b = xrecv[tid];
+            int ib = xi[tid];
+#pragma unroll
+            for (int r = 1; r < C; ++r) {      // ranks hold ascending row ranges: strict > keeps the lower index
+                const float ob = xrecv[r * slc + tid];
+                if (ob > b) {
+                    b = ob;
+                    ib = xi[r * slc + tid];
+                }
+            }
+            merged_seg[j] = __ldcg(ord + M + j);
+            partner_seg[j] = ib;
+            weight_seg[j] = b * vs[j];          // (K U) V, the product the plan stores
+        }
+    }
+}
+
+// grid = batch * 8 CTAs, clusters of 8 along x.  Takes the images that the cluster kernels ahead of it
+// left (fast_c, fast_floats: their cluster size and shared-memory floats) and whose B <= kTallMaxB; every
+// early return depends on the image only, so a cluster leaves as a whole.
+__global__ void __launch_bounds__(kTallThreads, 1)
+sinkhorn_tall_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__ counts,
+                     const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ order,
+                     float *__restrict__ kmat, int kmat_stride, int max_tokens, int total, OtParams p,
+                     __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch, int32_t *__restrict__ merged_idx,
+                     int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
+                     float *__restrict__ stats, int fast_c, int fast_floats)
+{
+    extern __shared__ __align__(16) float sm[];
+    const uint32_t rank = ptx::cluster_ctarank();
+    const int img = blockIdx.x / kTallC;
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();         // scores, counts and order come from the kernels ahead
+    int t_begin, N;
+    if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
+    const int M = __ldcg(counts + img), B = N - M;
+    if (B == 0 || B > kTallMaxB) return;
+    if (fast_c > 0 && sinkhorn_cluster_handles(M, B, fast_c, fast_floats)) return;   // solved ahead of this kernel
+    const int rows_per = (M + kTallC - 1) / kTallC;
+    const int row_lo = min(M, (int)rank * rows_per);
+    const int Ml = min(M, row_lo + rows_per) - row_lo;       // this CTA's rows (may be 0)
+    const int ldS = score_pitch(B);
+    float *Kg = kmat + kmat_offset(kmat_stride, t_begin, img) + (size_t)row_lo * ldS;
+    const int seg = t_begin - __ldcg(out_offsets + img);
+    __nv_bfloat16 *Pimg = pbuf ? pbuf + (size_t)t_begin * pbuf_pitch : nullptr;
+    const int qpr = ldS >> 2;
+#define RTP_TALL(W, NQ, R)                                                                                     \
+    sinkhorn_tall_solve<W, NQ, R>(Kg, ldS, M, B, Ml, row_lo, rank, p, sm, rows_per, order + t_begin, Pimg,     \
+                                  pbuf_pitch, merged_idx + seg, merge_partner + seg, merge_weight + seg,      \
+                                  stats + (size_t)img * kStats)
+    if (qpr <= 256) RTP_TALL(256, 1, 8);
+    else if (qpr <= 512) RTP_TALL(512, 1, 8);
+    else RTP_TALL(512, 2, 4);
+#undef RTP_TALL
+}
+
+}  // namespace rtp

@@ -10,6 +10,7 @@ namespace rtp {
 struct RatioParams {
     int dynamic;
     float r_fixed, phi_lo, phi_hi, r_max;
+    int criterion;      // 0 l2 norm (Eq. 1), 1 variance, 2 entropy of the softmax of the features
 };
 
 constexpr int kS1Threads = 256;
@@ -64,8 +65,9 @@ __device__ inline int block_excl_scan(int v, int *scratch)
 
 // ---------------------------------------------------------------------------------------------
 // Selection of one image by one CTA (256 threads): phi from the chunk partials; r and
-// B = floor(r N + 1/2) clamped to [0, N-1], M = N - B; the M tokens of largest norm (ties to the lower
-// index) are T_kept.  The M-th largest norm is found by a radix select over the norm bits (four
+// B = floor(r N + 1/2) clamped to [0, N-1], M = N - B; the M tokens of largest criterion (`norms`: the
+// l2 norms, or the variance / entropy values of a run that ranks by those; ties to the lower
+// index) are T_kept.  The M-th largest value is found by a radix select over its bits (four
 // 8-bit digits, a 256-bin histogram each), tokens equal to it are admitted in index order.  Writes
 // order[] = kept indices ascending, then pruned indices ascending, and its inverse kpos[]; counts,
 // stats.
@@ -136,18 +138,25 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
             local = fmaf(a4[a].w, a4[a].w, local);
         }
     }
-    // norm bits: for non-negative floats the unsigned order is the float order, and a NaN still ranks
+    // norm bits: for non-negative floats the unsigned order is the float order, and a NaN still ranks.
+    // The other criteria may round to just below zero: sign-aware map of the bits to unsigned order.
+    const bool signed_keys = rp.criterion != 0;
+    auto key_bits = [&](float c) -> uint32_t {
+        const uint32_t b = __float_as_uint(c);
+        if (!signed_keys) return b & 0x7fffffffu;
+        return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    };
 #pragma unroll
     for (int q = 0; q < kKeysAhead; ++q) {
         const int k = tid + q * nth;
         if (k < N) {
-            s_keys[k] = __float_as_uint(key_r[q]) & 0x7fffffffu;
+            s_keys[k] = key_bits(key_r[q]);
             if (norms_out) norms_out[t_begin + k] = key_r[q];
         }
     }
     for (int k = tid + kKeysAhead * nth; k < N; k += nth) {
         const float key = __ldcg(norms + t_begin + k);
-        s_keys[k] = __float_as_uint(key) & 0x7fffffffu;
+        s_keys[k] = key_bits(key);
         if (norms_out) norms_out[t_begin + k] = key;
     }
     const float ssum = block_sum(local, s_redf);
@@ -314,7 +323,7 @@ template <typename T, int VPL>  // VPL = 16-byte vectors per lane = ceil(d / (32
 __global__ void __launch_bounds__(kS1Threads, 2)
 stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int batch, int d, int chunks,
               int chunk_tokens, int max_tokens, int total, RatioParams rp, const float *__restrict__ rho,
-              float *norms, float *spart, uint32_t *img_done, int32_t *__restrict__ order,
+              float *norms, float *critv, float *spart, uint32_t *img_done, int32_t *__restrict__ order,
               int32_t *__restrict__ kpos, int32_t *counts, int32_t *__restrict__ out_offsets,
               float *__restrict__ stats, float *__restrict__ norms_out, int32_t *__restrict__ order_out,
               WsHeader *hdr, int scan_here)
@@ -400,6 +409,65 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
                 if (!(ss <= 3.0e38f)) bad = true;  // inf or NaN
                 const float inv = 1.f / fmaxf(n, kNormFloor);
                 if (lane == 0) norms[t] = n;
+                if (rp.criterion != 0) {           // uniform over the grid: the ranking of the ablation
+                    float cval;
+                    if (rp.criterion == 1) {
+                        // variance over the d features, two passes over the row held in registers
+                        float sum = 0.f;
+#pragma unroll
+                        for (int j = 0; j < VPL; ++j) {
+                            float f[EPV];
+                            Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) sum += f[e];      // lanes past the row hold zeros
+                        }
+                        const float mean = warp_sum(sum) / (float)d;
+                        float dev2 = 0.f;
+#pragma unroll
+                        for (int j = 0; j < VPL; ++j) {
+                            if (lane + 32 * j < nvec) {
+                                float f[EPV];
+                                Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                                for (int e = 0; e < EPV; ++e) dev2 = fmaf(f[e] - mean, f[e] - mean, dev2);
+                            }
+                        }
+                        cval = warp_sum(dev2) / (float)d;
+                    } else {
+                        // entropy of softmax(row): log(sum e^(x-m)) - sum (x-m) e^(x-m) / sum e^(x-m)
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < VPL; ++j) {
+                            if (lane + 32 * j < nvec) {
+                                float f[EPV];
+                                Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                                for (int e = 0; e < EPV; ++e) mx = fmaxf(mx, f[e]);
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                        float se = 0.f, sxe = 0.f;
+#pragma unroll
+                        for (int j = 0; j < VPL; ++j) {
+                            if (lane + 32 * j < nvec) {
+                                float f[EPV];
+                                Elem<T>::unpack(cur[j], f);
+#pragma unroll
+                                for (int e = 0; e < EPV; ++e) {
+                                    const float dx = f[e] - mx;
+                                    const float ex = expf(dx);
+                                    se += ex;
+                                    sxe = fmaf(dx, ex, sxe);
+                                }
+                            }
+                        }
+                        se = warp_sum(se);
+                        sxe = warp_sum(sxe);
+                        cval = logf(se) - sxe / se;
+                    }
+                    if (lane == 0) critv[t] = cval;
+                }
 #pragma unroll
                 for (int j = 0; j < VPL; ++j) {
                     float f[EPV];
@@ -449,7 +517,7 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
         __syncthreads();
         if (!s_last) return;
         __threadfence();
-        select_image(img, t_begin, n_img, d, chunks, chunk_tokens, rp, rho, norms, spart, order, kpos, counts, stats,
+        select_image(img, t_begin, n_img, d, chunks, chunk_tokens, rp, rho, critv, spart, order, kpos, counts, stats,
                      norms_out, order_out, reinterpret_cast<uint32_t *>(s_dyn));
     }
 

@@ -36,7 +36,7 @@ def oracle_params(p: Dict[str, float]) -> oracle.Params:
                          phi_lo=float(np.float32(p["phi_lo"])), phi_hi=float(np.float32(p["phi_hi"])),
                          r_max=float(np.float32(p["r_max"])), z=float(np.float32(p["z"])),
                          alpha=float(np.float32(p["alpha"])), eps=float(np.float32(p["eps"])),
-                         iters=int(p["iters"]))
+                         iters=int(p["iters"]), criterion=int(p.get("criterion", 0)))
 
 
 def cpu_threads() -> int:
@@ -82,7 +82,7 @@ def run_gpu(w: synth.Workload, *, overrides: Optional[Dict[str, float]] = None,
         plan = binding.Plan(w.d, w.X.dtype, max(w.batch, 1), max(w.total_tokens, 1),
                             max(w.max_tokens, 1), device=dev)
     rho_dev = torch.from_numpy(w.rho.copy()).to(dev) if w.batch else None
-    fields = {k: (int(v) if k in ("dynamic", "iters", "form", "stop_at_fixed_point") else float(v))
+    fields = {k: (int(v) if k in ("dynamic", "iters", "form", "stop_at_fixed_point", "criterion") else float(v))
               for k, v in p.items()}
     if host_path:
         params = binding.make_params(None, **fields)

@@ -34,7 +34,7 @@ def test_host_only_calls():
     assert abs(p.r_fixed - 0.25) < 1e-7 and abs(p.z - 0.2) < 1e-7 and abs(p.alpha - 0.1) < 1e-7
     assert p.eps == 1.0 and p.tol == 0.0 and p.rho is None
     assert lib.rtprune_default_params(None) == 1
-    assert ctypes.sizeof(binding.CParams) == 56      # static_assert-ed in the library too
+    assert ctypes.sizeof(binding.CParams) == 64      # static_assert-ed in the library too
 
 
 def test_plan_argument_checks_come_before_any_cuda_call():
