@@ -15,6 +15,7 @@
 #include "scores_umma.cuh"
 #include "sinkhorn.cuh"
 #include "sinkhorn_cluster.cuh"
+#include "sinkhorn_tall.cuh"
 #include "stage1.cuh"
 
 using namespace rtp;
@@ -419,16 +420,33 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 launched(plan, st, "sinkhorn_wide");
             }
         }
+        // Scaling form, tiles the cluster kernels left (more than 32 * kSfMaxNc columns): clusters of 8
+        // CTAs iterate on K in the workspace tile; the general kernel keeps only what is wider still.
+        const bool tall = !use_log_form(params) && !all_fast;
+        if (tall) {
+            const size_t tall_smem = sizeof(float) * sinkhorn_tall_smem_floats(std::min(maxB, kTallMaxB), maxN);
+            if (tall_smem > 48 * 1024 &&
+                !c.ok(cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)tall_smem)))
+                return RTPRUNE_ERR_CUDA;
+            if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * kTallC)), dim3(kTallThreads),
+                                 tall_smem, st, (unsigned)kTallC, offsets, o.counts, o.out_offsets, order, kmat,
+                                 L.kmat_stride, maxN, total, op, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
+                                 o.merge_weight, o.stats, fast_c, fast_floats)))
+                return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "sinkhorn_tall");
+            if (maxB <= kTallMaxB) all_fast = true;       // nothing is left for the general kernel
+        }
         if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                o.stats, 0, 0);
+                o.stats, 0, 0, 0);
         else if (!all_fast)
             sinkhorn_kernel<false><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                o.stats, fast_c, fast_floats);
+                o.stats, fast_c, fast_floats, tall ? kTallMaxB : 0);
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
         if (use_log_form(params) || !all_fast) launched(plan, st, "sinkhorn");
     }

@@ -86,7 +86,7 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
                 int smem_floats, __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch,
                 int32_t *__restrict__ merged_idx,
                 int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
-                float *__restrict__ stats, int fast_cluster, int fast_smem_floats)
+                float *__restrict__ stats, int fast_cluster, int fast_smem_floats, int tall_max_b)
 {
     extern __shared__ __align__(16) float sm[];
     __shared__ float s_red[32];
@@ -100,6 +100,7 @@ sinkhorn_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__
     if (B == 0) return;
     // images the cluster kernel launched before this one takes were solved there
     if (fast_cluster > 0 && sinkhorn_cluster_handles(M, B, fast_cluster, fast_smem_floats)) return;
+    if (B <= tall_max_b) return;     // solved by the kernel for wide tiles (sinkhorn_tall.cuh)
     const int R = M + 1, Cc = B + 1;
 
     float *u = sm;

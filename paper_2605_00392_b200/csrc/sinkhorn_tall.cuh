@@ -34,6 +34,47 @@ __host__ __device__ inline size_t sinkhorn_tall_smem_floats(int maxB, int maxM)
     return (4 * qpr + 4) + 2 * kTallC * 4 * sl + 2048 + 256 + 64 + 48 + 2 * (rows_cap + 4);
 }
 
+// Sums of R values over the 32 lanes of a warp in 9 (R = 8) or 6 (R = 4) shuffles: every step halves the
+// values a lane carries (it keeps one half and hands the other to its partner), so the lanes end up
+// holding the total of row `row_of_lane<R>(lane)`.  The order of the additions is the same in every warp.
+template <int R> __device__ inline int row_of_lane(int lane)
+{
+    if constexpr (R == 8) return ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+    else return ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+}
+template <int R> __device__ inline float warp_rows_sum(const float (&s)[R], int lane)
+{
+    static_assert(R == 8 || R == 4, "rows per block");
+    float t2[2];
+    if constexpr (R == 8) {
+        float t4[4];
+        const bool hi = lane & 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            t4[i] = (hi ? s[i + 4] : s[i]) + __shfl_xor_sync(0xffffffffu, hi ? s[i] : s[i + 4], 16);
+        const bool hi8 = lane & 8;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            t2[i] = (hi8 ? t4[i + 2] : t4[i]) + __shfl_xor_sync(0xffffffffu, hi8 ? t4[i] : t4[i + 2], 8);
+        const bool hi4 = lane & 4;
+        float t = (hi4 ? t2[1] : t2[0]) + __shfl_xor_sync(0xffffffffu, hi4 ? t2[0] : t2[1], 4);
+        t += __shfl_xor_sync(0xffffffffu, t, 2);
+        t += __shfl_xor_sync(0xffffffffu, t, 1);
+        return t;
+    } else {
+        const bool hi = lane & 16;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            t2[i] = (hi ? s[i + 2] : s[i]) + __shfl_xor_sync(0xffffffffu, hi ? s[i] : s[i + 2], 16);
+        const bool hi8 = lane & 8;
+        float t = (hi8 ? t2[1] : t2[0]) + __shfl_xor_sync(0xffffffffu, hi8 ? t2[0] : t2[1], 8);
+        t += __shfl_xor_sync(0xffffffffu, t, 4);
+        t += __shfl_xor_sync(0xffffffffu, t, 2);
+        t += __shfl_xor_sync(0xffffffffu, t, 1);
+        return t;
+    }
+}
+
 // One image's tile on one CTA of the cluster.  W threads share a row (G = 512 / W row groups), a thread
 // owns NQ 16-byte column chunks, rows are taken R per group at a time.
 template <int W, int NQ, int R>
@@ -164,26 +205,28 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
                     a = fmaf(k[r][q].z, V[q].z, a);
                     a = fmaf(k[r][q].w, V[q].w, a);
                 }
-                s[r] = warp_sum(a);
+                s[r] = a;
             }
+            // this warp's part of the R row sums: one lane per row writes it
+            const float wsum = warp_rows_sum<R>(s, lane);
             float *rb = red + (blk & 1) * 128;
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < R; ++r) rb[warp * 8 + r] = s[r];
-            }
+            if ((lane & (32 / R - 1)) == 0) rb[warp * 8 + row_of_lane<R>(lane)] = wsum;
             __syncthreads();
+            // every warp adds the WPG parts of each row in the same order: lane l takes row l % R
+            const int rr = lane % R, wq = lane / R;
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < WPG * R / 32; ++w) t += rb[(g * WPG + wq + w * (32 / R)) * 8 + rr];
+#pragma unroll
+            for (int o = R; o < 32; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            const int i0 = (blk * G + g) * R;
+            const bool valid_own = i0 + rr < Ml;
+            const float Uown = valid_own ? rcp_fast(t + kVd) : 0.f;
+            if (ct < R && valid_own) us[i0 + rr] = Uown;      // ct < R: lane ct of the group's first warp, rr = ct
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                float t = 0.f;
-#pragma unroll
-                for (int w = 0; w < WPG; ++w) t += rb[(g * WPG + w) * 8 + r];
-                const int i = (blk * G + g) * R + r;
-                const bool valid = i < Ml;
-                const float U = valid ? rcp_fast(t + kVd) : 0.f;
-                if (ct == 0 && valid) {
-                    us[i] = U;
-                    usum += U;
-                }
+                const float U = __shfl_sync(0xffffffffu, Uown, r);
+                if (ct == 0) usum += U;
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     colacc[q].x = fmaf(k[r][q].x, U, colacc[q].x);

@@ -104,11 +104,11 @@ def test_large_tile_leaves_shared_memory(parity):
 
 def test_tile_wider_than_the_cluster_kernel_takes(parity):
     # N = 1400 at r = 0.5: 700 pruned tokens, more than the 640 columns the cluster kernels cover, so
-    # this image is solved by the general kernel (K iterated in the workspace) while the other two are
-    # solved by the two instances of the cluster kernel in the same run
+    # this image is solved by the kernel for wide tiles (clusters of 8 CTAs, K iterated in the workspace)
+    # while the other two are solved by the two instances of the cluster kernel in the same run
     w = synth.ragged([1400, 300, 1000], params=dict(r_fixed=0.5))
     rep = parity.check_workload(w)
-    assert rep["launches"] == 7      # stage1, gather, scores, sinkhorn_cluster, sinkhorn_wide, sinkhorn, merge
+    assert rep["launches"] == 7      # stage1, gather, scores, sinkhorn_cluster, sinkhorn_wide, sinkhorn_tall, merge
 
 
 def test_exact_ties_keep_lower_index(parity):
