@@ -208,10 +208,86 @@ def run_density(args) -> None:
     print(json.dumps(line))
 
 
+LARGE_N = {   # token counts before -> after pruning of the OCR models with large visual token sets (the paper's
+              # cross-model table); the fixed ratio is 1 - after / before
+    "2137": dict(tokens=2137, kept=1238, batch=16),
+    "4512": dict(tokens=4512, kept=2783, batch=8),
+}
+
+
+def run_large_n(args) -> None:
+    """`--step largen`: the whole path on images of thousands of tokens (score tiles of 4 to 19 MB that
+    no cluster's shared memory holds: the Sinkhorn kernel for wide tiles).  One GPU; one JSON line with
+    one entry per shape."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruning path has no CPU fallback")
+    from paper_2605_00392_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    hbm_peak, _, peak_kind = measured_peaks()
+    steps, warm = max(1, min(args.steps, 30)), max(args.warmup, 3)
+    shapes = {}
+    for name, cfg in LARGE_N.items():
+        n, batch = cfg["tokens"], cfg["batch"]
+        r = float(np.float32(1.0 - cfg["kept"] / n))
+        w = synth.ragged([n] * batch, seed=21, params=dict(r_fixed=r))
+        plan = binding.Plan(w.d, w.X.dtype, w.batch, w.total_tokens, w.max_tokens, device=dev)
+        fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w.params.items()}
+        params = binding.make_params(None, **fields)
+        out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, dev)
+        X, offs = w.X.to(dev), torch.from_numpy(w.offsets.copy()).to(dev)
+        flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)      # larger than L2
+        for _ in range(warm):
+            plan.run(X, offs, params, out)
+        torch.cuda.synchronize()
+        assert plan.query_status() == 0
+        plan.profile_enable(True)
+        total_ms, per_kernel = 0.0, {}
+        for _ in range(steps):
+            flush.zero_()                                  # no step finds its input in L2
+            plan.run(X, offs, params, out)
+            for kname, ms in plan.profile_read():
+                per_kernel.setdefault(kname, []).append(ms)
+                total_ms += ms
+        plan.profile_enable(False)
+        st = out.stats.cpu().numpy()[:batch]
+        M, B, it = st[:, 3].astype(np.int64), st[:, 4].astype(np.int64), st[:, 5]
+        avg = {k: float(np.mean(v)) for k, v in per_kernel.items()}
+        ms_step = total_ms / steps
+        # the wide-tile Sinkhorn kernel must read K (M rows of pitch (B+4)&~3 floats) once per iteration
+        k_bytes = float(np.sum(it * M * ((B + 4) & ~3) * 4))
+        tall_ms = avg.get("sinkhorn_tall", 0.0)
+        path_bytes = w.total_tokens * w.d * 2 + int(M.sum()) * w.d * 2 + 12 * w.total_tokens
+        shapes[name] = {
+            "workload": "%d images x %d tokens x %d bf16, fixed r = %.4f (%d kept), T=100" % (batch, n, w.d, r, int(M[0])),
+            "ms_per_step": ms_step, "images_per_s": batch / (ms_step / 1e3),
+            "tokens_per_s": w.total_tokens / (ms_step / 1e3), "kernel_ms": avg,
+            "mean_iterations_run": float(it.mean()), "max_iterations_run": float(it.max()),
+            "roofline": {"kernel": "sinkhorn_tall", "bound": "hbm", "achieved": k_bytes / (tall_ms / 1e3) / 1e9 if tall_ms else None,
+                         "peak": hbm_peak, "unit": "GB/s", "frac": k_bytes / (tall_ms / 1e3) / 1e9 / hbm_peak if tall_ms else None,
+                         "peak_source": peak_kind, "traffic": None, "avg_launch_ms": tall_ms,
+                         "note": "bytes = executed iterations x the image's K tile; the tiles of a batch stay in L2 when they fit"},
+            "path_roofline": {"bound": "hbm", "algorithmic_bytes": path_bytes,
+                              "frac": path_bytes / (ms_step / 1e3) / 1e9 / hbm_peak},
+            "gpu_launches": plan.last_launch_count * steps,
+        }
+        if name == "2137" and not args.no_cpu_baseline:
+            threads = cpu_threads()
+            sec = time_oracle(w, list(range(batch)), threads)
+            shapes[name]["cpu_baseline"] = {"value": batch / sec, "unit": "images/s", "cores": threads, "kind": "oracle",
+                                            "sample": "all %d images of this batch, once" % batch}
+        plan.close()
+    print(json.dumps({"metric": "pruned images/sec", "unit": "images/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "timing": "sum of the kernels' CUDA-event times per step, L2 flushed between steps",
+                      "shapes": shapes}), flush=True)
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("--step", default="prune", choices=["prune", "density"],
-                    help="prune: the pruning path (the headline); density: the textual-density kernel alone")
+    ap.add_argument("--step", default="prune", choices=["prune", "density", "largen"],
+                    help="prune: the pruning path (the headline); density: the textual-density kernel alone; "
+                         "largen: the pruning path on images of 2137 and 4512 tokens")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
@@ -230,6 +306,10 @@ def main() -> None:
     if args.step == "density":
         if rank == 0:
             run_density(args)
+        return
+    if args.step == "largen":
+        if rank == 0:
+            run_large_n(args)
         return
 
     if not torch.cuda.is_available():

@@ -422,17 +422,20 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         }
         // Scaling form, tiles the cluster kernels left (more than 32 * kSfMaxNc columns): clusters of 8
         // CTAs iterate on K in the workspace tile; the general kernel keeps only what is wider still.
-        const bool tall = !use_log_form(params) && !all_fast;
+        // It takes all the shared memory a CTA can have: what its fixed regions leave is the ring of row blocks.
+        const size_t tall_smem = (size_t)std::max(plan->smem_optin - 1024, 0);
+        const bool tall = !use_log_form(params) && !all_fast &&
+                          sizeof(float) * (sinkhorn_tall_smem_floats(std::min(maxB, kTallMaxB), maxN) +
+                                           kTallStageFloatsMax) <= tall_smem;
         if (tall) {
-            const size_t tall_smem = sizeof(float) * sinkhorn_tall_smem_floats(std::min(maxB, kTallMaxB), maxN);
-            if (tall_smem > 48 * 1024 &&
-                !c.ok(cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (!c.ok(cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)tall_smem)))
                 return RTPRUNE_ERR_CUDA;
             if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * kTallC)), dim3(kTallThreads),
                                  tall_smem, st, (unsigned)kTallC, offsets, o.counts, o.out_offsets, order, kmat,
                                  L.kmat_stride, maxN, total, op, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
-                                 o.merge_weight, o.stats, fast_c, fast_floats)))
+                                 o.merge_weight, o.stats, fast_c, fast_floats, (int)(tall_smem / sizeof(float)),
+                                 (WsHeader *)(ws + L.header))))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_tall");
             if (maxB <= kTallMaxB) all_fast = true;       // nothing is left for the general kernel

@@ -3,7 +3,9 @@
 // per image, as the OCR models with large visual token sets produce), up to 4092 pruned tokens.  One
 // cluster of 8 CTAs per image; the tile's rows (kept tokens) are split over the CTAs; K =
 // exp((S - c)/eps) is built in place in the image's workspace tile and read once per iteration
-// through L2.
+// through L2: a CTA's rows are contiguous there, so one thread streams them block by block into a ring
+// of shared-memory stages with 1-D bulk copies, a few blocks ahead of the threads (the tile does not
+// change between iterations, so the stream runs on across the end of an iteration).
 //
 // Same recursion and notation as sinkhorn_cluster.cuh (U = e^u, V = e^{v + c/eps}, the dustbin row and
 // column carried as scalars).  What differs is the layout: a thread owns fixed columns (16-byte chunks
@@ -31,8 +33,10 @@ __host__ __device__ inline size_t sinkhorn_tall_smem_floats(int maxB, int maxM)
     const size_t qpr = (size_t)score_pitch(maxB) / 4;
     const size_t sl = (qpr + kTallC - 1) / kTallC;
     const size_t rows_cap = ((size_t)maxM + kTallC - 1) / kTallC;
-    return (4 * qpr + 4) + 2 * kTallC * 4 * sl + 2048 + 256 + 64 + 48 + 2 * (rows_cap + 4);
+    return (4 * qpr + 4) + 2 * kTallC * 4 * sl + 2048 + 256 + 64 + 48 + 2 * (rows_cap + 4) + 4;
 }
+constexpr int kTallMaxStages = 4;
+constexpr int kTallStageFloatsMax = 16384;      // a block of rows is at most 64 KB (see the three layouts)
 
 // Sums of R values over the 32 lanes of a warp in 9 (R = 8) or 6 (R = 4) shuffles: every step halves the
 // values a lane carries (it keeps one half and hands the other to its partner), so the lanes end up
@@ -79,7 +83,8 @@ template <int R> __device__ inline float warp_rows_sum(const float (&s)[R], int 
 // owns NQ 16-byte column chunks, rows are taken R per group at a time.
 template <int W, int NQ, int R>
 __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int Ml, int row_lo, uint32_t rank,
-                                           const OtParams &p, float *sm, int rows_cap,
+                                           const OtParams &p, float *sm, int smem_floats, uint64_t *full,
+                                           WsHeader *__restrict__ hdr, int rows_cap,
                                            const int32_t *__restrict__ ord, __nv_bfloat16 *__restrict__ Pimg,
                                            int pbuf_pitch, int32_t *__restrict__ merged_seg,
                                            int32_t *__restrict__ partner_seg, float *__restrict__ weight_seg,
@@ -104,6 +109,10 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
     float *xs = wred + 64;                    // [4][C]         per-CTA sums of U, sums of V, continue flags, moves
     float *us = xs + 48;                      // [rows_cap + 4] U of this CTA's rows
     int *toks = reinterpret_cast<int *>(us + rows_cap + 4);   // [rows_cap] token position of this CTA's rows
+    const int fixed_floats = (int)((us + rows_cap + 4 + rows_cap) - sm + 3) & ~3;
+    float *ring = sm + fixed_floats;          // [NS][G R ldS]  blocks of rows of K on their way to the threads
+    const int stage_floats = G * R * ldS;
+    const int NS = max(1, min(kTallMaxStages, (smem_floats - fixed_floats) / stage_floats));
 
     int cq[NQ];
     bool cv[NQ];
@@ -151,6 +160,11 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         }
     }
     for (int j = tid; j < ldc; j += kTallThreads) vs[j] = (j < B) ? v_init : 0.f;
+    if (tid == 0) {
+        for (int s = 0; s < kTallMaxStages; ++s) ptx::mbar_init(&full[s], 1);
+        ptx::fence_mbar_init();
+    }
+    ptx::fence_proxy_async_all();     // K was stored through the generic proxy; the bulk copies read it
     __syncthreads();              // K (re-read from L2 below by other threads of this CTA), vs, us, toks
     // every CTA of the cluster is running and has its shared memory laid out before anyone writes into it
     ptx::cluster_sync_all();
@@ -167,6 +181,23 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         }
     };
     const int nblk = (Ml + G * R - 1) / (G * R);
+    // The stream of blocks: load n brings block n % nblk into stage n % NS; it is issued once every thread
+    // has taken block n - NS out of that stage (the __syncthreads of that block).  At most iters * nblk
+    // loads are ever needed; those still in flight when the loop ends early are waited for below.
+    const uint32_t n_max = (uint32_t)min((long long)p.iters * nblk, 0x7fffffffLL);
+    const uint32_t ring_u32 = ptx::smem_u32(ring);
+    auto issue = [&](uint32_t n) {
+        const int blk = (int)(n % (uint32_t)nblk), s = (int)(n % (uint32_t)NS);
+        const int rows = min(G * R, Ml - blk * G * R);
+        const uint32_t bytes = (uint32_t)rows * (uint32_t)ldS * 4u;
+        ptx::mbar_arrive_expect_tx(&full[s], bytes);
+        ptx::bulk_load(ring_u32 + (uint32_t)s * (uint32_t)stage_floats * 4u, Kg + (size_t)blk * G * R * ldS, bytes,
+                       &full[s]);
+    };
+    if (tid == 0)
+        for (uint32_t n = 0; n < min((uint32_t)NS, n_max); ++n) issue(n);
+    uint32_t n = 0;               // blocks taken so far, over all iterations
+    bool gave_up = false;
     const uint32_t xrecv_u32 = ptx::smem_u32(xrecv), xs_u32 = ptx::smem_u32(xs), vs_u32 = ptx::smem_u32(vs);
 
     // ---- the iterations --------------------------------------------------------------------------------
@@ -185,15 +216,22 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         float usum = 0.f;
 
-        float4 kn[R][NQ];
-        load_block(0, kn);
-        for (int blk = 0; blk < nblk; ++blk) {
+        for (int blk = 0; blk < nblk; ++blk, ++n) {
+            const int stg = (int)(n % (uint32_t)NS);
+            if (!gave_up && !ptx::mbar_wait(&full[stg], (n / (uint32_t)NS) & 1u)) gave_up = true;
             float4 k[R][NQ];
+            {
+                const float *rows = ring + (size_t)stg * stage_floats + (size_t)g * R * ldS;
 #pragma unroll
-            for (int r = 0; r < R; ++r)
+                for (int r = 0; r < R; ++r) {
+                    const int i = (blk * G + g) * R + r;
 #pragma unroll
-                for (int q = 0; q < NQ; ++q) k[r][q] = kn[r][q];
-            if (blk + 1 < nblk) load_block(blk + 1, kn);      // in flight during the reduction below
+                    for (int q = 0; q < NQ; ++q)
+                        k[r][q] = (i < Ml && cv[q] && !gave_up)
+                                      ? *reinterpret_cast<const float4 *>(rows + (size_t)r * ldS + 4 * cq[q])
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
             float s[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -212,6 +250,7 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
             float *rb = red + (blk & 1) * 128;
             if ((lane & (32 / R - 1)) == 0) rb[warp * 8 + row_of_lane<R>(lane)] = wsum;
             __syncthreads();
+            if (tid == 0 && n + (uint32_t)NS < n_max) issue(n + (uint32_t)NS);    // the stage is free again
             // every warp adds the WPG parts of each row in the same order: lane l takes row l % R
             const int rr = lane % R, wq = lane / R;
             float t = 0.f;
@@ -336,6 +375,13 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         stats_img[5] = (float)done;
         stats_img[6] = last_move;
     }
+    // loads issued for iterations that did not run: wait for them before this CTA's shared memory goes away
+    if (tid == 0) {
+        const uint32_t n_issued = min(n + (uint32_t)NS, n_max);
+        for (uint32_t m = n; m < n_issued; ++m)
+            if (!ptx::mbar_wait(&full[m % (uint32_t)NS], (m / (uint32_t)NS) & 1u)) gave_up = true;
+    }
+    if (gave_up) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
 
     // ---- plan P = U K V of this CTA's rows, and per column the best K_ij U_i over them ------------------
     const int kpad = (B + 63) & ~63;          // the tensor-core merge reads whole 64-column blocks
@@ -463,9 +509,11 @@ sinkhorn_tall_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
                      float *__restrict__ kmat, int kmat_stride, int max_tokens, int total, OtParams p,
                      __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch, int32_t *__restrict__ merged_idx,
                      int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight,
-                     float *__restrict__ stats, int fast_c, int fast_floats)
+                     float *__restrict__ stats, int fast_c, int fast_floats, int smem_floats,
+                     WsHeader *__restrict__ hdr)
 {
     extern __shared__ __align__(16) float sm[];
+    __shared__ uint64_t s_full[kTallMaxStages];
     const uint32_t rank = ptx::cluster_ctarank();
     const int img = blockIdx.x / kTallC;
     ptx::grid_dep_launch();
@@ -484,7 +532,8 @@ sinkhorn_tall_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     __nv_bfloat16 *Pimg = pbuf ? pbuf + (size_t)t_begin * pbuf_pitch : nullptr;
     const int qpr = ldS >> 2;
 #define RTP_TALL(W, NQ, R)                                                                                     \
-    sinkhorn_tall_solve<W, NQ, R>(Kg, ldS, M, B, Ml, row_lo, rank, p, sm, rows_per, order + t_begin, Pimg,     \
+    sinkhorn_tall_solve<W, NQ, R>(Kg, ldS, M, B, Ml, row_lo, rank, p, sm, smem_floats, s_full, hdr, rows_per,  \
+                                  order + t_begin, Pimg,                                                      \
                                   pbuf_pitch, merged_idx + seg, merge_partner + seg, merge_weight + seg,      \
                                   stats + (size_t)img * kStats)
     if (qpr <= 256) RTP_TALL(256, 1, 8);
