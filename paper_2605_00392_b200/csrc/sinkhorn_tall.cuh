@@ -198,6 +198,13 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         for (uint32_t n = 0; n < min((uint32_t)NS, n_max); ++n) issue(n);
     uint32_t n = 0;               // blocks taken so far, over all iterations
     bool gave_up = false;
+    // byte offsets inside a stage: this thread's row slot, a row, its chunks (a chunk past the row's end is
+    // replaced by the thread's first one: it is read, weighted by V = 0, and its column sums are dropped)
+    const uint32_t stage_bytes = (uint32_t)stage_floats * 4u, row_bytes = (uint32_t)ldS * 4u;
+    const uint32_t lane_off = (uint32_t)g * (uint32_t)R * row_bytes;
+    uint32_t chunk_off[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) chunk_off[q] = 16u * (uint32_t)(cv[q] ? cq[q] : (cv[0] ? cq[0] : 0));
     const uint32_t xrecv_u32 = ptx::smem_u32(xrecv), xs_u32 = ptx::smem_u32(xs), vs_u32 = ptx::smem_u32(vs);
 
     // ---- the iterations --------------------------------------------------------------------------------
@@ -216,42 +223,66 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         float usum = 0.f;
 
-        for (int blk = 0; blk < nblk; ++blk, ++n) {
-            const int stg = (int)(n % (uint32_t)NS);
-            if (!gave_up && !ptx::mbar_wait(&full[stg], (n / (uint32_t)NS) & 1u)) gave_up = true;
-            float4 k[R][NQ];
-            {
-                const float *rows = ring + (size_t)stg * stage_floats + (size_t)g * R * ldS;
+        // A block's work has two halves: (a) its rows out of the ring, their partial sums against V, this
+        // warp's part of the R row sums to shared memory; (b) after a __syncthreads, the row sums, U, and the
+        // column accumulation.  Half (a) of block b + 1 is issued ahead of half (b) of block b, so the two
+        // dependent chains (shuffle trees, the reciprocal) overlap; one __syncthreads per block.
+        auto first_half = [&](int blk, uint32_t nn, float4 (&kk)[R][NQ]) {
+            const uint32_t stg = nn % (uint32_t)NS;
+            if (!gave_up && !ptx::mbar_wait(&full[stg], (nn / (uint32_t)NS) & 1u)) gave_up = true;
+            const uint32_t base = ring_u32 + stg * stage_bytes + lane_off;
+            float s[R];
+            if ((blk * G + g + 1) * R <= Ml && !gave_up) {       // all R rows exist: nothing to mask but the columns
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float a = 0.f;
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        // (threads past the row's end read a chunk of their own row slot: finite values
+                        // from the tile, multiplied by V = 0 here and never sent on)
+                        kk[r][q] = ptx::ld_shared_v4(base + (uint32_t)r * row_bytes + chunk_off[q]);
+                        a = fmaf(kk[r][q].x, V[q].x, a);
+                        a = fmaf(kk[r][q].y, V[q].y, a);
+                        a = fmaf(kk[r][q].z, V[q].z, a);
+                        a = fmaf(kk[r][q].w, V[q].w, a);
+                    }
+                    s[r] = a;
+                }
+            } else {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     const int i = (blk * G + g) * R + r;
+                    float a = 0.f;
 #pragma unroll
-                    for (int q = 0; q < NQ; ++q)
-                        k[r][q] = (i < Ml && cv[q] && !gave_up)
-                                      ? *reinterpret_cast<const float4 *>(rows + (size_t)r * ldS + 4 * cq[q])
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int q = 0; q < NQ; ++q) {
+                        kk[r][q] = (i < Ml && cv[q] && !gave_up)
+                                       ? ptx::ld_shared_v4(base + (uint32_t)r * row_bytes + chunk_off[q])
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                        a = fmaf(kk[r][q].x, V[q].x, a);
+                        a = fmaf(kk[r][q].y, V[q].y, a);
+                        a = fmaf(kk[r][q].z, V[q].z, a);
+                        a = fmaf(kk[r][q].w, V[q].w, a);
+                    }
+                    s[r] = a;
                 }
-            }
-            float s[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float a = 0.f;
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    a = fmaf(k[r][q].x, V[q].x, a);
-                    a = fmaf(k[r][q].y, V[q].y, a);
-                    a = fmaf(k[r][q].z, V[q].z, a);
-                    a = fmaf(k[r][q].w, V[q].w, a);
-                }
-                s[r] = a;
             }
             // this warp's part of the R row sums: one lane per row writes it
             const float wsum = warp_rows_sum<R>(s, lane);
-            float *rb = red + (blk & 1) * 128;
-            if ((lane & (32 / R - 1)) == 0) rb[warp * 8 + row_of_lane<R>(lane)] = wsum;
-            __syncthreads();
-            if (tid == 0 && n + (uint32_t)NS < n_max) issue(n + (uint32_t)NS);    // the stage is free again
+            if ((lane & (32 / R - 1)) == 0) red[(blk & 1) * 128 + warp * 8 + row_of_lane<R>(lane)] = wsum;
+        };
+        float4 kn[R][NQ];
+        if (nblk > 0) first_half(0, n, kn);
+        for (int blk = 0; blk < nblk; ++blk, ++n) {
+            __syncthreads();      // the parts of block blk's row sums are in; every thread holds its K values
+            if (tid == 0 && n + (uint32_t)NS < n_max) issue(n + (uint32_t)NS);    // so its stage is free again
+            float4 k[R][NQ];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) k[r][q] = kn[r][q];
+            if (blk + 1 < nblk) first_half(blk + 1, n + 1, kn);
             // every warp adds the WPG parts of each row in the same order: lane l takes row l % R
+            const float *rb = red + (blk & 1) * 128;
             const int rr = lane % R, wq = lane / R;
             float t = 0.f;
 #pragma unroll
@@ -265,7 +296,7 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const float U = __shfl_sync(0xffffffffu, Uown, r);
-                if (ct == 0) usum += U;
+                usum += U;                                    // (only the group's first thread's sum is used)
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     colacc[q].x = fmaf(k[r][q].x, U, colacc[q].x);
