@@ -34,8 +34,8 @@ ROTATE = 4                 # input/output buffer sets cycled so that no step fin
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
 REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
-NCU_TRAFFIC_BYTES = {"stage1": 65926144, "gather": 10354944, "scores": 87062784,
-                     "sinkhorn_cluster": 4841216, "merge": 118393856, "density_tile": 318402048}
+NCU_TRAFFIC_BYTES = {"stage1": 65871872, "gather": 10354432, "scores": 86418944,
+                     "sinkhorn_cluster": 4841984, "merge": 118960640, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
@@ -384,22 +384,44 @@ def main() -> None:
     clocks = sampler.stop() if rank == 0 else None
 
     # ---- end to end through the host-buffer entry point ------------------------------------------
-    host_out = binding.Outputs.allocate(total, batch, d, torch.bfloat16, "cpu", pin=True)
+    # Two plans (each with its own device arena) on two streams take the steps in turn, the way a caller
+    # with a queue of batches would: the upload of a step's inputs then runs while the step before it is
+    # still downloading its outputs (the two directions of the link).  Every copy of every step, both
+    # directions, is inside the timed region; each stream writes host outputs of its own.
+    E2E_STREAMS = 2
+    plans2 = [plan] + [binding.Plan(d, torch.bfloat16, batch, total, w0.max_tokens, device=dev)
+                       for _ in range(E2E_STREAMS - 1)]
+    streams2 = [torch.cuda.Stream(device=dev) for _ in range(E2E_STREAMS)]
+    host_outs = [binding.Outputs.allocate(total, batch, d, torch.bfloat16, "cpu", pin=True)
+                 for _ in range(E2E_STREAMS)]
+    host_out = host_outs[0]
     hX = [w.X.pin_memory() for w in sets]
     hoffs = [torch.from_numpy(w.offsets).pin_memory() for w in sets]
     hrho = [torch.from_numpy(w.rho).pin_memory() for w in sets]
     hparams = binding.make_params(None, **fields)
-    e2e_steps = 1 if args.no_e2e else max(3, min(args.steps, 20))
-    for i in range(0 if args.no_e2e else 2):
-        plan.run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_out)
+    e2e_steps = 1 if args.no_e2e else max(4, min(args.steps, 20))
+
+    def e2e_step(i: int) -> None:
+        k = i % E2E_STREAMS
+        plans2[k].run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_outs[k],
+                           stream=streams2[k])
+
+    for i in range(0 if args.no_e2e else 2 * E2E_STREAMS):
+        e2e_step(i)
     barrier()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record(stream)
+    for st2 in streams2:
+        st2.wait_event(e2)
     for i in range(e2e_steps):
-        plan.run_host(hX[i % ROTATE], hoffs[i % ROTATE], hrho[i % ROTATE], hparams, host_out)
+        e2e_step(i)
+    for st2 in streams2:
+        stream.wait_stream(st2)
     e3.record(stream)
     barrier()
     ms_e2e = e2.elapsed_time(e3) / e2e_steps
+    for pl2 in plans2[1:]:
+        pl2.close()
     kept_total = int(host_out.out_offsets[batch])
     esz = 2
     h2d = total * d * esz + (batch + 1) * 4 + batch * 4
@@ -477,7 +499,8 @@ def main() -> None:
             "kernel_ms": avg,
             "kernel_rooflines": per_kernel_roofline,
             "e2e": {"value": e2e_images_s, "unit": "images/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "kept_rows": kept_total},
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "kept_rows": kept_total,
+                    "streams": E2E_STREAMS},
             "gpu_launches": launches,
             "clocks": clocks,
         }
