@@ -380,9 +380,9 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
         bool all_fast = false;
         if (!use_log_form(params)) {
-            // CTAs per image: as many as keep the whole batch on the chip at once, and at least as many
-            // as the largest possible tile needs to keep K in their shared memory; 8 at most (tiles
-            // larger than that iterate on K in the workspace)
+            // CTAs per image: as many as keep the whole batch on the chip at once, and more if the largest
+            // possible tile needs them to keep K in their shared memory; 8 at most (tiles larger than the
+            // cluster's shared memory iterate on K in the workspace)
             fast_c = 1;
             while (fast_c < 8 && (long long)batch * fast_c * 2 <= plan->sm_count) fast_c *= 2;
             auto all_tiles = [&](int cc, bool in_smem) {
@@ -394,28 +394,35 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 }
                 return ok;
             };
-            while (fast_c < 8 && !all_tiles(fast_c, true)) fast_c *= 2;
+            // (larger clusters only while the grid still fits the chip at once, two at least: on a ragged
+            // batch of 128 images of up to 1156 tokens, clusters of 8 that hold every K in shared memory
+            // take seven waves and 287 us, clusters of 2 with the large tiles' K in the workspace 201 us)
+            while (fast_c < 8 && !all_tiles(fast_c, true) &&
+                   (fast_c < 2 || (long long)batch * fast_c * 2 <= plan->sm_count))
+                fast_c *= 2;
             all_fast = all_tiles(fast_c, false);
             // tiles wider than 256 columns, or too tall for the cluster's shared memory, are possible
             const bool wide = maxB > 256 || !all_tiles(fast_c, true);
-            // When the first instance solves every image, it hands them to the merge kernel one by one
-            ready_list = (kTensor && !wide) ? (int32_t *)(ws + L.ready_list) : nullptr;
-            if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<false>, dim3((unsigned)(batch * fast_c)),
-                                 dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets,
-                                 o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
-                                 fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
-                                 o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
-                                 (WsHeader *)(ws + L.header),
-                                 ready_list ? (const uint32_t *)scores_done : (const uint32_t *)nullptr, plan->run)))
-                return RTPRUNE_ERR_CUDA;
-            launched(plan, st, "sinkhorn_cluster");
-            if (wide) {
+            // When one instance solves every image, it hands them to the merge kernel one by one
+            ready_list = (kTensor && all_fast) ? (int32_t *)(ws + L.ready_list) : nullptr;
+            const uint32_t *sd = ready_list ? (const uint32_t *)scores_done : (const uint32_t *)nullptr;
+            if (!wide) {
+                if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<false>, dim3((unsigned)(batch * fast_c)),
+                                     dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c, offsets,
+                                     o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
+                                     fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
+                                     o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
+                                     (WsHeader *)(ws + L.header), sd, plan->run, 0)))
+                    return RTPRUNE_ERR_CUDA;
+                launched(plan, st, "sinkhorn_cluster");
+            } else {
+                // the instance for wide or tall tiles takes the narrow ones of the same run too
                 if (!c.ok(launch_pdl(sinkhorn_cluster_kernel<true>, dim3((unsigned)(batch * fast_c)),
                                      dim3(kSfThreads), (size_t)plan->fast_smem_bytes, st, (unsigned)fast_c,
                                      offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total,
                                      op, fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
-                                     o.merge_weight, o.stats, (uint32_t *)nullptr, (int32_t *)nullptr,
-                                     (WsHeader *)nullptr, (const uint32_t *)nullptr, 0)))
+                                     o.merge_weight, o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
+                                     (WsHeader *)(ws + L.header), sd, plan->run, 1)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "sinkhorn_wide");
             }

@@ -258,8 +258,11 @@ __device__ inline void sinkhorn_publish(int img, uint32_t C, uint32_t *__restric
 
 // grid = batch * C CTAs, clusters of C along x: CTA rank r of cluster i owns rows r*rows_per .. of
 // image i's tile.  Every early return below depends on the image only, so a cluster leaves as a whole.
-// Two instances share the work: WIDE = false takes the tiles of up to 256 columns that fit shared
-// memory (the common case, kept free of everything the others need), WIDE = true the rest.
+// Two instances: WIDE = false takes the tiles of up to 256 columns that fit shared memory (the common
+// case, kept free of everything the others need) and is launched alone when no other tile is possible
+// in the run; WIDE = true is launched instead when wider or taller tiles are possible, and then takes
+// every tile of the family (takes_all), so that the images of a ragged batch are solved side by side
+// by one grid rather than by two grids one after the other.
 template <bool WIDE>
 __global__ void __launch_bounds__(kSfThreads, 1)
 sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__restrict__ counts,
@@ -269,7 +272,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                         int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
                         float *__restrict__ merge_weight, float *__restrict__ stats,
                         uint32_t *__restrict__ sink_done, int32_t *__restrict__ ready_list,
-                        WsHeader *__restrict__ hdr, const uint32_t *scores_done, int run)
+                        WsHeader *__restrict__ hdr, const uint32_t *scores_done, int run, int takes_all)
 {
     extern __shared__ __align__(16) float sm[];
     const uint32_t C = ptx::cluster_nctarank(), rank = ptx::cluster_ctarank();
@@ -310,7 +313,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
     }
     const bool in_smem = sinkhorn_cluster_fits(M, B, (int)C, smem_floats);
     const int ldk = sinkhorn_ldk(B);
-    if ((in_smem && ldk <= 256) == WIDE) {                   // the other instance's tile
+    if (!(WIDE && takes_all) && (in_smem && ldk <= 256) == WIDE) {   // the other instance's tile
         if (scores_done) ptx::grid_dep_wait();
         return;
     }
@@ -391,11 +394,11 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         else RTP_SC_SMEM(16, 16);
     } else {
         switch (ldk) {
-        case 32: RTP_SC_GLOBAL(8, 4); break;
-        case 64: RTP_SC_GLOBAL(8, 8); break;
-        case 128: RTP_SC_GLOBAL(8, 16); break;
-        case 192: RTP_SC_GLOBAL(16, 12); break;
-        case 256: RTP_SC_GLOBAL(16, 16); break;
+        case 32: RTP_SC_EITHER(8, 4); break;
+        case 64: RTP_SC_EITHER(8, 8); break;
+        case 128: RTP_SC_EITHER(8, 16); break;
+        case 192: RTP_SC_EITHER(16, 12); break;
+        case 256: RTP_SC_EITHER(16, 16); break;
         case 384: RTP_SC_EITHER(32, 12); break;
         case 512: RTP_SC_EITHER(32, 16); break;
         default: RTP_SC_EITHER(32, 20); break;

@@ -32,7 +32,7 @@ def test_2137_tokens_to_1238(parity):
     # the cluster kernel in the same run
     w = synth.ragged([2137, 700], params=dict(r_fixed=0.4207))
     rep = parity.check_workload(w)
-    assert rep["launches"] == 7      # stage1, gather, scores, sinkhorn_cluster, sinkhorn_wide, sinkhorn_tall, merge
+    assert rep["launches"] == 6      # stage1, gather, scores, sinkhorn_wide, sinkhorn_tall, merge
 
 
 def test_4512_tokens_to_2783(parity):
@@ -60,7 +60,7 @@ def test_largest_image_goes_to_the_general_kernel(parity):
     # N = 8192, the plan's limit, with more than 4092 pruned tokens: wider than the wide-tile kernel takes
     w = synth.ragged([8192], d=64, dtype=torch.float32, params=dict(r_fixed=0.55, iters=8))
     rep = parity.check_workload(w)
-    assert rep["launches"] == 7      # stage1, scores, sinkhorn_cluster, sinkhorn_wide, sinkhorn_tall (leaves it), sinkhorn, merge
+    assert rep["launches"] == 6      # stage1, scores, sinkhorn_wide, sinkhorn_tall (leaves it), sinkhorn, merge
 
 
 def test_wide_tile_runs_reproduce_bit_for_bit(parity, binding):
