@@ -394,12 +394,14 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 }
                 return ok;
             };
-            // (larger clusters only while the grid still fits the chip at once, two at least: on a ragged
-            // batch of 128 images of up to 1156 tokens, clusters of 8 that hold every K in shared memory
-            // take seven waves and 287 us, clusters of 2 with the large tiles' K in the workspace 201 us)
-            while (fast_c < 8 && !all_tiles(fast_c, true) &&
-                   (fast_c < 2 || (long long)batch * fast_c * 2 <= plan->sm_count))
+            // Larger clusters so that every K stays in shared memory only while the grid still fits the chip
+            // at once.  Beyond that the tiles that do not fit iterate on K in the workspace: with 2 CTAs per
+            // image when they are far larger than one CTA's shared memory (128 ragged images of up to 1156
+            // tokens: clusters of 8 take seven waves and 287 us, clusters of 2 take 199 us, single CTAs 311 us),
+            // with 1 when only the very largest exceed it (1024 images of 400 tokens: 272 us against 379 us).
+            while (fast_c < 8 && !all_tiles(fast_c, true) && (long long)batch * fast_c * 2 <= plan->sm_count)
                 fast_c *= 2;
+            if (fast_c < 2 && !all_tiles(2, true)) fast_c = 2;
             all_fast = all_tiles(fast_c, false);
             // tiles wider than 256 columns, or too tall for the cluster's shared memory, are possible
             const bool wide = maxB > 256 || !all_tiles(fast_c, true);
