@@ -34,8 +34,8 @@ ROTATE = 4                 # input/output buffer sets cycled so that no step fin
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
 REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
-NCU_TRAFFIC_BYTES = {"stage1": 65871872, "gather": 10354432, "scores": 86418944,
-                     "sinkhorn_cluster": 4841984, "merge": 118960640, "density_tile": 318402048}
+NCU_TRAFFIC_BYTES = {"stage1": 66109952, "gather": 10354432, "scores": 85585408,
+                     "sinkhorn_cluster": 4840960, "merge": 119804416, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
