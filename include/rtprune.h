@@ -163,7 +163,8 @@ rtprune_status_t rtprune_workspace_init(rtprune_plan_t *plan, void *cuda_stream,
 /*
  * Stage 1 alone (Eq. 1, Eq. 8, Eq. 10, top-M selection): fills counts, out_offsets, stats[0..4]
  * and, in the workspace, the per-image selection the later stages use.  norms_out (DEVICE float
- * [total_tokens], may be NULL) receives C_k; order_out (DEVICE int32 [total_tokens], may be NULL)
+ * [total_tokens], may be NULL) receives the criterion C_k the run ranks by (the l2 norms unless
+ * params->criterion says otherwise); order_out (DEVICE int32 [total_tokens], may be NULL)
  * receives, for image i at offsets[i], its kept indices (ascending) followed by its pruned indices
  * (ascending).  Same argument rules as rtprune_run.
  */
