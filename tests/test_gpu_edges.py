@@ -274,18 +274,22 @@ def test_runs_back_to_back_on_one_plan_leave_no_state(parity, binding):
         parity.check_workload(w)
 
 
-@pytest.mark.parametrize("name,batch,bursts", [("base", 32, 40), ("large", 64, 12)])
+@pytest.mark.parametrize("name,batch,bursts", [("base", 32, 40), ("large", 64, 12), ("gundam", 24, 8),
+                                               ("sweep", 160, 6)])
 def test_many_runs_in_bursts_reproduce_bit_for_bit(binding, name, batch, bursts):
     # The kernels of a run hand images to one another through counters and lists in the workspace while
     # later kernels of the run (programmatic dependents) may already be resident.  Bursts of runs
     # without a synchronisation, on inputs that alternate, must each reproduce the first result of
     # their input bit for bit: a kernel that reads a counter left by the run before shows up here (the
-    # small batch leaves SMs free for dependents to become resident early).
+    # small batch leaves SMs free for dependents to become resident early).  The ragged batch and the batch
+    # of 160 images take the cluster kernel's instance for wide tiles, which then also feeds the merge
+    # kernel image by image (clusters of 4 and single CTAs, the largest tiles iterating in the workspace).
     dev = torch.device("cuda", 0)
     sets = [synth.make(name, seed_offset=s, batch=batch) for s in range(3)]
     w0 = sets[0]
     fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
-    plan = binding.Plan(w0.d, w0.X.dtype, batch, max(s.total_tokens for s in sets), w0.max_tokens, device=dev)
+    plan = binding.Plan(w0.d, w0.X.dtype, batch, max(s.total_tokens for s in sets),
+                        max(s.max_tokens for s in sets), device=dev)
     keys = ("out_offsets", "counts", "kept_idx", "Y", "merged_idx", "merge_partner", "merge_weight")
     try:
         ins, ref = [], []
