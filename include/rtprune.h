@@ -87,7 +87,9 @@ typedef struct {
                              of the scaling form all within one unit in the last place of their
                              previous values (bit-identical log-domain duals in the LOG form) -- later
                              iterations could only move them within rounding, so the result is that
-                             of all `iters` iterations to fp32 accuracy.  0: always run `iters`.     */
+                             of all `iters` iterations to fp32 accuracy.  (Images with more than 640
+                             pruned tokens: within four units, the rounding noise of their long sums.)
+                             0: always run `iters`.                                                  */
     float tol;            /* > 0: also stop once no dual moved by more than tol (log units) in an
                              iteration.  0 (default): never stop on a tolerance.                    */
     int32_t criterion;    /* rtprune_criterion_t: what stage 1 ranks by (default L2NORM, Eq. 1)     */

@@ -41,6 +41,7 @@ struct rtprune_plan_s {
     cudaEvent_t ev[RTPRUNE_PROFILE_MAX + 1];
     const char *ev_name[RTPRUNE_PROFILE_MAX];
     int ev_count;  // kernels recorded by the most recent run
+    int tall_c16_clusters;  // clusters of 16 CTAs of the wide-tile Sinkhorn kernel the device runs at once (0: none)
     int run;       // number of the most recent run's second stage, unique in the process: what the kernels
                    // that share counters through the workspace wait for before they read them
 };
@@ -441,8 +442,10 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             if (!c.ok(cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)tall_smem)))
                 return RTPRUNE_ERR_CUDA;
-            if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * kTallC)), dim3(kTallThreads),
-                                 tall_smem, st, (unsigned)kTallC, offsets, o.counts, o.out_offsets, order, kmat,
+            // 16 CTAs per image when all the images' clusters then still run at once, else 8
+            const int tall_c = (batch <= plan->tall_c16_clusters) ? kTallCMax : kTallC;
+            if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * tall_c)), dim3(kTallThreads),
+                                 tall_smem, st, (unsigned)tall_c, offsets, o.counts, o.out_offsets, order, kmat,
                                  L.kmat_stride, maxN, total, op, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
                                  o.merge_weight, o.stats, fast_c, fast_floats, (int)(tall_smem / sizeof(float)),
                                  (WsHeader *)(ws + L.header))))
@@ -658,6 +661,32 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
             delete p;
             return RTPRUNE_ERR_CUDA;
         }
+    }
+    // Clusters of 16 CTAs (beyond the portable size) for the wide-tile Sinkhorn kernel: ask the device how
+    // many it can run at once; a run uses them only if all its images fit that number.
+    p->tall_c16_clusters = 0;
+    {
+        const int tall_smem = std::max(p->smem_optin - 1024, 0);
+        if (cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tall_smem) ==
+                cudaSuccess &&
+            cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(kTallCMax);
+            cfg.blockDim = dim3(kTallThreads);
+            cfg.dynamicSmemBytes = (size_t)tall_smem;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = kTallCMax;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, sinkhorn_tall_kernel, &cfg) == cudaSuccess && nclusters > 0)
+                p->tall_c16_clusters = nclusters;
+        }
+        (void)cudaGetLastError();
     }
     *workspace_bytes = p->ws.total;
     *plan_out = p;

@@ -1,7 +1,7 @@
 // Dustbin-augmented optimal transport by Sinkhorn iterations (Eq. 5, Appendix C) in scaling form for
 // score tiles too wide for the kernels of sinkhorn_cluster.cuh: images with many tokens (thousands
 // per image, as the OCR models with large visual token sets produce), up to 4092 pruned tokens.  One
-// cluster of 8 CTAs per image; the tile's rows (kept tokens) are split over the CTAs; K =
+// cluster of 8 CTAs per image (16 when the batch is small enough to leave SMs idle otherwise); the tile's rows (kept tokens) are split over the CTAs; K =
 // exp((S - c)/eps) is built in place in the image's workspace tile and read once per iteration
 // through L2: a CTA's rows are contiguous there, so one thread streams them block by block into a ring
 // of shared-memory stages with 1-D bulk copies, a few blocks ahead of the threads (the tile does not
@@ -24,16 +24,23 @@
 namespace rtp {
 
 constexpr int kTallC = 8;             // CTAs per image
+constexpr int kTallCMax = 16;         // with few images and a device that schedules such clusters: 16
 constexpr int kTallThreads = 512;
 constexpr int kTallMaxB = 4092;       // row pitch (B + 4) & ~3 <= 4096 floats = 512 threads x 2 chunks
+// The fixed-point test of this kernel: a dual here is the reciprocal of a sum of a thousand or more
+// products, whose rounding noise is a few units in the last place, so "the iteration reproduces its
+// input" is tested within four units (4 x 2^-23 relative).  With the one-unit test of the smaller tiles,
+// images of 4512 tokens spent up to 81 iterations on noise of one or two units after reaching this level
+// in 6; against all 100 iterations the plan then differs by 5.5e-7 relative at most.
+constexpr float kTallFixedPointTol = 4.76837158e-7f;
 
 // Dynamic shared memory (floats) of sinkhorn_tall_kernel for tiles of at most maxB columns and maxM rows.
-__host__ __device__ inline size_t sinkhorn_tall_smem_floats(int maxB, int maxM)
+__host__ __device__ inline size_t sinkhorn_tall_smem_floats(int maxB, int maxM, int C = kTallC)
 {
     const size_t qpr = (size_t)score_pitch(maxB) / 4;
-    const size_t sl = (qpr + kTallC - 1) / kTallC;
-    const size_t rows_cap = ((size_t)maxM + kTallC - 1) / kTallC;
-    return (4 * qpr + 4) + 2 * kTallC * 4 * sl + 2048 + 256 + 64 + 48 + 2 * (rows_cap + 4) + 4;
+    const size_t sl = (qpr + C - 1) / C;
+    const size_t rows_cap = ((size_t)maxM + C - 1) / C;
+    return (4 * qpr + 4) + 2 * C * 4 * sl + 2048 + 256 + 64 + 64 + 2 * (rows_cap + 4) + 4;
 }
 constexpr int kTallMaxStages = 4;
 constexpr int kTallStageFloatsMax = 16384;      // a block of rows is at most 64 KB (see the three layouts)
@@ -90,7 +97,7 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
                                            int32_t *__restrict__ partner_seg, float *__restrict__ weight_seg,
                                            float *__restrict__ stats_img)
 {
-    constexpr int C = kTallC;
+    const int C = (int)ptx::cluster_nctarank();      // 8 or 16
     constexpr int G = kTallThreads / W;
     constexpr int WPG = W / 32;
     constexpr int kWarps = kTallThreads / 32;
@@ -107,7 +114,7 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
     float *red = cpart + 2048;                // [2][16][8]     per-warp row-sum partials, double-buffered by block
     float *wred = red + 256;                  // [2][16] + [2]  per-warp sums of V and moves; the groups' sums of U
     float *xs = wred + 64;                    // [4][C]         per-CTA sums of U, sums of V, continue flags, moves
-    float *us = xs + 48;                      // [rows_cap + 4] U of this CTA's rows
+    float *us = xs + 64;                      // [rows_cap + 4] U of this CTA's rows
     int *toks = reinterpret_cast<int *>(us + rows_cap + 4);   // [rows_cap] token position of this CTA's rows
     const int fixed_floats = (int)((us + rows_cap + 4 + rows_cap) - sm + 3) & ~3;
     float *ring = sm + fixed_floats;          // [NS][G R ldS]  blocks of rows of K on their way to the threads
@@ -347,21 +354,18 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
 
         // ---- this CTA's slice of V from the completed column sums, broadcast to the cluster -----------
         float su_all = 0.f;
-#pragma unroll
         for (int r = 0; r < C; ++r) su_all += xs[r];          // read here: the next pass may overwrite it early
         int cont = 0;
         float move = 0.f, nv = 0.f;
         const int j = (int)rank * slc + tid;
         if (tid < slc && j < B) {
             float cs = 0.f;
-#pragma unroll
             for (int r = 0; r < C; ++r) cs += xrecv[r * slc + tid];
             nv = rcp_fast(cs + kappa * Ud);
             const float ov = vs[j];
             move = fabsf(nv - ov) * rcp_fast(ov);
-            cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
+            cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? (move > kTallFixedPointTol) : 1);
             const uint32_t a = vs_u32 + (uint32_t)j * 4u;
-#pragma unroll
             for (uint32_t r = 0; r < (uint32_t)C; ++r) ptx::st_cluster_f32(ptx::map_to_rank(a, r), nv);
         }
         const float wv = warp_sum(nv), wm = warp_max(move);
@@ -388,9 +392,8 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
         // every thread of every CTA: the sums, the dustbin column, the decision to go on
         const float nVd = Mf * rcp_fast(kappa * (su_all + Ud));
         const float md = fabsf(nVd - Vd) * rcp_fast(Vd);
-        bool go = p.tol > 0.f ? (md > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : true);
+        bool go = p.tol > 0.f ? (md > p.tol) : (p.stop_fp ? (md > kTallFixedPointTol) : true);
         float sv_all = 0.f, mv_all = md;
-#pragma unroll
         for (int r = 0; r < C; ++r) {
             sv_all += xs[C + r];
             go = go || (xs[2 * C + r] != 0.f);
@@ -516,7 +519,6 @@ __device__ inline void sinkhorn_tall_solve(float *Kg, int ldS, int M, int B, int
             const int *xi = reinterpret_cast<const int *>(xrecv + C * slc);
             float b = xrecv[tid];
             int ib = xi[tid];
-#pragma unroll
             for (int r = 1; r < C; ++r) {      // ranks hold ascending row ranges: strict > keeps the lower index
                 const float ob = xrecv[r * slc + tid];
                 if (ob > b) {
@@ -546,7 +548,8 @@ sinkhorn_tall_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     extern __shared__ __align__(16) float sm[];
     __shared__ uint64_t s_full[kTallMaxStages];
     const uint32_t rank = ptx::cluster_ctarank();
-    const int img = blockIdx.x / kTallC;
+    const int nC = (int)ptx::cluster_nctarank();
+    const int img = blockIdx.x / nC;
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();         // scores, counts and order come from the kernels ahead
     int t_begin, N;
@@ -554,7 +557,7 @@ sinkhorn_tall_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     const int M = __ldcg(counts + img), B = N - M;
     if (B == 0 || B > kTallMaxB) return;
     if (fast_c > 0 && sinkhorn_cluster_handles(M, B, fast_c, fast_floats)) return;   // solved ahead of this kernel
-    const int rows_per = (M + kTallC - 1) / kTallC;
+    const int rows_per = (M + nC - 1) / nC;
     const int row_lo = min(M, (int)rank * rows_per);
     const int Ml = min(M, row_lo + rows_per) - row_lo;       // this CTA's rows (may be 0)
     const int ldS = score_pitch(B);
