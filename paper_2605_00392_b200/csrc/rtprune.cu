@@ -443,6 +443,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                            (int)tall_smem)))
                 return RTPRUNE_ERR_CUDA;
             // 16 CTAs per image when all the images' clusters then still run at once, else 8
+            // (never fewer than 8: a CTA owns a slice of at most 512 columns, one per thread)
             const int tall_c = (batch <= plan->tall_c16_clusters) ? kTallCMax : kTallC;
             if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * tall_c)), dim3(kTallThreads),
                                  tall_smem, st, (unsigned)tall_c, offsets, o.counts, o.out_offsets, order, kmat,
