@@ -443,8 +443,14 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                            (int)tall_smem)))
                 return RTPRUNE_ERR_CUDA;
             // 16 CTAs per image when all the images' clusters then still run at once, else 8
-            // (never fewer than 8: a CTA owns a slice of at most 512 columns, one per thread)
-            const int tall_c = (batch <= plan->tall_c16_clusters) ? kTallCMax : kTallC;
+            // (a CTA owns a slice of at most 512 columns, one per thread: 8 CTAs cover every pitch, 4 cover
+            // pitches of up to 2048 floats).  Batches whose clusters of 8 need several waves get clusters of 4
+            // when their tiles are narrow (pitch <= 1024 floats): 64 images of 2137 tokens 0.63 -> 0.54 ms in
+            // this kernel; wider tiles lose (32 images of 4512 tokens: 1.6 -> 4.2 ms, too many tiles in flight
+            // for L2).
+            int tall_c = (batch <= plan->tall_c16_clusters) ? kTallCMax : kTallC;
+            if ((long long)batch * kTallC > plan->sm_count && score_pitch(std::min(maxB, kTallMaxB)) <= 1024)
+                tall_c = 4;
             if (!c.ok(launch_pdl(sinkhorn_tall_kernel, dim3((unsigned)(batch * tall_c)), dim3(kTallThreads),
                                  tall_smem, st, (unsigned)tall_c, offsets, o.counts, o.out_offsets, order, kmat,
                                  L.kmat_stride, maxN, total, op, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,

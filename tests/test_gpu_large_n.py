@@ -50,6 +50,14 @@ def test_two_chunks_per_thread_and_fp32_storage(parity):
     parity.check_workload(w)
 
 
+def test_many_images_with_narrow_wide_tiles_take_clusters_of_four(parity):
+    # 20 images whose clusters of 8 would not all run at once, tiles of 700 columns: clusters of 4 CTAs
+    w = synth.ragged([1400] * 20, d=64, dtype=torch.float32, params=dict(r_fixed=0.5, iters=30))
+    parity.check_workload(w)
+    w = synth.ragged([1400] * 19 + [700], params=dict(r_fixed=0.5))
+    parity.check_workload(w, images=[0, 7, 18, 19])
+
+
 def test_single_kept_row_leaves_seven_ctas_without_rows(parity):
     w = synth.ragged([1400], d=64, dtype=torch.float32, params=dict(r_fixed=0.9995, iters=25))
     rep = parity.check_workload(w)
