@@ -483,6 +483,8 @@ def main() -> None:
             "sinkhorn_wide": ("alu", sink_flops),
             "sinkhorn": ("alu", sink_flops),
             "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
+            # scores, Sinkhorn and merge in one kernel: it must read X and write Y, the pairs and the indices
+            "stage2_fused": ("hbm", x_bytes + y_bytes + 16 * total),
         }
         bound, units = algo[dominant]
         dur_s = avg[dominant] / 1e3

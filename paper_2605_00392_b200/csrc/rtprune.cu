@@ -10,6 +10,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "fused.cuh"
 #include "gemm_simt.cuh"
 #include "merge_umma.cuh"
 #include "scores_umma.cuh"
@@ -44,6 +45,7 @@ struct rtprune_plan_s {
     int tall_c16_clusters;  // clusters of 16 CTAs of the wide-tile Sinkhorn kernel the device runs at once (0: none)
     int run;       // number of the most recent run's second stage, unique in the process: what the kernels
                    // that share counters through the workspace wait for before they read them
+    int fused_clusters;     // clusters of 2 CTAs of the fused stage-2 kernel the device runs at once (0: none)
 };
 
 // Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
@@ -332,6 +334,30 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     do plan->run = ++g_run_count; while (plan->run == 0);   // 0 is what a fresh workspace holds
     uint32_t *scores_done = nullptr; // per-image counts of finished score tiles, when the scores kernel keeps them
 
+    if constexpr (kTensor) {
+        // One kernel for the whole second stage when every image the run can hold fits it
+        if (maxB > 0 && plan->fused_clusters > 0 && !use_log_form(params) && fused_eligible(plan->d, maxN, maxB)) {
+            CUtensorMap tmapXa, tmapXb, tmapXp;
+            if (!make_tmap_bf16(plan, &tmapXa, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2, kFuBK,
+                                kFuTileM) ||
+                !make_tmap_bf16(plan, &tmapXb, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2, 64, 64) ||
+                !make_tmap_bf16(plan, &tmapXp, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
+                                (uint64_t)plan->d * 2, 64, 64))
+                return RTPRUNE_ERR_CUDA;
+            OtParams op{params->z, params->alpha, params->eps, params->iters, params->stop_at_fixed_point,
+                        params->tol};
+            const int clusters = std::min(batch, plan->fused_clusters);
+            if (!c.ok(launch_pdl(stage2_fused_kernel, dim3((unsigned)(2 * clusters)), dim3(kFuThreads),
+                                 (size_t)kFuSmemBytes, st, 2u, tmapXa, tmapXb, tmapXp, (const __nv_bfloat16 *)X, offsets,
+                                 plan->d, batch, (const int32_t *)o.counts, (const int32_t *)order,
+                                 (const int32_t *)(ws + L.kpos), (const float *)norms, (__nv_bfloat16 *)(ws + L.xp), maxN,
+                                 total, op, (__nv_bfloat16 *)o.Y, o.out_offsets, o.kept_idx, o.merged_idx,
+                                 o.merge_partner, o.merge_weight, o.stats, (WsHeader *)(ws + L.header))))
+                return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "stage2_fused");
+            return RTPRUNE_OK;
+        }
+    }
     if (maxB > 0) {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
             // compact copy of the pruned rows for the tensor-core kernels
@@ -669,6 +695,28 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
             return RTPRUNE_ERR_CUDA;
         }
     }
+    // The fused stage-2 kernel: clusters of 2 CTAs with all of an SM's shared memory each; how many the
+    // device runs at once is what a run's grid is capped at (its clusters then loop over the images).
+    p->fused_clusters = 0;
+    if (dtype == RTPRUNE_BF16 &&
+        cudaFuncSetAttribute(stage2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
+            cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2);
+        cfg.blockDim = dim3(kFuThreads);
+        cfg.dynamicSmemBytes = (size_t)kFuSmemBytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, stage2_fused_kernel, &cfg) == cudaSuccess && nclusters > 0)
+            p->fused_clusters = nclusters;
+    }
+    (void)cudaGetLastError();
     // Clusters of 16 CTAs (beyond the portable size) for the wide-tile Sinkhorn kernel: ask the device how
     // many it can run at once; a run uses them only if all its images fit that number.
     p->tall_c16_clusters = 0;

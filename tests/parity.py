@@ -7,8 +7,13 @@ Tolerances (stated once, used by every parity test):
     PARTNER_GAP (1e-3); below that several answers are correct to working precision (near-duplicate
     background tokens make most columns of the document batches such near-ties), so in addition
     EVERY chosen partner must reach the oracle's column maximum of log P to within PARTNER_REGRET.
-  * merged features Y: |y - y*| <= tol * max(|y*|, rms(y* row)) with tol = 1e-2 for bf16 storage
-    (fp32 accumulation) and 1e-5 for fp32 storage; y* is the oracle's fp64 value.
+  * merged features Y: |y - y*| <= tol * max(|y*|, rms(y* row)) with tol = 6.5e-3 for bf16 storage
+    (fp32 accumulation; the output's rounding to bf16 is at most 2^-8 = 3.9e-3 and the plan's, whose entries
+    enter the tensor cores in bf16, at most 2^-9 = 2.0e-3 of the merge term; inside the 1e-2 the method's statement allows) and 1e-5
+    for fp32 storage; y* is the oracle's fp64 value.
+  * the merge term of Eq. 7 on its own (see compare_image): its gain against a reference that carries the
+    tensor-core merge's documented operand precision, and, in bf16 storage, the share of elements that
+    differ from that reference at all.
   * phi: 2e-5 absolute (fp32 sum of ~N unit vectors); r: 1e-5; plan weights: 1e-4 relative.
 Inputs have sorted-norm gaps >= 1.2e-3 (generator) and, for dynamic ratios, |frac(r N) - 1/2| >= 1e-3
 (enforced here by nudging rho, an input), so every integer decision is the same in fp32 and fp64.
@@ -16,6 +21,7 @@ Inputs have sorted-norm gaps >= 1.2e-3 (generator) and, for dynamic ratios, |fra
 from __future__ import annotations
 
 import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass
 from typing import Dict, List, Optional, Sequence
 
@@ -27,8 +33,12 @@ from paper_2605_00392_b200 import binding, synth
 
 PARTNER_GAP = 1e-3
 PARTNER_REGRET = 5e-5      # every chosen partner's log P must be this close to the column maximum
-FEATURE_TOL = {torch.bfloat16: 1e-2, torch.float32: 1e-5}
+FEATURE_TOL = {torch.bfloat16: 6.5e-3, torch.float32: 1e-5}
+MERGE_GAIN_TOL = {torch.float32: 1e-4}        # per image
+MERGE_ROW_GAIN_TOL = {torch.float32: 1e-3}    # per row with a visible term
+BF16_MODEL_MISMATCH = 0.01      # share of a bf16 image's elements that may differ from the reference
 ROUND_MARGIN = 1e-3
+ORACLE_CHUNK = 64          # images per oracle call: bounds the fp64 copies held at once
 
 
 def oracle_params(p: Dict[str, float]) -> oracle.Params:
@@ -52,13 +62,15 @@ def settle_rho(w: synth.Workload, images: Sequence[int]) -> None:
     if not w.params["dynamic"]:
         return
     p = oracle_params(w.params)
-    for i in images:
-        T = w.image_f64(i)
-        ph = oracle.phi(T)
+    images = list(images)
+    with ThreadPoolExecutor(max_workers=cpu_threads()) as ex:      # the C loops release the GIL
+        phis = list(ex.map(lambda i: oracle.phi(w.image_f64(i)), images))
+    for i, ph in zip(images, phis):
+        n_i = int(w.offsets[i + 1] - w.offsets[i])
         for _ in range(50):
-            r, _, _ = oracle.ratio(ph, float(w.rho[i]), T.shape[0], dynamic=True, phi_lo=p.phi_lo,
+            r, _, _ = oracle.ratio(ph, float(w.rho[i]), n_i, dynamic=True, phi_lo=p.phi_lo,
                                    phi_hi=p.phi_hi, r_max=p.r_max)
-            frac = r * T.shape[0] - np.floor(r * T.shape[0])
+            frac = r * n_i - np.floor(r * n_i)
             if abs(frac - 0.5) >= ROUND_MARGIN or r in (0.0, p.r_max):
                 break
             w.rho[i] = np.float32(min(1.0, float(w.rho[i]) + 0.003))
@@ -137,6 +149,54 @@ def compare_image(w: synth.Workload, i: int, ref: oracle.ImageResult, g: binding
         assert torch.equal(g.Y[o0:o1], w.X[int(w.offsets[i]):int(w.offsets[i + 1])]), tag
         return
 
+    # the merge term alone (Eq. 7): how much of alpha P T_p the output carries.  With alpha = 0.1 the term
+    # is a few percent of a row (a fraction of a bf16 ulp of it), so the feature tolerance alone would let
+    # a third of it go missing.  Reference: the oracle's fp64 result in fp32 storage; in bf16 storage the
+    # fp64 product T_k + bf16(alpha P*) T_p of the oracle's plan P*, rounded once to bf16 -- the operand
+    # precision the tensor-core merge documents (the plan's own rounding, up to 2^-9 per entry and alike
+    # for the near-duplicate tokens of a page, shifts a term of a third of an ulp by more than any
+    # tolerance that would still catch a missing k-block).  Against that reference:
+    #   * fp32 storage: the gain <Y - T_k, t*> / <reference - T_k, t*> over the exact term t* is 1 within
+    #     MERGE_GAIN_TOL per image and MERGE_ROW_GAIN_TOL per row whose term stands clear of rounding;
+    #   * bf16 storage: at most BF16_MODEL_MISMATCH of an image's elements differ from the reference at all
+    #     (fp32 accumulation leaves the device within ~1e-6 of it: only values next to a rounding boundary
+    #     round the other way; a missing k-block of the plan shifts every element by a tenth of an ulp and
+    #     flips a tenth of them).  The gain is reported, not asserted: it moves only through those flips.
+    alpha = float(np.float32(w.params["alpha"]))
+    if alpha != 0.0:
+        a0 = int(w.offsets[i])
+        Xi = w.X[a0:a0 + N].to(torch.float64).numpy()
+        xk = Xi[ref.kept]
+        term = ystar - xk                               # alpha P T_p, exact
+        if w.X.dtype == torch.bfloat16 and ref.Pbar is not None:
+            aP = torch.from_numpy(np.float32(alpha) * ref.Pbar[:-1, :-1].astype(np.float32)).to(torch.bfloat16)
+            model = xk + aP.to(torch.float64).numpy() @ Xi[ref.prop]
+        else:
+            model = ystar
+        want = torch.from_numpy(model).to(w.X.dtype).to(torch.float64).numpy() - xk
+        got = y - xk
+        den = float((want * term).sum())
+        if den > 0.0:
+            gain = float((got * term).sum()) / den
+            report["max_merge_gain_err"] = max(report.get("max_merge_gain_err", 0.0), abs(gain - 1.0))
+            exact_store = w.X.dtype != torch.bfloat16   # bf16: got and want differ only where an element rounds the
+            if exact_store:                             # other way, which the mismatch share below bounds directly
+                assert abs(gain - 1.0) <= MERGE_GAIN_TOL[w.X.dtype], (tag, "merge-term gain", gain)
+            trow = np.sqrt((term * term).mean(axis=1))
+            yrow = np.sqrt((ystar * ystar).mean(axis=1))
+            unit = 2.0 ** -9 if w.X.dtype == torch.bfloat16 else 2.0 ** -24
+            clear = trow >= 8.0 * unit * yrow
+            if clear.any():
+                rg = (got[clear] * term[clear]).sum(axis=1) / (want[clear] * term[clear]).sum(axis=1)
+                worst_row = float(np.abs(rg - 1.0).max())
+                report["max_merge_row_gain_err"] = max(report.get("max_merge_row_gain_err", 0.0), worst_row)
+                if exact_store:
+                    assert worst_row <= MERGE_ROW_GAIN_TOL[w.X.dtype], (tag, "merge-term row gain", worst_row)
+        if w.X.dtype == torch.bfloat16:
+            differ = float((got != want).mean())
+            report["max_rounding_mismatch"] = max(report.get("max_rounding_mismatch", 0.0), differ)
+            assert differ <= BF16_MODEL_MISMATCH, (tag, "merge-term rounding mismatch", differ)
+
     # pairs
     gp = g.merge_partner[seg:seg + ref.B].numpy()
     gw = g.merge_weight[seg:seg + ref.B].numpy().astype(np.float64)
@@ -182,14 +242,25 @@ def check_workload(w: synth.Workload, *, images: Optional[Sequence[int]] = None,
         assert np.all(np.diff(k) > 0) and np.all(np.diff(m) > 0)
         both = np.concatenate([k, m])
         assert len(both) == lens[i] and np.array_equal(np.sort(both), np.arange(lens[i]))
-    refs = oracle.run_batch(w.X_f64() if images is None else _SparseX(w), w.offsets,
-                            oracle_params(w.params), w.rho, images=imgs, threads=cpu_threads(),
-                            want_plan=True)
-    report: Dict[str, float] = {"launches": res.launches}
-    for i, ref in zip(imgs, refs.images):
-        compare_image(w, i, ref, g, report)
+    report: Dict[str, float] = {"launches": res.launches, "images_compared": len(imgs)}
+    X = _SparseX(w)
+    for c0 in range(0, len(imgs), ORACLE_CHUNK):       # a chunk at a time: the oracle's fp64 results are large
+        part = imgs[c0:c0 + ORACLE_CHUNK]
+        refs = oracle.run_batch(X, w.offsets, oracle_params(w.params), w.rho, images=part,
+                                threads=cpu_threads(), want_plan=True)
+        for i, ref in zip(part, refs.images):
+            compare_image(w, i, ref, g, report)
     report["mean_retention"] = float(counts.sum()) / float(lens.sum())
     report["mean_iters"] = float(g.stats[:w.batch, 5].mean())
+    pairs = report.get("pairs", 0)
+    # share of the pairs held to bit-exactness (oracle's top-2 gap >= PARTNER_GAP); the rest were held to
+    # the regret bound only
+    report["bit_exact_pair_share"] = 1.0 - report.get("pairs_within_gap", 0) / pairs if pairs else 1.0
+    print("parity %s: %d images compared, %d pairs, bit-exact share %.4f, max regret %.2e, max feature err %.2e, "
+          "merge gain err %.2e (row %.2e)" % (w.name, len(imgs), pairs, report["bit_exact_pair_share"],
+                                              report.get("max_partner_regret", 0.0), report.get("max_feature_err", 0.0),
+                                              report.get("max_merge_gain_err", 0.0),
+                                              report.get("max_merge_row_gain_err", 0.0)))
     return report
 
 
