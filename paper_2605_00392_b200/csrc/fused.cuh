@@ -1,77 +1,97 @@
 // Stage 2 of Algorithm 1 in ONE kernel, one cluster of two CTAs per image: cosine scores (Section
 // 3.3.2) on the tcgen05 tensor cores, dustbin augmentation and Sinkhorn iterations (Eq. 5, Appendix C)
 // with the kernel matrix K held in REGISTERS, and the merge T_k + alpha P T_p (Eq. 7) on the tensor
-// cores again, written packed.  Nothing but the compact copy of the pruned rows goes through global
-// memory between the steps: S lives in tensor memory, K in registers, the plan P in shared memory.
+// cores again, written packed.  Nothing goes through global memory between the steps: S lives in
+// tensor memory, K in registers, the plan P in shared memory.
 //
 // Taken by runs whose images all have at most kFuMaxTok tokens and at most kFuMaxB pruned tokens, bf16
 // storage, width a multiple of 64, scaling form (fused_eligible() on the host); everything else keeps
 // the separate kernels.
 //
-// Work split inside a cluster (rank r = 0, 1):
-//   * tokens: rank r owns the image's tokens [r * tpc, min(N, (r + 1) * tpc)), tpc = ceil(N / 2): at most
-//     two tiles of 128 CONSECUTIVE tokens, fetched by tiled TMA (kept and pruned alike; rows of pruned
-//     tokens are computed and dropped, as contiguous rows are what TMA moves at full speed: a
-//     tile::gather4 load moves 512 bytes in about 70 cycles, a tiled load 16 KB in about 400).
-//   * pruned rows: the cluster first copies the image's B pruned rows to a compact scratch in global
-//     memory (they are L2 hits: stage 1 has just read them), so that both contractions can fetch them
-//     as tiles too.
-//   * kept rows of the Sinkhorn problem: rank r owns kept positions [r * half, ...), half = ceil(M / 2),
-//     whatever tokens they are; the scores epilogue sends K = exp((S - c) / eps) of a row to its owner
-//     through distributed shared memory, and the owner sends the row of alpha P back to the owner of the
-//     token when the iterations are done.
+// Work split inside a cluster (rank r = 0, 1): rank r owns the kept positions [r * half, ...) of the
+// image, half = ceil(M / 2): its rows of S, K, P and of the output Y.  Both CTAs need all B pruned rows.
+//
+// Operand fetch: kept and pruned rows are scattered over the image, so the operand tiles are gathered
+// by eleven producer warps with 16-byte cp.async copies straight into the 128-byte-swizzled layout
+// the UMMA descriptors expect, k-block by k-block, several k-blocks in flight.  Measured on a B200, per
+// SM, on rows that sit in L2: 16-byte loads through the load/store path 70 B/clk, tiled TMA boxes of
+// 128-byte rows 31 B/clk, tile::gather4 7 B/clk; so the gather is faster than a tiled copy of a compact
+// copy would be, and moves only the rows that are needed.
+//
 // Sinkhorn iteration: as in sinkhorn_cluster.cuh (one pass per iteration, LR lanes share a row, column
 // sums completed over the warps in shared memory and over the two CTAs through distributed shared
-// memory, one cluster barrier), but a thread's K values never leave its registers.
-// Merge: for each tile of 64 output columns, D = [I | alpha P] . [T_v rows of the token tile ; T_p]
-// (the identity block carries the kept token's own row through the tensor cores, exact in the fp32
+// memory), but a thread's K values never leave its registers.
+// Merge: for each tile of 64 output columns, D = [I | alpha P] . [T_k rows of the tile ; T_p] (the
+// identity block carries the kept token's own row through the tensor cores, exact in the fp32
 // accumulator); four accumulator stages in tensor memory; the epilogue converts to bf16, stages a
-// warp's 32 rows in shared memory and writes the kept ones with coalesced 16-byte stores.
+// warp's 32 rows in shared memory and writes them with coalesced 16-byte stores (the rows of a CTA are
+// consecutive rows of Y).
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
 #include "sinkhorn.cuh"
 #include "sinkhorn_cluster.cuh"
+#include "stage1.cuh"
 
 namespace rtp {
 
 constexpr int kFuThreads = 512;
 constexpr int kFuWarps = kFuThreads / 32;
-constexpr int kFuMaxTok = 512;            // tokens per image: two tiles of 128 per CTA
+// Warp roles.  Scores: warp 0 lane 0 issues the UMMAs, warps 1-15 gather the operands.  Merge: warps 0-7 are
+// the epilogue (TMEM lane quarter warp % 4 of row tile warp / 4), warp 8 lane 0 issues the UMMAs, warps
+// 9-15 gather the operands.
+constexpr int kFuScProducers = (kFuWarps - 1) * 32;
+constexpr int kFuEpiWarps = 8;
+constexpr int kFuMmaWarp = 8;
+constexpr int kFuMgProducers = (kFuWarps - kFuMmaWarp - 1) * 32;
+constexpr int kFuStageRowsMax = 448;      // rows of a stage (kept rows of the CTA + pruned rows, each rounded up to 16)
+constexpr int kFuScChunks = (8 * kFuStageRowsMax + kFuScProducers - 1) / kFuScProducers;   // copies per producer thread and stage
+constexpr int kFuMgChunks = (8 * kFuStageRowsMax + kFuMgProducers - 1) / kFuMgProducers;
+constexpr int kFuMaxTok = 512;            // tokens per image
 constexpr int kFuMaxB = 256;              // pruned tokens per image: one UMMA N, half of tensor memory
+constexpr int kFuMaxRows = 256;           // kept rows per CTA: two tiles of 128
 constexpr int kFuKRegs = 64;              // K values a thread may hold
 constexpr int kFuTileM = 128;
 constexpr int kFuBK = 64;                 // bf16 per k-block = one 128-byte swizzle row
 constexpr int kFuNT = 64;                 // output columns per merge tile
 constexpr int kFuABytes = kFuTileM * 128; // 16 KB: 128 rows x 64 bf16, K-major
 constexpr int kFuBoxBytes = 64 * 128;     // 8 KB: 64 rows x 64 bf16
-constexpr int kFuIdentBytes = 3 * (kFuABytes / 2);
-constexpr int kFuScStages = 4;            // at most
-constexpr int kFuMgStages = 4;            // B-operand ring of the merge
+constexpr int kFuScStages = 6;            // at most
+constexpr int kFuMgStages = 6;            // at most
 constexpr int kFuAccStages = 4;           // accumulator stages of the merge (128 TMEM columns each)
-constexpr int kFuSharedBytes = 12288;     // FuShared, rounded up
-constexpr int kFuArenaBytes = 180 * 1024;
-constexpr int kFuPartOffset = 128 * 1024; // arena offsets: P tiles at 0, column partials / merge ring here
-constexpr int kFuStagePitch = kFuNT * 2 + 16;                 // bytes per staged output row
-constexpr int kFuStagingOffset = kFuPartOffset + 32 * 1024;   // 4 warps x 32 rows x kFuStagePitch
-constexpr int kFuSmemBytes = 1024 + kFuIdentBytes + kFuSharedBytes + kFuArenaBytes;
+constexpr int kFuS1Stages = 8;            // at most, of the streaming pass
+constexpr int kFuS1Rows = kFuWarps;       // rows per stage of the streaming pass: one per warp
+constexpr int kFuS1Vpl = 8;               // 16-byte vectors of a row per lane, at most: widths up to 2048
+constexpr int kFuSharedBytes = 18432;     // FuShared, rounded up
+constexpr int kFuArenaBytes = 207 * 1024;
+constexpr int kFuPartBytes = 32 * 1024;   // column partials of the iterations, then of the pairing
+constexpr int kFuPartOffset = kFuArenaBytes - kFuPartBytes;
+constexpr int kFuSmemBytes = 1024 + kFuSharedBytes + kFuArenaBytes;
+static_assert(kFuSmemBytes <= 227 * 1024, "more shared memory than a CTA can have");
 
 struct FuShared {
     uint64_t sc_full[kFuScStages], sc_empty[kFuScStages], sc_accum;
     uint64_t mg_full[kFuMgStages], mg_empty[kFuMgStages];
     uint64_t acc_full[kFuAccStages], acc_empty[kFuAccStages];
+    uint64_t xbar[2];                           // the other CTA's column sums of an iteration have arrived (by parity)
+    uint64_t s1_full[kFuS1Stages], s1_empty[kFuS1Stages];   // ring of the streaming pass
     uint32_t tmem_base;
     volatile int abort_flag;
     int out0;
+    int sel_m;                                  // M of the image, from the thread that computes the ratio
+    float red[32];
     float vsum[kFuWarps];
     float wsum[kFuWarps];
-    float xusum[2][2];
-    __align__(16) float inv_nj[kFuMaxB];   // 1 / |x_j| of the pruned tokens
-    __align__(16) float vs[kFuMaxB + 8];   // V_j, V_d at [ldk]: read as 16-byte vectors
-    int toks[kFuMaxTok / 2 + 8];      // image-local token of each of this CTA's kept rows
-    __align__(16) float xpart[2][2][kFuMaxB];   // per-CTA column partials by iteration parity
-    float pairv[2][kFuMaxB];          // rank 0: per-CTA column maxima of K U ...
-    int pairi[2][kFuMaxB];            // ... and their rows
+    __align__(16) float xusum[2][4];            // the other CTA's sum of U, by iteration parity
+    __align__(16) float inv_nj[kFuMaxB];        // 1 / |x_j| of the pruned tokens
+    __align__(16) float inv_ni[kFuMaxRows];     // 1 / |x_i| of this CTA's kept rows
+    __align__(16) float vs[kFuMaxB + 8];        // V_j, V_d at [ldk]: read as 16-byte vectors
+    int rowtok[kFuMaxRows + kFuMaxB + 32];      // image-local token of each row of a stage (-1: a row of zeros)
+    __align__(16) float xpart[2][kFuMaxB];      // the other CTA's column partials, by iteration parity
+    __align__(16) float nrm[kFuMaxTok + 4];     // l2 norms of all the image's tokens (streaming pass in this kernel)
+    int wcount[2][kFuWarps];                    // kept / pruned tokens per warp of the selection
+    float pairv[2][kFuMaxB];                    // rank 0: per-CTA column maxima of K U ...
+    int pairi[2][kFuMaxB];                      // ... and their rows
 };
 static_assert(sizeof(FuShared) <= kFuSharedBytes, "FuShared outgrew its region");
 
@@ -86,27 +106,50 @@ __host__ __device__ inline int fused_k_regs(int rows, int B)
     return (ns < 1 ? 1 : ns) * (ldk / lr);
 }
 
-// Every image of a run with at most max_tokens tokens and max_b pruned tokens fits the fused kernel.
+// Operand arrays in shared memory are rows of 128 bytes (64 bf16), eight-row groups of 1024 bytes, the
+// 16-byte pieces of a row XOR-swizzled by the row's place in its group: what a UMMA descriptor with the
+// 128-byte swizzle addresses, as a K-major operand (rows = M or N index) or as an MN-major one (rows = k
+// index).  A stage of either ring holds this CTA's kept rows (rounded up to 16 rows, zeros past the last)
+// followed by the pruned rows (likewise); the plan is one such array of the CTA's rows per 64 columns.
+// A 128-row UMMA operand that starts at row 128 t of an array with fewer than 128 (t + 1) rows reads on
+// into whatever follows (rows nobody uses): sizes below keep those reads inside the arena.
+__host__ __device__ inline int fused_stage_bytes(int rows, int B)
+{
+    return (((rows + 15) & ~15) + ((B + 15) & ~15)) * 128;
+}
+__host__ __device__ inline int fused_plan_bytes(int rows, int B)
+{
+    return ((B + 63) / 64) * ((rows + 15) & ~15) * 128;
+}
+
+// The streaming pass of stage 1 can run inside the kernel too: rows of at most 32 * kFuS1Vpl vectors, two
+// stages of 16 rows in the arena, the warps' partial sums of unit tokens and the two CTAs' sums after them.
+__host__ inline bool fused_stage1_eligible(int d)
+{
+    return d % 8 == 0 && d / 8 <= 32 * kFuS1Vpl && 2 * kFuS1Rows * d * 2 <= kFuArenaBytes &&
+           (kFuWarps + 2) * d * 4 <= kFuArenaBytes;
+}
+
+// Every image of a run with at most max_tokens tokens and max_b pruned tokens fits the fused kernel:
+// K in 64 registers per thread, at least two stages in either ring.
 __host__ inline bool fused_eligible(int d, int max_tokens, int max_b)
 {
     if (d % 64 != 0 || max_tokens > kFuMaxTok || max_b > kFuMaxB) return false;
-    for (int b = 1; b <= max_b; ++b) {
+    for (int b = 0; b <= max_b; ++b) {
         const int m = max_tokens - b > 1 ? max_tokens - b : 1;
-        const int regs = fused_k_regs((m + 1) / 2, b);
-        if (regs == 0 || regs > kFuKRegs) return false;
+        const int rows = (m + 1) / 2;
+        if (rows > kFuMaxRows) return false;
+        if (b > 0) {
+            const int regs = fused_k_regs(rows, b);
+            if (regs == 0 || regs > kFuKRegs) return false;
+        }
+        if (fused_stage_bytes(rows, b) > kFuStageRowsMax * 128) return false;
+        if (2 * fused_stage_bytes(rows, b) + kFuABytes > kFuArenaBytes) return false;
+        if (fused_plan_bytes(rows, b) + 2 * fused_stage_bytes(rows, b) + kFuABytes > kFuArenaBytes) return false;
     }
     return true;
 }
 
-__device__ inline void st_cluster_v4(uint32_t addr, float4 v)
-{
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
-                 : "memory");
-}
-__device__ inline void st_cluster_v2_u32(uint32_t addr, uint32_t a, uint32_t b)
-{
-    asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
-}
 __device__ inline void mbar_inval(uint64_t *bar)
 {
     asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(ptx::smem_u32(bar)) : "memory");
@@ -114,10 +157,9 @@ __device__ inline void mbar_inval(uint64_t *bar)
 
 struct FuImage {
     int t_begin, N, M, B;
-    int tok_lo, ntok, ntile;      // this CTA's tokens
-    int half, row_lo, Ml;         // this CTA's kept rows of the Sinkhorn problem
-    int ldk, nkb, nbox, BN;
-    int tpc;
+    int half, row_lo, Ml, ntile;  // this CTA's kept rows
+    int ldk, nkb;
+    int Ra, Rb;                   // rows a stage holds: kept rows and pruned rows, each rounded up to 16
 };
 
 struct FuIterState {
@@ -125,14 +167,26 @@ struct FuIterState {
     float last_move;
 };
 
+// One 32-bit word into the other CTA's shared memory, counted (4 bytes) on a barrier there when it has landed.
+__device__ inline void st_async_peer(uint32_t remote_addr, uint32_t value, uint32_t remote_bar)
+{
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];" ::"r"(remote_addr), "r"(value),
+                 "r"(remote_bar)
+                 : "memory");
+}
+
 // The iterations, K in registers.  Row i of this CTA (kept position row_lo + i) lives in the LR lanes
 // (step s, warp w, slot) with i = (s * 16 + w) * (32 / LR) + slot; lane `sub` of a row holds the 16-byte
-// column chunks sub, sub + LR, ...  On return vs[] holds the final V (V_d at [ldk]) and U[] the final
-// U of the thread's rows (0 for rows past Ml).
+// column chunks sub, sub + LR, ...  Column sums: over a warp's row slots by shuffles, over the warps in
+// shared memory, over the two CTAs by sending this CTA's sums into the other's shared memory with
+// asynchronous stores that are counted on a barrier there: no cluster-wide barrier in the loop.  Both
+// CTAs add the two partial sums of a column (a + b = b + a), so they hold bit-identical V and leave the
+// loop together.  `round` counts the exchanges of the kernel (the barriers' phases run on across images).
+// On return vs[] holds the final V (V_d at [ldk]) and U[] the final U of the thread's rows.
 template <int LR, int CPL, int NS>
 __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], float (&U)[NS], FuShared *sh, float *part,
                                             int Ml, int M, int B, uint32_t rank, const OtParams &p, float kappa,
-                                            float v_init)
+                                            float v_init, uint32_t &round, WsHeader *hdr)
 {
     constexpr int ldk = LR * CPL;
     constexpr int RPS = 32 / LR;
@@ -141,17 +195,20 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LR, slot = lane / LR;
     const float Bf = (float)B, Mf = (float)M;
-    constexpr uint32_t C = 2;
 
     for (int j = tid; j <= ldk; j += kFuThreads) sh->vs[j] = (j < B || j == ldk) ? v_init : 0.f;
     if (tid < kFuWarps) sh->vsum[tid] = (tid == 0) ? Bf * v_init : 0.f;
 #pragma unroll
     for (int s = 0; s < NS; ++s) U[s] = 0.f;
     __syncthreads();
-    const uint32_t xpart_u32 = ptx::smem_u32(&sh->xpart[0][0][0]), xusum_u32 = ptx::smem_u32(&sh->xusum[0][0]);
+    const uint32_t peer = rank ^ 1u;
+    const uint32_t xpart_peer = ptx::map_to_rank(ptx::smem_u32(&sh->xpart[0][0]), peer);
+    const uint32_t xusum_peer = ptx::map_to_rank(ptx::smem_u32(&sh->xusum[0][0]), peer);
+    const uint32_t xbar_peer = ptx::map_to_rank(ptx::smem_u32(&sh->xbar[0]), peer);
     FuIterState st{0, 0.f};
 
-    for (int it = 0; it < p.iters; ++it) {
+    for (int it = 0; it < p.iters; ++it, ++round) {
+        const uint32_t par = round & 1u, phase = (round >> 1) & 1u;
         float4 V[NQ];
 #pragma unroll
         for (int q = 0; q < NQ; ++q) V[q] = *reinterpret_cast<const float4 *>(sh->vs + 4 * (q * LR + sub));
@@ -165,6 +222,8 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
 #pragma unroll
         for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         float usum = 0.f;
+        // this round's arrival on the local barrier: the other CTA's ldk column sums and its sum of U
+        if (tid == 0) ptx::mbar_arrive_expect_tx(&sh->xbar[par], (uint32_t)(ldk + 1) * 4u);
 
 #pragma unroll
         for (int s = 0; s < NS; ++s) {
@@ -211,36 +270,21 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
         if (lane == 0) sh->wsum[warp] = usum;
         __syncthreads();
 
-        // this CTA's column sums and sum of U go to both CTAs of the cluster
-        const uint32_t slot_x = (uint32_t)(it & 1) * C + rank;
+        // V: thread j completes column j over the warps, sends the sum to the other CTA, waits for that CTA's
+        int cont = 0;
+        float move = 0.f;
         if (tid < ldk) {
             float cs = 0.f;
 #pragma unroll
             for (int w = 0; w < kFuWarps; ++w) cs += part[w * ldk + tid];
-            const uint32_t a = xpart_u32 + (slot_x * (uint32_t)kFuMaxB + (uint32_t)tid) * 4u;
-            ptx::st_cluster_f32(ptx::map_to_rank(a, 0), cs);
-            ptx::st_cluster_f32(ptx::map_to_rank(a, 1), cs);
-        }
-        if (tid == kFuThreads - 1) {
-            float su = 0.f;
-#pragma unroll
-            for (int w = 0; w < kFuWarps; ++w) su += sh->wsum[w];
-            const uint32_t a = xusum_u32 + slot_x * 4u;
-            ptx::st_cluster_f32(ptx::map_to_rank(a, 0), su);
-            ptx::st_cluster_f32(ptx::map_to_rank(a, 1), su);
-        }
-        ptx::cluster_sync_all();
-
-        // V from the completed column sums: one thread per column, the same in both CTAs
-        const float *xb = &sh->xpart[it & 1][0][0];
-        const float *ub = &sh->xusum[it & 1][0];
-        int cont = 0;
-        float move = 0.f;
-        if (tid < ldk) {
+            st_async_peer(xpart_peer + (par * (uint32_t)kFuMaxB + (uint32_t)tid) * 4u, __float_as_uint(cs), xbar_peer + par * 8u);
+            if (!ptx::mbar_wait(&sh->xbar[par], phase)) {
+                sh->abort_flag = 1;
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+            }
             float nv = 0.f;
             if (tid < B) {
-                const float cs = xb[tid] + xb[kFuMaxB + tid];
-                nv = rcp_fast(cs + kappa * Ud);
+                nv = rcp_fast((cs + sh->xpart[par][tid]) + kappa * Ud);
                 const float ov = sh->vs[tid];
                 move = fabsf(nv - ov) * rcp_fast(ov);
                 cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
@@ -250,8 +294,15 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
             if (lane == 0) sh->vsum[warp] = wv;
         }
         if (tid == kFuThreads - 1) {              // the dustbin column
-            const float su = ub[0] + ub[1];
-            const float nVd = Mf * rcp_fast(kappa * (su + Ud));
+            float su = 0.f;
+#pragma unroll
+            for (int w = 0; w < kFuWarps; ++w) su += sh->wsum[w];
+            st_async_peer(xusum_peer + par * 16u, __float_as_uint(su), xbar_peer + par * 8u);
+            if (!ptx::mbar_wait(&sh->xbar[par], phase)) {
+                sh->abort_flag = 1;
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+            }
+            const float nVd = Mf * rcp_fast(kappa * ((su + sh->xusum[par][0]) + Ud));
             const float mj = fabsf(nVd - Vd) * rcp_fast(Vd);
             move = fmaxf(move, mj);
             cont |= p.tol > 0.f ? (mj > p.tol) : (p.stop_fp ? ulp_far(nVd, Vd) : 1);
@@ -259,7 +310,10 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
         }
         st.last_move = move;
         ++st.done;
-        if (!__syncthreads_or(cont)) break;
+        if (!__syncthreads_or(cont)) {
+            ++round;
+            break;
+        }
     }
     // largest relative dual move of the last executed iteration, over the CTA
     float mv = warp_max(st.last_move);
@@ -273,12 +327,14 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
     return st;
 }
 
-// Everything between the K exchange and the merge for one tile layout: K into registers, the
-// iterations, alpha P into the A-operand tiles of the token owners, the per-CTA column maxima of
-// K U for the pairing (into rank 0's xpart).  kbuf: this CTA's K rows [Ml][ldk] in shared memory.
+// Everything between the scores and the merge for one tile layout: K into registers, the iterations,
+// alpha P of this CTA's rows into its plan arrays, the per-CTA column maxima of K U for the pairing
+// (sent to rank 0).  kbuf: this CTA's K rows, pitch ldk + 4 floats, in shared memory (the arena's start,
+// which the plan arrays then overwrite: every thread has its K in registers by then).
 template <int LR, int CPL, int NS>
 __device__ inline FuIterState fused_sinkhorn(FuShared *sh, const float *kbuf, uint8_t *arena, const FuImage &im,
-                                             uint32_t rank, const OtParams &p, float kappa, float v_init)
+                                             uint32_t rank, const OtParams &p, float kappa, float v_init,
+                                             uint32_t &round, WsHeader *hdr)
 {
     constexpr int ldk = LR * CPL;
     constexpr int RPS = 32 / LR;
@@ -294,54 +350,41 @@ __device__ inline FuIterState fused_sinkhorn(FuShared *sh, const float *kbuf, ui
         const int i = (s * kFuWarps + warp) * RPS + slot;
 #pragma unroll
         for (int q = 0; q < NQ; ++q)
-            k[s][q] = (i < im.Ml) ? *reinterpret_cast<const float4 *>(kbuf + (size_t)i * ldk + 4 * (q * LR + sub))
+            k[s][q] = (i < im.Ml) ? *reinterpret_cast<const float4 *>(kbuf + (size_t)i * (ldk + 4) + 4 * (q * LR + sub))
                                   : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    // with no iteration there is no barrier between this load and the plan rows the other CTA will write
-    // over the K buffer
-    if (p.iters == 0) ptx::cluster_sync_all();
 
-    const FuIterState st = fused_iterate<LR, CPL, NS>(k, U, sh, part, im.Ml, im.M, im.B, rank, p, kappa, v_init);
+    const FuIterState st = fused_iterate<LR, CPL, NS>(k, U, sh, part, im.Ml, im.M, im.B, rank, p, kappa, v_init, round, hdr);
     if (p.iters == 0) {
 #pragma unroll
         for (int s = 0; s < NS; ++s) U[s] = ((s * kFuWarps + warp) * RPS + slot < im.Ml) ? 1.f : 0.f;   // u = 0
+        __syncthreads();          // every thread has its K before the plan arrays overwrite the buffer
     }
 
-    // ---- alpha P = alpha U K V in bf16 into the A tiles (128 rows x 64 columns, K-major, 128-byte swizzle)
-    // of the CTA that owns the token: tile (token tile, k-block) at arena + (tile * nkb + kb) * 16 KB
+    // ---- alpha P = alpha U K V in bf16 into this CTA's plan arrays (A operand, K-major): one array of the
+    // CTA's Ra rows per 64 columns, at arena + kb * Ra * 128.  Columns from B up to the next multiple of 16
+    // are zeros (K is zero there): the contraction runs over whole 16-column steps.
     float4 V[NQ];
 #pragma unroll
     for (int q = 0; q < NQ; ++q) V[q] = *reinterpret_cast<const float4 *>(sh->vs + 4 * (q * LR + sub));
-    const uint32_t arena_u32 = ptx::smem_u32(arena);
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
         const int i = (s * kFuWarps + warp) * RPS + slot;
         if (i < im.Ml) {
-            const int tok = sh->toks[i];
-            const uint32_t owner = tok >= im.tpc ? 1u : 0u;
-            const int tr = tok - (int)owner * im.tpc;
-            const int tile = tr >> 7, r = tr & 127;
-            const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
+            const uint32_t row_off = (uint32_t)(i >> 3) * 1024u + (uint32_t)(i & 7) * 128u;
             const float au = p.alpha * U[s];
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 const int col = 4 * (q * LR + sub);
-                if (col < 64 * im.nkb) {
+                if (col < im.Rb) {
                     const int kb = col >> 6, c16 = (col & 63) >> 3;
                     const __nv_bfloat162 lo = __floats2bfloat162_rn((k[s][q].x * au) * V[q].x, (k[s][q].y * au) * V[q].y);
                     const __nv_bfloat162 hi = __floats2bfloat162_rn((k[s][q].z * au) * V[q].z, (k[s][q].w * au) * V[q].w);
-                    const uint32_t off = (uint32_t)(tile * im.nkb + kb) * (uint32_t)kFuABytes + row_off +
-                                         (uint32_t)((c16 ^ (r & 7)) << 4) + (uint32_t)(col & 4) * 2u;
-                    st_cluster_v2_u32(ptx::map_to_rank(arena_u32 + off, owner),
-                                      *reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
+                    const uint32_t off = (uint32_t)kb * (uint32_t)(im.Ra * 128) + row_off +
+                                         (uint32_t)((c16 ^ (i & 7)) << 4) + (uint32_t)(col & 4) * 2u;
+                    *reinterpret_cast<uint2 *>(arena + off) =
+                        make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
                 }
-            }
-            if (ldk < 64) {       // columns 32 .. 63 of the only k-block: zeros (they meet the zero rows of T_p)
-                const int col = 32 + 4 * sub;
-                const int c16 = col >> 3;
-                const uint32_t off = (uint32_t)(tile * im.nkb) * (uint32_t)kFuABytes + row_off +
-                                     (uint32_t)((c16 ^ (r & 7)) << 4) + (uint32_t)(col & 4) * 2u;
-                st_cluster_v2_u32(ptx::map_to_rank(arena_u32 + off, owner), 0u, 0u);
             }
         }
     }
@@ -399,68 +442,348 @@ __device__ inline FuIterState fused_sinkhorn(FuShared *sh, const float *kbuf, ui
                 ib = oi;
             }
         }
-        // to rank 0 (these arrays are not the ones the last iteration's V update may still be reading there)
         ptx::st_cluster_f32(ptx::map_to_rank(ptx::smem_u32(&sh->pairv[rank][tid]), 0), b);
         ptx::st_cluster_u32(ptx::map_to_rank(ptx::smem_u32(&sh->pairi[rank][tid]), 0), (uint32_t)ib);
     }
     return st;
 }
 
+// The 16-byte copies of one stage, shared out over NPROD producer threads (this one is number pt): piece
+// c = pt + NPROD q is the 16 bytes c & 7 of stage row c >> 3 and lands at its swizzled place; a row without
+// a token (rowtok < 0) is written as zeros.  The table holds, per piece, where it comes from in the image
+// (64-column block 0) and where it goes in a stage.
+template <int NCH>
+struct FuChunks {
+    uint32_t src_off[NCH];
+    uint32_t dst_off[NCH];
+    uint32_t real;      // bit q: the piece exists in the image
+    int n;              // pieces of this thread
+};
+
+template <int NCH, int NPROD>
+__device__ inline void fused_chunk_table(FuChunks<NCH> &ck, const FuShared *sh, const FuImage &im, int pt, uint32_t row_bytes)
+{
+    ck.real = 0;
+    ck.n = 0;
+    const int total = 8 * (im.Ra + im.Rb);
+#pragma unroll
+    for (int q = 0; q < NCH; ++q) {
+        const int c = pt + NPROD * q;
+        ck.src_off[q] = 0;
+        ck.dst_off[q] = 0;
+        if (c < total) {
+            ck.n = q + 1;
+            const int row = c >> 3, ch = c & 7;      // Ra is a multiple of 16: row & 7 is the row's place in its group
+            const int tok = sh->rowtok[row];
+            ck.dst_off[q] = (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((ch ^ (row & 7)) << 4));
+            ck.src_off[q] = (uint32_t)max(tok, 0) * row_bytes + (uint32_t)ch * 16u;
+            if (tok >= 0) ck.real |= 1u << q;
+        }
+    }
+}
+
+template <int NCH>
+__device__ inline void fused_issue_stage(const FuChunks<NCH> &ck, const uint8_t *img_base, uint32_t col_bytes, uint32_t stage_u32)
+{
+#pragma unroll
+    for (int q = 0; q < NCH; ++q)
+        if (q < ck.n)
+            ptx::cp_async_16(stage_u32 + ck.dst_off[q], img_base + ck.src_off[q] + col_bytes, ((ck.real >> q) & 1u) ? 16u : 0u);
+    ptx::cp_async_commit();
+}
+
+// Waits until all but the `lag` most recent copy groups of this thread have landed.
+__device__ inline void fused_wait_groups(int lag)
+{
+    if (lag >= 4) ptx::cp_async_wait<4>();
+    else if (lag == 3) ptx::cp_async_wait<3>();
+    else if (lag == 2) ptx::cp_async_wait<2>();
+    else if (lag == 1) ptx::cp_async_wait<1>();
+    else ptx::cp_async_wait<0>();
+}
+
+// Stage 1 of Algorithm 1 for one image inside the cluster (Eq. 1, Eq. 8, Eq. 10, the top-M selection of
+// Section 3.3.1): CTA r streams the image's tokens [r * tpc, ...), tpc = ceil(N / 2), through a ring of
+// shared-memory stages (1-D bulk copies of 16 contiguous rows, one row per warp): sum of squares by
+// shuffles, the norm, and the row divided by its norm into per-lane accumulators.  The two CTAs then
+// hand each other their norms and their sums of unit tokens through distributed shared memory, and both
+// compute phi = (|sum of unit tokens|^2 - N) / (N (N - 1)), the ratio, M, and the selection, in the same
+// order of operations: they agree bit for bit.  Selection: token k is kept iff fewer than M tokens rank
+// before it (larger norm, or equal norm and lower index): every thread counts the tokens that rank before
+// its own.  Fills rowtok, inv_ni, inv_nj; returns M.  Rank 0 writes counts and stats and publishes the
+// image's count to the other clusters (sel_flag[img] = run).
+__device__ inline int fused_stage1(FuShared *sh, uint8_t *arena, const uint8_t *img_base, int img, FuImage &im, int d,
+                                   uint32_t rank, const RatioParams &rp, const float *__restrict__ rho,
+                                   int32_t *__restrict__ counts, float *__restrict__ stats, int *__restrict__ sel_flag,
+                                   int run, WsHeader *hdr)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = im.N;
+    const int tpc = (N + 1) >> 1;
+    const int tok_lo = min(N, (int)rank * tpc);
+    const int ntok = min(N, tok_lo + tpc) - tok_lo;
+    const uint32_t row_bytes = (uint32_t)d * 2u;
+    const int nvec = d >> 3;
+    const uint32_t stage_bytes = (uint32_t)kFuS1Rows * row_bytes;
+    const int nst = min(kFuS1Stages, kFuArenaBytes / (int)stage_bytes);
+    const int nit = (ntok + kFuS1Rows - 1) / kFuS1Rows;
+    const uint32_t arena_u32 = ptx::smem_u32(arena);
+    const uint32_t peer = rank ^ 1u;
+    const float rho_i = (tid == 0 && rho) ? __ldg(rho + img) : 0.f;
+
+    float acc[kFuS1Vpl * 8];
+#pragma unroll
+    for (int e = 0; e < kFuS1Vpl * 8; ++e) acc[e] = 0.f;
+    bool bad = false, gave_up = false;
+    auto issue = [&](int it) {
+        const int s = it % nst;
+        const int r0 = it * kFuS1Rows;
+        const uint32_t bytes = (uint32_t)min(kFuS1Rows, ntok - r0) * row_bytes;
+        ptx::mbar_arrive_expect_tx(&sh->s1_full[s], bytes);
+        ptx::bulk_load(arena_u32 + s * stage_bytes, img_base + (size_t)(tok_lo + r0) * row_bytes, bytes, &sh->s1_full[s]);
+    };
+    if (tid == 0)
+        for (int it = 0; it < min(nst, nit); ++it) issue(it);
+    for (int it = 0; it < nit; ++it) {
+        const int s = it % nst;
+        if (!gave_up && !ptx::mbar_wait(&sh->s1_full[s], (it / nst) & 1)) gave_up = true;
+        const int t = it * kFuS1Rows + warp;
+        if (t < ntok && !gave_up) {
+            const uint4 *row = reinterpret_cast<const uint4 *>(arena + s * stage_bytes + warp * row_bytes);
+            uint4 cur[kFuS1Vpl];
+#pragma unroll
+            for (int j = 0; j < kFuS1Vpl; ++j) {
+                const int vi = lane + 32 * j;
+                cur[j] = (vi < nvec) ? row[vi] : make_uint4(0, 0, 0, 0);
+            }
+            float ss = 0.f;
+#pragma unroll
+            for (int j = 0; j < kFuS1Vpl; ++j) {
+                float f[8];
+                Elem<__nv_bfloat16>::unpack(cur[j], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+            }
+            ss = warp_sum(ss);
+            const float n = sqrtf(ss);
+            if (!(ss <= 3.0e38f)) bad = true;  // inf or NaN
+            const float inv = 1.f / fmaxf(n, kNormFloor);
+            if (lane == 0) {
+                sh->nrm[tok_lo + t] = n;
+                ptx::st_cluster_f32(ptx::map_to_rank(ptx::smem_u32(&sh->nrm[tok_lo + t]), peer), n);
+            }
+#pragma unroll
+            for (int j = 0; j < kFuS1Vpl; ++j) {
+                float f[8];
+                Elem<__nv_bfloat16>::unpack(cur[j], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[j * 8 + e] = fmaf(f[e], inv, acc[j * 8 + e]);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh->s1_empty[s]);
+        if (tid == 0 && it + nst < nit) {        // refill the stage once all the warps have left it
+            if (!gave_up && !ptx::mbar_wait(&sh->s1_empty[s], (it / nst) & 1)) gave_up = true;
+            if (!gave_up) issue(it + nst);
+        }
+    }
+    if (gave_up && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+    if (bad && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_NONFINITE);
+    __syncthreads();          // the ring is free: it now holds the warps' partial sums [16][d], then the CTAs' [2][d]
+    float *wacc = reinterpret_cast<float *>(arena);
+    float *spart = wacc + kFuWarps * d;
+#pragma unroll
+    for (int j = 0; j < kFuS1Vpl; ++j) {
+        const int vi = lane + 32 * j;
+        if (vi < nvec) {
+            *reinterpret_cast<float4 *>(wacc + warp * d + vi * 8) = make_float4(acc[j * 8], acc[j * 8 + 1], acc[j * 8 + 2], acc[j * 8 + 3]);
+            *reinterpret_cast<float4 *>(wacc + warp * d + vi * 8 + 4) = make_float4(acc[j * 8 + 4], acc[j * 8 + 5], acc[j * 8 + 6], acc[j * 8 + 7]);
+        }
+    }
+    // the other CTA is done with the image before (its merge used this part of its arena) before anything lands there
+    ptx::cluster_sync_all();
+    for (int c = tid; c < d; c += kFuThreads) {
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kFuWarps; ++w) sum += wacc[w * d + c];
+        const uint32_t a = ptx::smem_u32(spart + rank * d + c);
+        ptx::st_cluster_f32(ptx::map_to_rank(a, 0), sum);
+        ptx::st_cluster_f32(ptx::map_to_rank(a, 1), sum);
+    }
+    if (tid < 4) sh->nrm[N + tid] = 0.f;      // the ranking reads the norms four at a time
+    ptx::cluster_sync_all();                  // both CTAs hold all the norms and both sums of unit tokens
+
+    // phi (Eq. 8), the ratio (Eq. 10) and M: the same arithmetic in both CTAs
+    float local = 0.f;
+    for (int c = tid; c < d; c += kFuThreads) {
+        const float v = spart[c] + spart[d + c];
+        local = fmaf(v, v, local);
+    }
+    const float ssum = block_sum(local, sh->red);
+    if (tid == 0) {
+        const float Nf = (float)N;
+        const float phi = (N >= 2) ? (ssum - Nf) / (Nf * (Nf - 1.f)) : 0.f;
+        float r;
+        if (rp.dynamic) {
+            float f = (phi - rp.phi_lo) / (rp.phi_hi - rp.phi_lo);
+            f = fminf(fmaxf(f, 0.f), 1.f);
+            r = fminf(f * (1.f - rho_i), rp.r_max);
+        } else {
+            r = rp.r_fixed;
+        }
+        r = fmaxf(r, 0.f);
+        int B = (int)floorf(r * Nf + 0.5f);
+        B = max(0, min(B, N - 1));
+        sh->sel_m = N - B;
+        if (rank == 0) {
+            float *st = stats + (size_t)img * kStats;
+            st[0] = phi;
+            st[1] = rho_i;
+            st[2] = r;
+            st[3] = (float)(N - B);
+            st[4] = (float)B;
+            st[5] = 0.f;
+            st[6] = 0.f;
+            st[7] = 0.f;
+            counts[img] = N - B;
+            __threadfence();
+            ptx::st_release_gpu(sel_flag + img, run);     // the clusters of later images add this count to their out0
+        }
+    }
+    __syncthreads();
+    const int M = sh->sel_m;
+    im.M = M;
+    im.B = N - M;
+    im.half = (M + 1) >> 1;
+    im.row_lo = min(M, (int)rank * im.half);
+    im.Ml = min(M, im.row_lo + im.half) - im.row_lo;
+    im.ntile = (im.Ml + kFuTileM - 1) / kFuTileM;
+    im.ldk = im.B > 0 ? sinkhorn_ldk(im.B) : 32;
+    im.nkb = (im.B + 63) >> 6;
+    im.Ra = (im.Ml + 15) & ~15;
+    im.Rb = (im.B + 15) & ~15;
+
+    // ---- selection: thread k ranks token k among all N (norm bits: the unsigned order is the float order) ----
+    const int k = tid;
+    bool kept = false;
+    if (k < N) {
+        const uint32_t mine = __float_as_uint(sh->nrm[k]) & 0x7fffffffu;
+        int before = 0;
+        for (int j0 = 0; j0 < N; j0 += 4) {
+            const float4 v = *reinterpret_cast<const float4 *>(sh->nrm + j0);
+            const uint32_t kj[4] = {__float_as_uint(v.x) & 0x7fffffffu, __float_as_uint(v.y) & 0x7fffffffu,
+                                    __float_as_uint(v.z) & 0x7fffffffu, __float_as_uint(v.w) & 0x7fffffffu};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = j0 + e;
+                before += (j < N && (kj[e] > mine || (kj[e] == mine && j < k))) ? 1 : 0;
+            }
+        }
+        kept = before < M;
+    }
+    // positions in ascending token order: kept tokens before k, pruned tokens before k
+    const uint32_t kmask = __ballot_sync(0xffffffffu, kept);
+    const uint32_t pmask = __ballot_sync(0xffffffffu, k < N && !kept);
+    if (lane == 0) {
+        sh->wcount[0][warp] = __popc(kmask);
+        sh->wcount[1][warp] = __popc(pmask);
+    }
+    for (int r = tid; r < im.Ra + im.Rb; r += kFuThreads) sh->rowtok[r] = -1;
+    __syncthreads();
+    int kb = 0, pb = 0;
+    for (int w = 0; w < warp; ++w) {
+        kb += sh->wcount[0][w];
+        pb += sh->wcount[1][w];
+    }
+    const uint32_t lt = (1u << lane) - 1u;
+    if (k < N) {
+        if (kept) {
+            const int pos = kb + __popc(kmask & lt) - im.row_lo;      // among this CTA's kept rows?
+            if (pos >= 0 && pos < im.Ml) {
+                sh->rowtok[pos] = k;
+                sh->inv_ni[pos] = 1.f / fmaxf(sh->nrm[k], kNormFloor);
+            }
+        } else {
+            const int pos = pb + __popc(pmask & lt);
+            sh->rowtok[im.Ra + pos] = k;
+            sh->inv_nj[pos] = 1.f / fmaxf(sh->nrm[k], kNormFloor);
+        }
+    }
+    __syncthreads();
+    return M;
+}
+
+__device__ inline void fused_init_barriers(FuShared *sh, bool again)
+{
+    for (int s = 0; s < kFuScStages; ++s) {
+        if (again) {
+            mbar_inval(&sh->sc_full[s]);
+            mbar_inval(&sh->sc_empty[s]);
+        }
+        ptx::mbar_init(&sh->sc_full[s], kFuScProducers);
+        ptx::mbar_init(&sh->sc_empty[s], 1);
+    }
+    if (again) mbar_inval(&sh->sc_accum);
+    ptx::mbar_init(&sh->sc_accum, 1);
+    for (int s = 0; s < kFuMgStages; ++s) {
+        if (again) {
+            mbar_inval(&sh->mg_full[s]);
+            mbar_inval(&sh->mg_empty[s]);
+        }
+        ptx::mbar_init(&sh->mg_full[s], kFuMgProducers);
+        ptx::mbar_init(&sh->mg_empty[s], kFuEpiWarps * 32);
+    }
+    for (int s = 0; s < kFuAccStages; ++s) {
+        if (again) {
+            mbar_inval(&sh->acc_full[s]);
+            mbar_inval(&sh->acc_empty[s]);
+        }
+        ptx::mbar_init(&sh->acc_full[s], 1);
+        ptx::mbar_init(&sh->acc_empty[s], kFuEpiWarps * 32);
+    }
+    for (int s = 0; s < kFuS1Stages; ++s) {
+        if (again) {
+            mbar_inval(&sh->s1_full[s]);
+            mbar_inval(&sh->s1_empty[s]);
+        }
+        ptx::mbar_init(&sh->s1_full[s], 1);
+        ptx::mbar_init(&sh->s1_empty[s], kFuWarps);
+    }
+    ptx::fence_mbar_init();
+}
+
+template <bool WITH_S1>
 __global__ void __launch_bounds__(kFuThreads, 1)
-stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes of 64 columns x 128 rows
-                    const __grid_constant__ CUtensorMap tmapXb,    // X, boxes of 64 columns x 64 rows
-                    const __grid_constant__ CUtensorMap tmapXp,    // compact copy, boxes of 64 x 64
-                    const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ offsets, int d, int batch,
+stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ offsets, int d, int batch,
                     const int32_t *__restrict__ counts, const int32_t *__restrict__ order,
-                    const int32_t *__restrict__ kpos, const float *__restrict__ norms, __nv_bfloat16 *__restrict__ xp,
-                    int max_tokens, int total, OtParams p, __nv_bfloat16 *__restrict__ Y,
-                    int32_t *__restrict__ out_offsets, int32_t *__restrict__ kept_idx,
+                    const float *__restrict__ norms, int max_tokens, int total, OtParams p,
+                    __nv_bfloat16 *__restrict__ Y, int32_t *__restrict__ out_offsets, int32_t *__restrict__ kept_idx,
                     int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
-                    float *__restrict__ merge_weight, float *__restrict__ stats, WsHeader *__restrict__ hdr)
+                    float *__restrict__ merge_weight, float *__restrict__ stats, WsHeader *__restrict__ hdr,
+                    // stage 1 inside this kernel (WITH_S1: counts, order and norms are not inputs then; counts is
+                    // written here and sel_flag[img] = run tells the other clusters that it is)
+                    RatioParams rp, const float *__restrict__ rho, int32_t *counts_out,
+                    int *__restrict__ sel_flag, int run)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *ident = smem;
-    FuShared *sh = reinterpret_cast<FuShared *>(smem + kFuIdentBytes);
-    uint8_t *arena = smem + kFuIdentBytes + kFuSharedBytes;
+    FuShared *sh = reinterpret_cast<FuShared *>(smem);
+    uint8_t *arena = smem + kFuSharedBytes;
     const uint32_t arena_u32 = ptx::smem_u32(arena);
     const uint32_t rank = ptx::cluster_ctarank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cluster_id = blockIdx.x >> 1, nclusters = gridDim.x >> 1;
+    const uint32_t row_bytes = (uint32_t)d * 2u;
 
-    // ---- set-up that needs nothing from the kernels ahead: identity block, tensor memory ---------------
-    // rows 64 .. 127 of a 192-row region hold I_64 (ones at (64 + r, k = r)) in the swizzled K-major
-    // layout, the other rows are zero: the view that starts at row 64 has its ones in rows 0-63, the view
-    // that starts at row 0 in rows 64-127.
-    for (int v = tid; v < kFuIdentBytes / 16; v += kFuThreads) reinterpret_cast<uint4 *>(ident)[v] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
-    if (tid < 64) {
-        const int r = 64 + tid, k = tid;
-        const uint32_t off = (r >> 3) * 1024 + (r & 7) * 128 + (((k >> 3) ^ (r & 7)) << 4) + (k & 7) * 2;
-        *reinterpret_cast<uint16_t *>(ident + off) = 0x3F80;   // bf16 1.0
-    }
-    ptx::fence_proxy_async_smem();
+    // ---- set-up that needs nothing from the kernels ahead ------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kFuScStages; ++s) {
-            ptx::mbar_init(&sh->sc_full[s], 1);
-            ptx::mbar_init(&sh->sc_empty[s], 1);
-        }
-        ptx::mbar_init(&sh->sc_accum, 1);
-        for (int s = 0; s < kFuMgStages; ++s) {
-            ptx::mbar_init(&sh->mg_full[s], 1);
-            ptx::mbar_init(&sh->mg_empty[s], 1);
-        }
-        for (int s = 0; s < kFuAccStages; ++s) {
-            ptx::mbar_init(&sh->acc_full[s], 1);
-            ptx::mbar_init(&sh->acc_empty[s], 128);
-        }
+        fused_init_barriers(sh, false);
+        ptx::mbar_init(&sh->xbar[0], 1);
+        ptx::mbar_init(&sh->xbar[1], 1);
         sh->abort_flag = 0;
         ptx::fence_mbar_init();
-        ptx::prefetch_tensormap(&tmapXa);
-        ptx::prefetch_tensormap(&tmapXb);
-        ptx::prefetch_tensormap(&tmapXp);
     }
-    if (warp == 1) {
+    if (warp == kFuMmaWarp) {
         ptx::tmem_alloc(&sh->tmem_base, 512);
         ptx::tmem_relinquish();
     }
@@ -470,7 +793,7 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
     const uint32_t tmem_base = sh->tmem_base;
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();          // the selection comes from the kernel ahead
-    // both CTAs are running and have their shared memory laid out before anyone writes into the other's
+    // both CTAs are running and have their barriers in place before anyone writes into the other's shared memory
     ptx::cluster_sync_all();
 
     const float inv_eps = 1.f / p.eps;
@@ -479,6 +802,7 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
     const float v_init = expf(shift * inv_eps);
     const int nct = d / kFuNT;
     const int nkblk = d / kFuBK;
+    uint32_t round = 0;            // exchanges of column sums so far (the same in both CTAs)
     bool first = true;
 
     for (int img = cluster_id; img < batch; img += nclusters) {
@@ -486,8 +810,19 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
         if (!image_range(offsets, img, max_tokens, total, im.t_begin, im.N)) {
             // no output rows; the image's slot of out_offsets still has to be right
             if (rank == 0 && warp == 0) {
+                if (WITH_S1 && lane == 0) {      // offsets broke the contract: the image yields no output
+                    atomicOr(&hdr->status, RTPRUNE_DEV_BAD_OFFSETS);
+                    counts_out[img] = 0;
+                    float *st = stats + (size_t)img * kStats;
+                    for (int q = 0; q < kStats; ++q) st[q] = 0.f;
+                    __threadfence();
+                    ptx::st_release_gpu(sel_flag + img, run);
+                }
                 int s = 0;
-                for (int b = lane; b < img; b += 32) s += __ldcg(counts + b);
+                for (int b = lane; b < img; b += 32) {
+                    if (WITH_S1 && !ptx::wait_equal_gpu(sel_flag + b, run)) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                    s += __ldcg(counts + b);
+                }
                 for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
                 if (lane == 0) {
                     out_offsets[img] = s;
@@ -496,56 +831,42 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
             }
             continue;
         }
-        im.M = __ldcg(counts + img);
-        im.B = im.N - im.M;
-        im.tpc = (im.N + 1) >> 1;
-        im.tok_lo = min(im.N, (int)rank * im.tpc);
-        im.ntok = min(im.N, im.tok_lo + im.tpc) - im.tok_lo;
-        im.ntile = (im.ntok + kFuTileM - 1) / kFuTileM;
-        im.half = (im.M + 1) >> 1;
-        im.row_lo = min(im.M, (int)rank * im.half);
-        im.Ml = min(im.M, im.row_lo + im.half) - im.row_lo;
-        im.ldk = im.B > 0 ? sinkhorn_ldk(im.B) : 32;
-        im.nkb = (im.B + 63) >> 6;
-        im.nbox = im.nkb;
-        im.BN = (im.B + 15) & ~15;
-        const int xp0 = xp_row0(im.t_begin, img);
-        const int32_t *ord = order + im.t_begin;
-
-        if (!first) {
-            // the barriers start every image in phase 0 (their rings differ from image to image)
-            __syncthreads();
-            if (tid == 0) {
-                for (int s = 0; s < kFuScStages; ++s) {
-                    mbar_inval(&sh->sc_full[s]);
-                    mbar_inval(&sh->sc_empty[s]);
-                    ptx::mbar_init(&sh->sc_full[s], 1);
-                    ptx::mbar_init(&sh->sc_empty[s], 1);
-                }
-                mbar_inval(&sh->sc_accum);
-                ptx::mbar_init(&sh->sc_accum, 1);
-                for (int s = 0; s < kFuMgStages; ++s) {
-                    mbar_inval(&sh->mg_full[s]);
-                    mbar_inval(&sh->mg_empty[s]);
-                    ptx::mbar_init(&sh->mg_full[s], 1);
-                    ptx::mbar_init(&sh->mg_empty[s], 1);
-                }
-                for (int s = 0; s < kFuAccStages; ++s) {
-                    mbar_inval(&sh->acc_full[s]);
-                    mbar_inval(&sh->acc_empty[s]);
-                    ptx::mbar_init(&sh->acc_full[s], 1);
-                    ptx::mbar_init(&sh->acc_empty[s], 128);
-                }
-                ptx::fence_mbar_init();
-            }
-            __syncthreads();
-        }
+        const uint8_t *img_base = reinterpret_cast<const uint8_t *>(X + (size_t)im.t_begin * d);
+        // the ring barriers start every image in phase 0 (the rings differ from image to image)
+        if (!first && tid == 0) fused_init_barriers(sh, true);
+        if (!first) __syncthreads();
         first = false;
 
-        // ---- out0 = number of kept rows of the images before this one (warp 15) ----------------------------
+        if constexpr (WITH_S1) {
+            fused_stage1(sh, arena, img_base, img, im, d, rank, rp, rho, counts_out, stats, sel_flag, run, hdr);
+        } else {
+            im.M = __ldcg(counts + img);
+            im.B = im.N - im.M;
+            im.half = (im.M + 1) >> 1;
+            im.row_lo = min(im.M, (int)rank * im.half);
+            im.Ml = min(im.M, im.row_lo + im.half) - im.row_lo;
+            im.ntile = (im.Ml + kFuTileM - 1) / kFuTileM;
+            im.ldk = im.B > 0 ? sinkhorn_ldk(im.B) : 32;
+            im.nkb = (im.B + 63) >> 6;
+            im.Ra = (im.Ml + 15) & ~15;
+            im.Rb = (im.B + 15) & ~15;
+            // which token each row of a stage is (one trip to L2)
+            const int32_t *ord = order + im.t_begin;
+            for (int r = tid; r < im.Ra + im.Rb; r += kFuThreads) {
+                int tok = -1;
+                if (r < im.Ml) tok = __ldcg(ord + im.row_lo + r);
+                else if (r >= im.Ra && r - im.Ra < im.B) tok = __ldcg(ord + im.M + (r - im.Ra));
+                sh->rowtok[r] = tok;
+            }
+        }
+        // out0 = number of kept rows of the images before this one (with stage 1 in this kernel their counts
+        // come from other clusters, which publish them as soon as they have them)
         if (warp == kFuWarps - 1) {
             int s = 0;
-            for (int b = lane; b < img; b += 32) s += __ldcg(counts + b);
+            for (int b = lane; b < img; b += 32) {
+                if (WITH_S1 && !ptx::wait_equal_gpu(sel_flag + b, run)) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                s += __ldcg(counts + b);
+            }
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == 0) {
                 sh->out0 = s;
@@ -555,68 +876,49 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                 }
             }
         }
+        __syncthreads();
 
         FuIterState ist{0, 0.f};
         if (im.B > 0) {
-            // ---- compact copy of the pruned rows: rows j = warp of the cluster, + 32, ...; zero rows up to
-            // a multiple of 64 (whole 64-row boxes are fetched)
-            {
-                const int nvec = d >> 3;
-                const int gw = (int)rank * kFuWarps + warp;
-                uint4 *seg = reinterpret_cast<uint4 *>(xp + (size_t)xp0 * d);
-                for (int j = gw; j < 64 * im.nkb; j += 2 * kFuWarps) {
-                    const uint4 *src = (j < im.B)
-                                           ? reinterpret_cast<const uint4 *>(X + (size_t)(im.t_begin + __ldcg(ord + im.M + j)) * d)
-                                           : nullptr;
-                    for (int v0 = lane; v0 < nvec; v0 += 32 * 5) {
-                        uint4 t[5];
-#pragma unroll
-                        for (int b = 0; b < 5; ++b) {
-                            const int v = v0 + 32 * b;
-                            t[b] = (src && v < nvec) ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
-                        }
-#pragma unroll
-                        for (int b = 0; b < 5; ++b) {
-                            const int v = v0 + 32 * b;
-                            if (v < nvec) seg[(size_t)j * nvec + v] = t[b];
-                        }
+            // ---- scores: D[tile] = T_k[tile rows] . T_p^T over the full width ------------------------------
+            const int stage_bytes = fused_stage_bytes(im.Ml, im.B);
+            const int nstages = im.ntile > 0 ? min(kFuScStages, (kFuArenaBytes - kFuABytes) / stage_bytes) : 1;
+            const int lag = max(0, nstages - 2);          // copy groups a producer keeps in flight behind the newest
+            if (warp >= 1 && im.ntile > 0) {
+                const int pt = tid - 32;
+                FuChunks<kFuScChunks> ck;
+                fused_chunk_table<kFuScChunks, kFuScProducers>(ck, sh, im, pt, row_bytes);
+                bool ok = true;
+                for (int kb = 0; kb < nkblk; ++kb) {
+                    const int s = kb % nstages;
+                    if (ok && kb >= nstages && !ptx::mbar_wait(&sh->sc_empty[s], ((kb / nstages) - 1) & 1)) ok = false;
+                    if (ok) fused_issue_stage(ck, img_base, (uint32_t)kb * 128u, arena_u32 + s * stage_bytes);
+                    else ptx::cp_async_commit();
+                    if (kb >= lag) {
+                        fused_wait_groups(lag);
+                        ptx::fence_proxy_async_smem();
+                        ptx::mbar_arrive(&sh->sc_full[(kb - lag) % nstages]);
                     }
                 }
-            }
-            // 1 / |x_j| of the pruned tokens; tokens of this CTA's kept rows
-            for (int j = tid; j < im.B; j += kFuThreads)
-                sh->inv_nj[j] = 1.f / fmaxf(__ldcg(norms + im.t_begin + __ldcg(ord + im.M + j)), kNormFloor);
-            for (int i = tid; i < im.Ml; i += kFuThreads) sh->toks[i] = __ldcg(ord + im.row_lo + i);
-            __threadfence();
-            ptx::fence_proxy_async_all();      // the copy is read by TMA
-            ptx::cluster_sync_all();           // #0: the whole compact copy is in place
-
-            // ---- scores: D[tile] = X[tile rows] . T_p^T over the full width --------------------------------
-            const int stage_bytes = im.ntile * kFuABytes + im.nbox * kFuBoxBytes;
-            const int nstages = min(kFuScStages, kFuArenaBytes / stage_bytes);
-            if (warp == 0) {
-                if (lane == 0) {
-                    ptx::fence_proxy_async_all();
-                    for (int kb = 0; kb < nkblk && !sh->abort_flag; ++kb) {
-                        const int s = kb % nstages;
-                        if (kb >= nstages && !ptx::mbar_wait(&sh->sc_empty[s], ((kb / nstages) - 1) & 1)) {
-                            sh->abort_flag = 1;
-                            atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-                            break;
-                        }
-                        const uint32_t dst = arena_u32 + s * stage_bytes;
-                        ptx::mbar_arrive_expect_tx(&sh->sc_full[s], (uint32_t)stage_bytes);
-                        for (int t = 0; t < im.ntile; ++t)
-                            ptx::tma_load_2d(dst + t * kFuABytes, &tmapXa, &sh->sc_full[s], kb * kFuBK,
-                                             im.t_begin + im.tok_lo + t * kFuTileM);
-                        for (int b = 0; b < im.nbox; ++b)
-                            ptx::tma_load_2d(dst + im.ntile * kFuABytes + b * kFuBoxBytes, &tmapXp, &sh->sc_full[s],
-                                             kb * kFuBK, xp0 + b * 64);
-                    }
+                for (int kb = max(nkblk - lag, 0); kb < nkblk; ++kb) {
+                    ptx::cp_async_wait<0>();
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(&sh->sc_full[kb % nstages]);
                 }
-            } else if (warp == 1) {
-                if (lane == 0) {
-                    const uint32_t idesc = ptx::idesc_bf16(kFuTileM, im.BN, false, false);
+                if (!ok) {
+                    sh->abort_flag = 1;
+                    atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                }
+                // the norms of the rows, while the last k-blocks are multiplied (stage 1 in this kernel left them)
+                if (!WITH_S1) {
+                    for (int i = pt; i < im.Ml; i += kFuScProducers)
+                        sh->inv_ni[i] = 1.f / fmaxf(__ldcg(norms + im.t_begin + sh->rowtok[i]), kNormFloor);
+                    for (int j = pt; j < im.B; j += kFuScProducers)
+                        sh->inv_nj[j] = 1.f / fmaxf(__ldcg(norms + im.t_begin + sh->rowtok[im.Ra + j]), kNormFloor);
+                }
+            } else if (warp == 0) {
+                if (lane == 0 && im.ntile > 0) {
+                    const uint32_t idesc = ptx::idesc_bf16(kFuTileM, im.Rb, false, false);
                     for (int kb = 0; kb < nkblk && !sh->abort_flag; ++kb) {
                         const int s = kb % nstages;
                         if (!ptx::mbar_wait(&sh->sc_full[s], (kb / nstages) & 1)) {
@@ -626,7 +928,7 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                         }
                         ptx::tc_fence_after();
                         const uint32_t a_base = arena_u32 + s * stage_bytes;
-                        const uint32_t b_base = a_base + im.ntile * kFuABytes;
+                        const uint32_t b_base = a_base + im.Ra * 128;
                         for (int t = 0; t < im.ntile; ++t) {
 #pragma unroll
                             for (int k = 0; k < kFuBK / 16; ++k) {
@@ -642,35 +944,31 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
             }
             __syncwarp();
             // everybody: the accumulators are complete (and with them every read of the ring)
-            {
-                bool ok = im.ntile == 0 || ptx::mbar_wait(&sh->sc_accum, 0);
-                if (!ok) {
-                    sh->abort_flag = 1;
-                    atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-                }
+            if (im.ntile > 0 && !ptx::mbar_wait(&sh->sc_accum, 0)) {
+                sh->abort_flag = 1;
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
             }
             ptx::tc_fence_after();
-            ptx::cluster_sync_all();           // #1: both rings are free: the K rows may land on them
+            __syncthreads();               // inv_ni, inv_nj; and nobody still waits on the ring's barriers
 
-            // ---- epilogue: K = exp((S - c) / eps) of a kept token's row to the owner of its kept position --
-            // warp (quarter q = warp % 4, g = warp / 4): tile g & 1, column chunks of 32 from (g >> 1), step 2
+            // ---- epilogue: K = exp((S - c) / eps) of this CTA's rows into shared memory (the ring is free) ----
+            // warp (quarter q = warp % 4, g = warp / 4): tile g & 1, column chunks of 32 from (g >> 1), step 2.
+            // Row pitch ldk + 4 floats: a warp's 32 rows of 16 bytes fall into distinct banks.
+            float *kbuf = reinterpret_cast<float *>(arena);
             if (!sh->abort_flag) {
                 const int q = warp & 3, g = warp >> 2;
                 const int tile = g & 1;
                 const int nchunk = im.ldk >> 5;
                 if (tile < im.ntile) {
-                    const int tr = tile * kFuTileM + q * 32 + lane;
-                    const int tok = im.tok_lo + tr;
-                    const int pk = (tr < im.ntok) ? __ldcg(kpos + im.t_begin + tok) : -1;
-                    const float inv_ni = (pk >= 0) ? 1.f / fmaxf(__ldcg(norms + im.t_begin + tok), kNormFloor) : 0.f;
-                    const uint32_t owner = (pk >= im.half) ? 1u : 0u;
-                    const uint32_t krow = ptx::map_to_rank(arena_u32, owner) +
-                                          (uint32_t)(max(pk, 0) - (int)owner * im.half) * (uint32_t)im.ldk * 4u;
+                    const int i = tile * kFuTileM + q * 32 + lane;
+                    const bool have = i < im.Ml;
+                    const float inv_ni = have ? sh->inv_ni[i] : 0.f;
+                    float *krow = kbuf + (size_t)min(i, kFuMaxRows - 1) * (im.ldk + 4);
                     for (int c = (g >> 1); c < nchunk; c += 2) {
                         uint32_t r[32];
                         ptx::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tile * 256 + c * 32), r);
                         ptx::tmem_ld_wait();
-                        if (pk >= 0) {
+                        if (have) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v) {
                                 float4 kv;
@@ -679,21 +977,20 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                                 kv.y = (j + 1 < im.B) ? exp_fast((__uint_as_float(r[4 * v + 1]) * inv_ni * sh->inv_nj[min(j + 1, kFuMaxB - 1)] - shift) * inv_eps) : 0.f;
                                 kv.z = (j + 2 < im.B) ? exp_fast((__uint_as_float(r[4 * v + 2]) * inv_ni * sh->inv_nj[min(j + 2, kFuMaxB - 1)] - shift) * inv_eps) : 0.f;
                                 kv.w = (j + 3 < im.B) ? exp_fast((__uint_as_float(r[4 * v + 3]) * inv_ni * sh->inv_nj[min(j + 3, kFuMaxB - 1)] - shift) * inv_eps) : 0.f;
-                                st_cluster_v4(krow + (uint32_t)j * 4u, kv);
+                                *reinterpret_cast<float4 *>(krow + j) = kv;
                             }
                         }
                     }
                 }
             }
             ptx::tc_fence_before();
-            ptx::cluster_sync_all();           // #2: every K row is with its owner
+            __syncthreads();
             ptx::tc_fence_after();
 
             // ---- Sinkhorn on this CTA's rows ---------------------------------------------------------------
-            const float *kbuf = reinterpret_cast<const float *>(arena);
             const int rps = im.ldk <= 128 ? 4 : 2;
             const int ns = max(1, (im.half + kFuWarps * rps - 1) / (kFuWarps * rps));
-#define RTP_FU(LR, CPL, NS) ist = fused_sinkhorn<LR, CPL, NS>(sh, kbuf, arena, im, rank, p, kappa, v_init)
+#define RTP_FU(LR, CPL, NS) ist = fused_sinkhorn<LR, CPL, NS>(sh, kbuf, arena, im, rank, p, kappa, v_init, round, hdr)
 #define RTP_FU_NS(LR, CPL, NSMAX)                                 \
     switch (ns) {                                                 \
     case 1: RTP_FU(LR, CPL, 1); break;                            \
@@ -715,67 +1012,72 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                 stats[(size_t)img * kStats + 5] = (float)ist.done;
                 stats[(size_t)img * kStats + 6] = ist.last_move;
             }
-            ptx::fence_proxy_async_all();      // the plan rows (ordinary stores, some into the other CTA) feed UMMAs
-            ptx::cluster_sync_all();           // #3: plan tiles and pairing partials are in place
+            ptx::fence_proxy_async_smem();     // the plan arrays (ordinary stores) feed UMMAs
         }
+        // the pairing partials are with rank 0; the plan arrays and out0 are in place
+        ptx::cluster_sync_all();
 
-        __syncthreads();                       // out0 (with nothing pruned no barrier has passed since it was written)
-        // ---- rank 0, warps 8-15: the pairs ---------------------------------------------------------------
-        if (im.B > 0 && rank == 0 && warp >= 8) {
-            const int out0 = sh->out0;
-            const int seg = im.t_begin - out0;
-            for (int j = tid - 256; j < im.B; j += 256) {
-                float b = sh->pairv[0][j];
-                int ib = sh->pairi[0][j];
-                const float ob = sh->pairv[1][j];      // rank 1 holds the higher rows: strict > keeps the lower
-                if (ob > b) {
-                    b = ob;
-                    ib = sh->pairi[1][j];
-                }
-                merged_idx[seg + j] = __ldcg(ord + im.M + j);
-                merge_partner[seg + j] = ib;
-                merge_weight[seg + j] = b * sh->vs[j];
-            }
-        }
-
-        // ---- merge: for every tile of 64 output columns, [I | alpha P] . [X rows of the token tiles ; T_p] ----
-        const int nident0 = im.ntile > 0 ? (min(im.ntok, kFuTileM) > 64 ? 2 : 1) : 0;
-        const int nident1 = im.ntile > 1 ? (im.ntok - kFuTileM > 64 ? 2 : 1) : 0;
-        if (warp == 0) {
-            if (lane == 0 && im.ntile > 0) {
-                ptx::fence_proxy_async_all();
-                uint32_t it = 0;
-                for (int ct = 0; ct < nct && !sh->abort_flag; ++ct) {
-                    const int nload = nident0 + nident1 + im.nkb;
-                    for (int l = 0; l < nload; ++l, ++it) {
-                        const int s = it % kFuMgStages;
-                        if (it >= (uint32_t)kFuMgStages &&
-                            !ptx::mbar_wait(&sh->mg_empty[s], ((it / kFuMgStages) - 1) & 1)) {
-                            sh->abort_flag = 1;
-                            atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-                            break;
-                        }
-                        const uint32_t dst = arena_u32 + kFuPartOffset + s * kFuBoxBytes;
-                        ptx::mbar_arrive_expect_tx(&sh->mg_full[s], kFuBoxBytes);
-                        if (l < nident0 + nident1) {
-                            const int t = l < nident0 ? 0 : 1, kb = l < nident0 ? l : l - nident0;
-                            ptx::tma_load_2d(dst, &tmapXb, &sh->mg_full[s], ct * kFuNT,
-                                             im.t_begin + im.tok_lo + t * kFuTileM + kb * 64);
-                        } else {
-                            ptx::tma_load_2d(dst, &tmapXp, &sh->mg_full[s], ct * kFuNT, xp0 + (l - nident0 - nident1) * 64);
-                        }
+        const int out0 = sh->out0;
+        // ---- merge: for every tile of 64 output columns, acc = alpha P . T_p on the tensor cores; the epilogue
+        // adds the kept token's own row (it sits in the stage, fetched with the pruned rows), rounds to bf16
+        // in place there, and writes the rows out with coalesced 16-byte stores (they are consecutive rows of Y).
+        // arena: plan arrays | ring (it takes the place of the column partials, consumed before the barrier above)
+        const int plan_bytes = fused_plan_bytes(im.Ml, im.B);
+        const int mstage_bytes = fused_stage_bytes(im.Ml, im.B);
+        const int mstages = im.ntile > 0 ? min(kFuMgStages, (kFuArenaBytes - plan_bytes) / mstage_bytes) : 1;
+        const uint32_t ring_off = (uint32_t)plan_bytes;
+        const int ksteps_p = im.Rb >> 4;                        // 16-row steps over the pruned rows
+        if (warp > kFuMmaWarp && im.ntile > 0) {
+            const int pt = tid - (kFuMmaWarp + 1) * 32;
+            if (im.B > 0 && rank == 0) {
+                // the pairs: rank 1 holds the higher rows, so strict > keeps the lower row on ties
+                const int seg = im.t_begin - out0;
+                for (int j = pt; j < im.B; j += kFuMgProducers) {
+                    float b = sh->pairv[0][j];
+                    int ib = sh->pairi[0][j];
+                    const float ob = sh->pairv[1][j];
+                    if (ob > b) {
+                        b = ob;
+                        ib = sh->pairi[1][j];
                     }
+                    merged_idx[seg + j] = sh->rowtok[im.Ra + j];
+                    merge_partner[seg + j] = ib;
+                    merge_weight[seg + j] = b * sh->vs[j];
                 }
             }
-        } else if (warp == 1) {
+            for (int i = pt; i < im.Ml; i += kFuMgProducers) kept_idx[out0 + im.row_lo + i] = sh->rowtok[i];
+            // the rows sit in L2 (this SM fetched them for the scores): a group lands while the next one is issued
+            const int mlag = min(1, mstages - 1);
+            FuChunks<kFuMgChunks> ck;
+            fused_chunk_table<kFuMgChunks, kFuMgProducers>(ck, sh, im, pt, row_bytes);
+            bool ok = true;
+            for (int ct = 0; ct < nct; ++ct) {
+                const int s = ct % mstages;
+                if (ok && ct >= mstages && !ptx::mbar_wait(&sh->mg_empty[s], ((ct / mstages) - 1) & 1)) ok = false;
+                if (ok) fused_issue_stage(ck, img_base, (uint32_t)ct * (kFuNT * 2), arena_u32 + ring_off + s * mstage_bytes);
+                else ptx::cp_async_commit();
+                if (ct >= mlag) {
+                    fused_wait_groups(mlag);
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(&sh->mg_full[(ct - mlag) % mstages]);
+                }
+            }
+            for (int ct = max(nct - mlag, 0); ct < nct; ++ct) {
+                ptx::cp_async_wait<0>();
+                ptx::fence_proxy_async_smem();
+                ptx::mbar_arrive(&sh->mg_full[ct % mstages]);
+            }
+            if (!ok) {
+                sh->abort_flag = 1;
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+            }
+        } else if (warp == kFuMmaWarp) {
             if (lane == 0 && im.ntile > 0) {
                 ptx::fence_proxy_async_smem();
                 const uint32_t idesc = ptx::idesc_bf16(kFuTileM, kFuNT, false, true);
-                const uint32_t ident_u32 = ptx::smem_u32(ident);
-                uint32_t it = 0;
                 bool failed = false;
                 for (int ct = 0; ct < nct && !sh->abort_flag && !failed; ++ct) {
-                    const int as = ct % kFuAccStages;
+                    const int s = ct % mstages, as = ct % kFuAccStages;
                     if (ct >= kFuAccStages) {
                         if (!ptx::mbar_wait(&sh->acc_empty[as], ((ct / kFuAccStages) - 1) & 1)) {
                             failed = true;
@@ -783,70 +1085,49 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                         }
                         ptx::tc_fence_after();
                     }
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
-                    for (int t = 0; t < im.ntile && !failed; ++t) {
-                        const int ni = t == 0 ? nident0 : nident1;
-                        for (int kb = 0; kb < ni; ++kb, ++it) {
-                            const int s = it % kFuMgStages;
-                            if (!ptx::mbar_wait(&sh->mg_full[s], (it / kFuMgStages) & 1)) {
-                                failed = true;
-                                break;
-                            }
-                            ptx::tc_fence_after();
-                            const uint32_t a_base = ident_u32 + (1 - kb) * (kFuABytes / 2);
-                            const uint32_t b_base = arena_u32 + kFuPartOffset + s * kFuBoxBytes;
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const uint64_t da = ptx::smem_desc_sw128(a_base + k * 32, 16, 1024);
-                                const uint64_t db = ptx::smem_desc_sw128(b_base + k * 2048, kFuBoxBytes, 1024);
-                                ptx::umma_bf16(d_tmem + (uint32_t)(t * 64), da, db, idesc, (kb | k) != 0);
-                            }
-                            ptx::umma_commit(&sh->mg_empty[s]);
+                    if (!ptx::mbar_wait(&sh->mg_full[s], (ct / mstages) & 1)) {
+                        failed = true;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t stage = arena_u32 + ring_off + s * mstage_bytes;
+                    for (int t = 0; t < im.ntile; ++t) {
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128 + t * 64);
+                        for (int ks = 0; ks < ksteps_p; ++ks) {
+                            const int kb = ks >> 2, k = ks & 3;
+                            const uint64_t da = ptx::smem_desc_sw128(arena_u32 + (uint32_t)(kb * im.Ra * 128 + t * kFuABytes) + k * 32, 16, 1024);
+                            const uint64_t db = ptx::smem_desc_sw128(stage + (im.Ra + ks * 16) * 128, kFuBoxBytes, 1024);
+                            ptx::umma_bf16(d_tmem, da, db, idesc, ks != 0);
                         }
                     }
-                    for (int kb = 0; kb < im.nkb && !failed; ++kb, ++it) {
-                        const int s = it % kFuMgStages;
-                        if (!ptx::mbar_wait(&sh->mg_full[s], (it / kFuMgStages) & 1)) {
-                            failed = true;
-                            break;
-                        }
-                        ptx::tc_fence_after();
-                        const uint32_t b_base = arena_u32 + kFuPartOffset + s * kFuBoxBytes;
-                        for (int t = 0; t < im.ntile; ++t) {
-                            const uint32_t a_base = arena_u32 + (uint32_t)(t * im.nkb + kb) * kFuABytes;
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const uint64_t da = ptx::smem_desc_sw128(a_base + k * 32, 16, 1024);
-                                const uint64_t db = ptx::smem_desc_sw128(b_base + k * 2048, kFuBoxBytes, 1024);
-                                ptx::umma_bf16(d_tmem + (uint32_t)(t * 64), da, db, idesc, 1u);
-                            }
-                        }
-                        ptx::umma_commit(&sh->mg_empty[s]);
-                    }
-                    if (!failed) ptx::umma_commit(&sh->acc_full[as]);
+                    ptx::umma_commit(&sh->acc_full[as]);      // (at once when nothing is pruned: no UMMA was issued)
                 }
                 if (failed) {
                     sh->abort_flag = 1;
                     atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
                 }
             }
-        } else if (warp >= 4 && warp < 8 && im.ntile > 0) {
-            // ---- epilogue: TMEM -> bf16 -> this warp's staging rows -> coalesced stores of the kept rows ------
-            const int q = warp - 4;
-            const int out0 = sh->out0;
-            uint8_t *stg = arena + kFuStagingOffset + q * 32 * kFuStagePitch;
-            int pk[2], tokv[2];
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const int tr = t * kFuTileM + q * 32 + lane;
-                tokv[t] = im.tok_lo + tr;
-                pk[t] = (t < im.ntile && tr < im.ntok) ? __ldcg(kpos + im.t_begin + tokv[t]) : -1;
-                if (pk[t] >= 0) kept_idx[out0 + pk[t]] = tokv[t];
-            }
+        } else if (warp < kFuEpiWarps && im.ntile > 0) {
+            // ---- epilogue: warp (tile t = warp / 4, quarter q = warp % 4) owns rows 128 t + 32 q .. + 31 -------------
+            const int q = warp & 3, t = warp >> 2;
+            const int i0 = t * kFuTileM + q * 32;
+            const int i = i0 + lane;
+            const bool has_rows = t < im.ntile && i0 < im.Ml;
+            const uint32_t my_row = (uint32_t)((i >> 3) * 1024 + (i & 7) * 128);
             bool dead = false;
             for (int ct = 0; ct < nct; ++ct) {
-                const int as = ct % kFuAccStages;
-                bool ok = !dead && !sh->abort_flag && ptx::mbar_wait(&sh->acc_full[as], (ct / kFuAccStages) & 1);
+                const int s = ct % mstages, as = ct % kFuAccStages;
+                uint8_t *stage = arena + ring_off + s * mstage_bytes;
+                uint8_t *xrow = stage + my_row;              // this thread's row: T_k now, the output row below
+                // the stage first (it has been there for a while: the copies run ahead), and the row's eight
+                // 16-byte cells while the accumulator is waited for
+                bool ok = !dead && !sh->abort_flag && ptx::mbar_wait(&sh->mg_full[s], (ct / mstages) & 1);
+                uint4 xv[8];
+                if (ok && has_rows) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) xv[g] = *reinterpret_cast<const uint4 *>(xrow + ((g ^ (i & 7)) << 4));
+                }
+                ok = ok && ptx::mbar_wait(&sh->acc_full[as], (ct / kFuAccStages) & 1);
                 if (!__all_sync(0xffffffffu, ok)) {
                     if (!dead) {
                         sh->abort_flag = 1;
@@ -856,41 +1137,56 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
                     continue;
                 }
                 ptx::tc_fence_after();
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    // a warp whose 32 rows all lie past the CTA's tokens has nothing to convert or store
-                    if (t >= im.ntile || t * kFuTileM + q * 32 >= im.ntok) continue;
-#pragma unroll
-                    for (int c0 = 0; c0 < kFuNT; c0 += 32) {
-                        uint32_t r[32];
-                        ptx::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * 128 + t * 64 + c0), r);
+                if (has_rows) {
+                    // both halves of the accumulator row into registers, then the accumulator stage is free
+                    uint32_t r0[32], r1[32];
+                    if (im.B > 0) {
+                        ptx::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * 128 + t * 64), r0);
+                        ptx::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * 128 + t * 64 + 32), r1);
                         ptx::tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) r0[e] = r1[e] = 0u;
+                    }
+                    ptx::tc_fence_before();
+                    ptx::mbar_arrive(&sh->acc_empty[as]);
+                    __nv_bfloat16 *yrow0 = Y + (size_t)(out0 + im.row_lo + i0) * d + ct * kFuNT;
+                    // 32 columns at a time: add, round, back into the row's cells; then 4 lanes write a row's 64
+                    // bytes, 8 rows per instruction
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
+                            const __nv_bfloat162 *xh = reinterpret_cast<const __nv_bfloat162 *>(&xv[4 * h + g]);
                             __nv_bfloat162 o[4];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                o[e] = __floats2bfloat162_rn(__uint_as_float(r[8 * g + 2 * e]),
-                                                             __uint_as_float(r[8 * g + 2 * e + 1]));
-                            *reinterpret_cast<uint4 *>(stg + lane * kFuStagePitch + (c0 + 8 * g) * 2) =
-                                *reinterpret_cast<uint4 *>(o);
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 xf = __bfloat1622float2(xh[e]);
+                                const uint32_t a0 = h ? r1[8 * g + 2 * e] : r0[8 * g + 2 * e];
+                                const uint32_t a1 = h ? r1[8 * g + 2 * e + 1] : r0[8 * g + 2 * e + 1];
+                                o[e] = __floats2bfloat162_rn(xf.x + __uint_as_float(a0), xf.y + __uint_as_float(a1));
+                            }
+                            *reinterpret_cast<uint4 *>(xrow + (((4 * h + g) ^ (i & 7)) << 4)) = *reinterpret_cast<uint4 *>(o);
                         }
-                    }
-                    __syncwarp();
-                    // 8 lanes write one row's 128 bytes: 4 rows per instruction
+                        __syncwarp();
+                        uint4 yv[4];
 #pragma unroll
-                    for (int rr = 0; rr < 32; rr += 4) {
-                        const int row = rr + (lane >> 3);
-                        const int prow = __shfl_sync(0xffffffffu, pk[t], row);
-                        if (prow >= 0) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(stg + row * kFuStagePitch + (lane & 7) * 16);
-                            *reinterpret_cast<uint4 *>(Y + (size_t)(out0 + prow) * d + ct * kFuNT + (lane & 7) * 8) = v;
+                        for (int rr = 0; rr < 4; ++rr) {
+                            const int ir = i0 + 8 * rr + (lane >> 2);
+                            yv[rr] = *reinterpret_cast<const uint4 *>(stage + (ir >> 3) * 1024 + (ir & 7) * 128 +
+                                                                      (((4 * h + (lane & 3)) ^ (ir & 7)) << 4));
+                        }
+#pragma unroll
+                        for (int rr = 0; rr < 4; ++rr) {
+                            const int row = 8 * rr + (lane >> 2);
+                            if (i0 + row < im.Ml)
+                                *reinterpret_cast<uint4 *>(yrow0 + (size_t)row * d + (4 * h + (lane & 3)) * 8) = yv[rr];
                         }
                     }
-                    __syncwarp();
+                } else {
+                    ptx::mbar_arrive(&sh->acc_empty[as]);
                 }
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(&sh->acc_empty[as]);
+                ptx::mbar_arrive(&sh->mg_empty[s]);          // the stage's rows have been read (and written out)
             }
         }
         // every role is done with the image before the next one reuses the arena and the barriers
@@ -903,7 +1199,7 @@ stage2_fused_kernel(const __grid_constant__ CUtensorMap tmapXa,    // X, boxes o
     __syncthreads();
     // no CTA leaves while the other may still write into its shared memory
     ptx::cluster_sync_all();
-    if (warp == 1) {
+    if (warp == kFuMmaWarp) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, 512);
     }

@@ -79,6 +79,8 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
     L.scores_done = off;
     off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
+    L.sel_flag = off;
+    off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
     L.clear_bytes = off;
     L.norms = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
@@ -228,8 +230,11 @@ template <typename T>
 cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, const void *X,
                                  const int32_t *offsets, int batch, int total, const RatioParams &rp,
                                  const float *rho, char *ws, int32_t *out_offsets, int32_t *counts,
-                                 float *stats, float *norms_out, int32_t *order_out, int scan_here)
+                                 float *stats, float *norms_out, int32_t *order_out, int scan_here,
+                                 int attr_only = 0)
 {
+    // attr_only > 0: no launch; give the plan's instance of the kernel that much dynamic shared memory (the
+    // attribute belongs to the function: rtprune_plan sets it once, to what the device allows)
     constexpr int EPV = Elem<T>::kPerVec;
     const WsLayout &L = pl->ws;
     const int d = pl->d;
@@ -247,11 +252,7 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
 #define RTP_CASE(V)                                                                              \
     case V: {                                                                                    \
         auto k = stage1_kernel<T, V>;                                                            \
-        if (smem > 48 * 1024) {                                                                  \
-            cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                                 (int)smem);                                     \
-            if (e != cudaSuccess) return e;                                                      \
-        }                                                                                        \
+        if (attr_only) return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, attr_only); \
         cudaError_t e = launch_pdl(k, grid, dim3(kS1Threads), smem, st, 1u,                      \
             (const T *)X, offsets, batch, d, L.chunks, chunk_tokens, pl->max_tokens, total, rp, rho, \
             (float *)(ws + L.norms), (float *)(ws + (rp.criterion ? L.crit : L.norms)),          \
@@ -277,11 +278,19 @@ struct DevOut {
     float *merge_weight, *stats;
 };
 
+// The plan's SM count, shared-memory limits and function attributes are those of the device it was made on.
+bool on_plan_device(const rtprune_plan_t *plan)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == plan->device;
+}
+
 rtprune_status_t check_common(rtprune_plan_t *plan, const void *X, const int32_t *offsets,
                               int32_t batch, int64_t total, const rtprune_params_t *params,
                               void *workspace, size_t workspace_bytes)
 {
     if (!plan || !params) return RTPRUNE_ERR_INVALID_ARG;
+    if (!on_plan_device(plan)) return RTPRUNE_ERR_INVALID_ARG;
     if (batch < 0 || total < 0) return RTPRUNE_ERR_INVALID_ARG;
     if (batch > plan->max_batch || total > plan->max_total) return RTPRUNE_ERR_INVALID_ARG;
     if (total < batch) return RTPRUNE_ERR_INVALID_ARG;  // every image has at least one token
@@ -314,10 +323,26 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
     return RTPRUNE_OK;
 }
 
+constexpr bool kFusedStage1 = false;   // stage 1 inside the fused kernel (slower than the separate kernel as it stands)
+
+// The fused kernel takes the run's second stage: bf16 storage, scaling form, every possible tile fits.
+bool fused_stage2_ok(const rtprune_plan_t *plan, const rtprune_params_t *params)
+{
+    const int maxB = max_pruned(params, plan->max_tokens);
+    return plan->dtype == RTPRUNE_BF16 && maxB > 0 && plan->fused_clusters > 0 && !use_log_form(params) &&
+           fused_eligible(plan->d, plan->max_tokens, maxB);
+}
+// ... and the first stage too (ranking by the l2 norm, rows that fit its streaming ring).
+bool fused_whole_path(const rtprune_plan_t *plan, const rtprune_params_t *params)
+{
+    return kFusedStage1 && fused_stage2_ok(plan, params) && params->criterion == RTPRUNE_CRITERION_L2NORM &&
+           fused_stage1_eligible(plan->d);
+}
+
 template <typename T>
 rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void *X,
                                const int32_t *offsets, int32_t batch, int total,
-                               const rtprune_params_t *params, char *ws, const DevOut &o)
+                               const rtprune_params_t *params, char *ws, const DevOut &o, bool with_stage1 = false)
 {
     Checked c{plan};
     const WsLayout &L = plan->ws;
@@ -336,25 +361,21 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
 
     if constexpr (kTensor) {
         // One kernel for the whole second stage when every image the run can hold fits it
-        if (maxB > 0 && plan->fused_clusters > 0 && !use_log_form(params) && fused_eligible(plan->d, maxN, maxB)) {
-            CUtensorMap tmapXa, tmapXb, tmapXp;
-            if (!make_tmap_bf16(plan, &tmapXa, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2, kFuBK,
-                                kFuTileM) ||
-                !make_tmap_bf16(plan, &tmapXb, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2, 64, 64) ||
-                !make_tmap_bf16(plan, &tmapXp, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
-                                (uint64_t)plan->d * 2, 64, 64))
-                return RTPRUNE_ERR_CUDA;
+        if (fused_stage2_ok(plan, params)) {
             OtParams op{params->z, params->alpha, params->eps, params->iters, params->stop_at_fixed_point,
                         params->tol};
             const int clusters = std::min(batch, plan->fused_clusters);
-            if (!c.ok(launch_pdl(stage2_fused_kernel, dim3((unsigned)(2 * clusters)), dim3(kFuThreads),
-                                 (size_t)kFuSmemBytes, st, 2u, tmapXa, tmapXb, tmapXp, (const __nv_bfloat16 *)X, offsets,
-                                 plan->d, batch, (const int32_t *)o.counts, (const int32_t *)order,
-                                 (const int32_t *)(ws + L.kpos), (const float *)norms, (__nv_bfloat16 *)(ws + L.xp), maxN,
-                                 total, op, (__nv_bfloat16 *)o.Y, o.out_offsets, o.kept_idx, o.merged_idx,
-                                 o.merge_partner, o.merge_weight, o.stats, (WsHeader *)(ws + L.header))))
+            RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max,
+                           params->criterion};
+            auto kern = with_stage1 ? stage2_fused_kernel<true> : stage2_fused_kernel<false>;
+            if (!c.ok(launch_pdl(kern, dim3((unsigned)(2 * clusters)), dim3(kFuThreads),
+                                 (size_t)kFuSmemBytes, st, 2u, (const __nv_bfloat16 *)X, offsets, plan->d, batch,
+                                 (const int32_t *)o.counts, (const int32_t *)order, (const float *)norms, maxN, total, op,
+                                 (__nv_bfloat16 *)o.Y, o.out_offsets, o.kept_idx, o.merged_idx, o.merge_partner,
+                                 o.merge_weight, o.stats, (WsHeader *)(ws + L.header), rp,
+                                 params->rho, o.counts, (int *)(ws + L.sel_flag), plan->run)))
                 return RTPRUNE_ERR_CUDA;
-            launched(plan, st, "stage2_fused");
+            launched(plan, st, with_stage1 ? "fused" : "stage2_fused");
             return RTPRUNE_OK;
         }
     }
@@ -464,10 +485,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         const bool tall = !use_log_form(params) && !all_fast &&
                           sizeof(float) * (sinkhorn_tall_smem_floats(std::min(maxB, kTallMaxB), maxN) +
                                            kTallStageFloatsMax) <= tall_smem;
-        if (tall) {
-            if (!c.ok(cudaFuncSetAttribute(sinkhorn_tall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)tall_smem)))
-                return RTPRUNE_ERR_CUDA;
+        if (tall) {      // (rtprune_plan gave the kernel its shared memory)
             // 16 CTAs per image when all the images' clusters then still run at once, else 8
             // (a CTA owns a slice of at most 512 columns, one per thread: 8 CTAs cover every pitch, 4 cover
             // pitches of up to 2048 floats).  Batches whose clusters of 8 need several waves get clusters of 4
@@ -541,6 +559,10 @@ rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X
         return RTPRUNE_OK;
     }
     prof_begin(plan, st);
+    // One kernel for the whole path when every image the run can hold fits the fused kernel and stage 1 ranks by
+    // the l2 norm: the clusters stream their images themselves.
+    if (fused_whole_path(plan, params))
+        return launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o, true);
     // with bf16 storage and anything to prune, the kernel that copies the pruned rows also turns the counts
     // into out_offsets, so that stage 1 ends with the last image's selection
     const bool scan_later = plan->dtype == RTPRUNE_BF16 && max_pruned(params, plan->max_tokens) > 0;
@@ -658,12 +680,30 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     const long long cap = (long long)optin - 1024;
     if (want > cap) want = cap;
     p->sink_smem_bytes = (int)(want / 16 * 16);
+    // The attribute belongs to the function, not to the plan: every plan sets it to what the device allows,
+    // so that a plan made later for smaller images does not lower it under an earlier plan's launches.
     if (!c.ok(cudaFuncSetAttribute(sinkhorn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   p->sink_smem_bytes)) ||
+                                   (int)(cap / 16 * 16))) ||
         !c.ok(cudaFuncSetAttribute(sinkhorn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   p->sink_smem_bytes))) {
+                                   (int)(cap / 16 * 16)))) {
         delete p;
         return RTPRUNE_ERR_CUDA;
+    }
+    {
+        const int s1_cap = std::max(optin - 4096, 0);       // the kernel's static shared memory is under 4 KB
+        RatioParams rp0{};
+        const cudaError_t e1 =
+            dtype == RTPRUNE_BF16
+                ? launch_stage1_kernel<__nv_bfloat16>(p, nullptr, nullptr, nullptr, 1, 1, rp0, nullptr, nullptr, nullptr,
+                                                      nullptr, nullptr, nullptr, nullptr, 0, s1_cap)
+                : launch_stage1_kernel<float>(p, nullptr, nullptr, nullptr, 1, 1, rp0, nullptr, nullptr, nullptr, nullptr,
+                                              nullptr, nullptr, nullptr, 0, s1_cap);
+        if (!c.ok(e1) ||
+            sizeof(float) * stage1_smem_floats(d, max_tokens_per_image, dtype == RTPRUNE_BF16 ? 2 : 4) > (size_t)s1_cap) {
+            if (!p->last_cuda_error) p->last_cuda_error = (int)cudaErrorInvalidValue;
+            delete p;
+            return RTPRUNE_ERR_CUDA;
+        }
     }
     p->fast_smem_bytes = (int)(cap / 16 * 16);
     if (!c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -699,7 +739,9 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     // device runs at once is what a run's grid is capped at (its clusters then loop over the images).
     p->fused_clusters = 0;
     if (dtype == RTPRUNE_BF16 &&
-        cudaFuncSetAttribute(stage2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
+        cudaFuncSetAttribute(stage2_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
+            cudaSuccess &&
+        cudaFuncSetAttribute(stage2_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
             cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2);
@@ -713,7 +755,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, stage2_fused_kernel, &cfg) == cudaSuccess && nclusters > 0)
+        if (cudaOccupancyMaxActiveClusters(&nclusters, stage2_fused_kernel<false>, &cfg) == cudaSuccess && nclusters > 0)
             p->fused_clusters = nclusters;
     }
     (void)cudaGetLastError();
@@ -810,6 +852,7 @@ rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, 
                                        int32_t *order_out)
 {
     if (!plan || !params) return RTPRUNE_ERR_INVALID_ARG;
+    if (!on_plan_device(plan)) return RTPRUNE_ERR_INVALID_ARG;
     if (batch < 0 || total_tokens < 0 || batch > plan->max_batch || total_tokens > plan->max_total ||
         total_tokens < batch)
         return RTPRUNE_ERR_INVALID_ARG;
@@ -867,6 +910,7 @@ rtprune_status_t rtprune_run_host(rtprune_plan_t *plan, void *cuda_stream, const
                                   float *stats_host)
 {
     if (!plan || !params || !arena || ((uintptr_t)arena & 255u)) return RTPRUNE_ERR_INVALID_ARG;
+    if (!on_plan_device(plan)) return RTPRUNE_ERR_INVALID_ARG;
     if (batch < 0 || total_tokens < 0 || batch > plan->max_batch ||
         total_tokens > plan->max_total || total_tokens < batch)
         return RTPRUNE_ERR_INVALID_ARG;
