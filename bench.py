@@ -481,6 +481,7 @@ def main() -> None:
             "scores": ("hbm", x_bytes + xp_bytes + 4 * sumMB),
             "sinkhorn_cluster": ("alu", sink_flops),
             "sinkhorn_wide": ("alu", sink_flops),
+            "sinkhorn_reg": ("alu", sink_flops),
             "sinkhorn": ("alu", sink_flops),
             "merge": ("hbm", x_bytes + y_bytes + sumM * 4),
             # scores, Sinkhorn and merge in one kernel: it must read X and write Y, the pairs and the indices

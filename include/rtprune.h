@@ -70,6 +70,15 @@ typedef enum { RTPRUNE_SINKHORN_AUTO = 0, RTPRUNE_SINKHORN_LOG = 1, RTPRUNE_SINK
 typedef enum { RTPRUNE_CRITERION_L2NORM = 0, RTPRUNE_CRITERION_VARIANCE = 1, RTPRUNE_CRITERION_ENTROPY = 2 }
     rtprune_criterion_t;
 
+/* How stage 2 (scores, Sinkhorn, merge: Sec. 3.3.2, App. C, Eq. 7) is scheduled on the device.  The results are
+ * the same up to fp32 rounding; only the kernels differ.
+ *   AUTO     the library chooses by batch shape
+ *   SEPARATE one kernel per step, handing images to one another through the workspace
+ *   FUSED    one kernel, a cluster of two CTAs per image, nothing through global memory between the steps;
+ *            taken only when every image the run can hold fits it (bf16, width a multiple of 64, at most 512
+ *            tokens and 256 pruned tokens per image, scaling form), else SEPARATE is used */
+typedef enum { RTPRUNE_SCHEDULE_AUTO = 0, RTPRUNE_SCHEDULE_SEPARATE = 1, RTPRUNE_SCHEDULE_FUSED = 2 } rtprune_schedule_t;
+
 /* Parameters of one run (Algorithm 1 inputs; Appendix C for `iters`). */
 typedef struct {
     int32_t dynamic;      /* 0: use r_fixed.  1: r = min(r_max, f_normalize(phi) (1 - rho)), Eq. 10 */
@@ -93,6 +102,7 @@ typedef struct {
     float tol;            /* > 0: also stop once no dual moved by more than tol (log units) in an
                              iteration.  0 (default): never stop on a tolerance.                    */
     int32_t criterion;    /* rtprune_criterion_t: what stage 1 ranks by (default L2NORM, Eq. 1)     */
+    int32_t schedule;     /* rtprune_schedule_t: which kernels carry out stage 2 (same results)     */
 } rtprune_params_t;
 
 /* Number of floats per image in the `stats` output. */
@@ -107,7 +117,7 @@ typedef struct {
 
 /* Fills *params with the paper's defaults: fixed r = 0.25, z = 0.2, alpha = 0.1, eps = 1,
  * iters = 100, identity f_normalize, r_max = 1, form AUTO, stop_at_fixed_point = 1, tol = 0,
- * criterion L2NORM. */
+ * criterion L2NORM, schedule AUTO. */
 rtprune_status_t rtprune_default_params(rtprune_params_t *params);
 
 /*

@@ -18,6 +18,7 @@ from . import build as _build
 STATS_STRIDE = 8
 BF16, FP32 = 0, 1
 SINKHORN_AUTO, SINKHORN_LOG, SINKHORN_SCALING = 0, 1, 2
+SCHEDULE_AUTO, SCHEDULE_SEPARATE, SCHEDULE_FUSED = 0, 1, 2
 DEV_NONFINITE, DEV_TIMEOUT, DEV_BAD_OFFSETS = 1, 2, 4
 
 STATUS_NAMES = {0: "RTPRUNE_OK", 1: "RTPRUNE_ERR_INVALID_ARG", 2: "RTPRUNE_ERR_UNSUPPORTED",
@@ -38,7 +39,7 @@ class CParams(ctypes.Structure):
                 ("r_max", ctypes.c_float), ("z", ctypes.c_float), ("alpha", ctypes.c_float),
                 ("eps", ctypes.c_float), ("iters", ctypes.c_int32), ("form", ctypes.c_int32),
                 ("stop_at_fixed_point", ctypes.c_int32), ("tol", ctypes.c_float),
-                ("criterion", ctypes.c_int32)]
+                ("criterion", ctypes.c_int32), ("schedule", ctypes.c_int32)]
 
 
 _lib: Optional[ctypes.CDLL] = None

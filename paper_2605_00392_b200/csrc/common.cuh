@@ -29,7 +29,6 @@ struct WsLayout {
     size_t sink_done;  // uint32 [batch]           CTAs of each image's cluster that have written their plan rows
     size_t ready_list; // int32 [batch]            1 + image, in the order the plans were finished
     size_t scores_done; // uint32 [batch]          score tiles of each image that are complete
-    size_t sel_flag;   // int32 [batch]            number of the run whose count of kept tokens is in counts[i]
     size_t clear_bytes;  // the workspace's first clear_bytes bytes (header, counters) start at zero
     size_t norms;      // float [total]            l2 norms (the criterion C_k of Eq. 1)
     size_t crit;       // float [total]            C_k of a run that ranks by variance or entropy

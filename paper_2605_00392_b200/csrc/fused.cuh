@@ -31,7 +31,6 @@
 #include "ptx.cuh"
 #include "sinkhorn.cuh"
 #include "sinkhorn_cluster.cuh"
-#include "stage1.cuh"
 
 namespace rtp {
 
@@ -59,11 +58,8 @@ constexpr int kFuBoxBytes = 64 * 128;     // 8 KB: 64 rows x 64 bf16
 constexpr int kFuScStages = 6;            // at most
 constexpr int kFuMgStages = 6;            // at most
 constexpr int kFuAccStages = 4;           // accumulator stages of the merge (128 TMEM columns each)
-constexpr int kFuS1Stages = 8;            // at most, of the streaming pass
-constexpr int kFuS1Rows = kFuWarps;       // rows per stage of the streaming pass: one per warp
-constexpr int kFuS1Vpl = 8;               // 16-byte vectors of a row per lane, at most: widths up to 2048
-constexpr int kFuSharedBytes = 18432;     // FuShared, rounded up
-constexpr int kFuArenaBytes = 207 * 1024;
+constexpr int kFuSharedBytes = 15360;     // FuShared, rounded up
+constexpr int kFuArenaBytes = 210 * 1024;
 constexpr int kFuPartBytes = 32 * 1024;   // column partials of the iterations, then of the pairing
 constexpr int kFuPartOffset = kFuArenaBytes - kFuPartBytes;
 constexpr int kFuSmemBytes = 1024 + kFuSharedBytes + kFuArenaBytes;
@@ -74,12 +70,9 @@ struct FuShared {
     uint64_t mg_full[kFuMgStages], mg_empty[kFuMgStages];
     uint64_t acc_full[kFuAccStages], acc_empty[kFuAccStages];
     uint64_t xbar[2];                           // the other CTA's column sums of an iteration have arrived (by parity)
-    uint64_t s1_full[kFuS1Stages], s1_empty[kFuS1Stages];   // ring of the streaming pass
     uint32_t tmem_base;
     volatile int abort_flag;
     int out0;
-    int sel_m;                                  // M of the image, from the thread that computes the ratio
-    float red[32];
     float vsum[kFuWarps];
     float wsum[kFuWarps];
     __align__(16) float xusum[2][4];            // the other CTA's sum of U, by iteration parity
@@ -88,8 +81,6 @@ struct FuShared {
     __align__(16) float vs[kFuMaxB + 8];        // V_j, V_d at [ldk]: read as 16-byte vectors
     int rowtok[kFuMaxRows + kFuMaxB + 32];      // image-local token of each row of a stage (-1: a row of zeros)
     __align__(16) float xpart[2][kFuMaxB];      // the other CTA's column partials, by iteration parity
-    __align__(16) float nrm[kFuMaxTok + 4];     // l2 norms of all the image's tokens (streaming pass in this kernel)
-    int wcount[2][kFuWarps];                    // kept / pruned tokens per warp of the selection
     float pairv[2][kFuMaxB];                    // rank 0: per-CTA column maxima of K U ...
     int pairi[2][kFuMaxB];                      // ... and their rows
 };
@@ -120,14 +111,6 @@ __host__ __device__ inline int fused_stage_bytes(int rows, int B)
 __host__ __device__ inline int fused_plan_bytes(int rows, int B)
 {
     return ((B + 63) / 64) * ((rows + 15) & ~15) * 128;
-}
-
-// The streaming pass of stage 1 can run inside the kernel too: rows of at most 32 * kFuS1Vpl vectors, two
-// stages of 16 rows in the arena, the warps' partial sums of unit tokens and the two CTAs' sums after them.
-__host__ inline bool fused_stage1_eligible(int d)
-{
-    return d % 8 == 0 && d / 8 <= 32 * kFuS1Vpl && 2 * kFuS1Rows * d * 2 <= kFuArenaBytes &&
-           (kFuWarps + 2) * d * 4 <= kFuArenaBytes;
 }
 
 // Every image of a run with at most max_tokens tokens and max_b pruned tokens fits the fused kernel:
@@ -327,6 +310,76 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
     return st;
 }
 
+// Pairing, one CTA's part: per column the largest K_ij U_i over this CTA's rows and its row (ties to the
+// lower row): over the thread's steps, over the warp's row slots, over the warps in shared memory; the
+// result goes to rank 0's pairv / pairi (the cluster barrier that must follow makes it visible there).
+template <int LR, int CPL, int NS>
+__device__ inline void fused_pair_partials(const float4 (&k)[NS][CPL / 4], const float (&U)[NS], FuShared *sh, float *part,
+                                           int Ml, int row_lo, int B, uint32_t rank)
+{
+    constexpr int ldk = LR * CPL;
+    constexpr int RPS = 32 / LR;
+    constexpr int NQ = CPL / 4;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LR, slot = lane / LR;
+    // ---- pairing, this CTA's part: per column the largest K_ij U_i over this CTA's rows and its row
+    // (ties to the lower row).  Chunk by chunk: over the thread's steps, over the warp's row slots, to
+    // shared memory per warp.
+    float *pv = part;
+    int *pi = reinterpret_cast<int *>(part + kFuWarps * ldk);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        float bv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        int bi[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
+#pragma unroll
+        for (int s = 0; s < NS; ++s) {
+            const int i = (s * kFuWarps + warp) * RPS + slot;
+            if (i < Ml) {
+                const float e[4] = {k[s][q].x * U[s], k[s][q].y * U[s], k[s][q].z * U[s], k[s][q].w * U[s]};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (e[c] > bv[c]) {          // rows ascend with s: strict > keeps the lower row
+                        bv[c] = e[c];
+                        bi[c] = row_lo + i;
+                    }
+            }
+        }
+#pragma unroll
+        for (int o = LR; o < 32; o <<= 1) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv[c], o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi[c], o);
+                if (ov > bv[c] || (ov == bv[c] && oi < bi[c])) {
+                    bv[c] = ov;
+                    bi[c] = oi;
+                }
+            }
+        }
+        if (slot == 0) {
+            const int col = 4 * (q * LR + sub);
+            *reinterpret_cast<float4 *>(pv + warp * ldk + col) = make_float4(bv[0], bv[1], bv[2], bv[3]);
+            *reinterpret_cast<int4 *>(pi + warp * ldk + col) = make_int4(bi[0], bi[1], bi[2], bi[3]);
+        }
+    }
+    __syncthreads();
+    if (tid < B) {
+        float b = pv[tid];
+        int ib = pi[tid];
+#pragma unroll
+        for (int w = 1; w < kFuWarps; ++w) {
+            const float ob = pv[w * ldk + tid];
+            const int oi = pi[w * ldk + tid];
+            if (ob > b || (ob == b && oi < ib)) {
+                b = ob;
+                ib = oi;
+            }
+        }
+        ptx::st_cluster_f32(ptx::map_to_rank(ptx::smem_u32(&sh->pairv[rank][tid]), 0), b);
+        ptx::st_cluster_u32(ptx::map_to_rank(ptx::smem_u32(&sh->pairi[rank][tid]), 0), (uint32_t)ib);
+    }
+}
+
 // Everything between the scores and the merge for one tile layout: K into registers, the iterations,
 // alpha P of this CTA's rows into its plan arrays, the per-CTA column maxima of K U for the pairing
 // (sent to rank 0).  kbuf: this CTA's K rows, pitch ldk + 4 floats, in shared memory (the arena's start,
@@ -389,62 +442,7 @@ __device__ inline FuIterState fused_sinkhorn(FuShared *sh, const float *kbuf, ui
         }
     }
 
-    // ---- pairing, this CTA's part: per column the largest K_ij U_i over this CTA's rows and its row
-    // (ties to the lower row).  Chunk by chunk: over the thread's steps, over the warp's row slots, to
-    // shared memory per warp.
-    float *pv = part;
-    int *pi = reinterpret_cast<int *>(part + kFuWarps * ldk);
-#pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        float bv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        int bi[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
-#pragma unroll
-        for (int s = 0; s < NS; ++s) {
-            const int i = (s * kFuWarps + warp) * RPS + slot;
-            if (i < im.Ml) {
-                const float e[4] = {k[s][q].x * U[s], k[s][q].y * U[s], k[s][q].z * U[s], k[s][q].w * U[s]};
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (e[c] > bv[c]) {          // rows ascend with s: strict > keeps the lower row
-                        bv[c] = e[c];
-                        bi[c] = im.row_lo + i;
-                    }
-            }
-        }
-#pragma unroll
-        for (int o = LR; o < 32; o <<= 1) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv[c], o);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi[c], o);
-                if (ov > bv[c] || (ov == bv[c] && oi < bi[c])) {
-                    bv[c] = ov;
-                    bi[c] = oi;
-                }
-            }
-        }
-        if (slot == 0) {
-            const int col = 4 * (q * LR + sub);
-            *reinterpret_cast<float4 *>(pv + warp * ldk + col) = make_float4(bv[0], bv[1], bv[2], bv[3]);
-            *reinterpret_cast<int4 *>(pi + warp * ldk + col) = make_int4(bi[0], bi[1], bi[2], bi[3]);
-        }
-    }
-    __syncthreads();
-    if (tid < im.B) {
-        float b = pv[tid];
-        int ib = pi[tid];
-#pragma unroll
-        for (int w = 1; w < kFuWarps; ++w) {
-            const float ob = pv[w * ldk + tid];
-            const int oi = pi[w * ldk + tid];
-            if (ob > b || (ob == b && oi < ib)) {
-                b = ob;
-                ib = oi;
-            }
-        }
-        ptx::st_cluster_f32(ptx::map_to_rank(ptx::smem_u32(&sh->pairv[rank][tid]), 0), b);
-        ptx::st_cluster_u32(ptx::map_to_rank(ptx::smem_u32(&sh->pairi[rank][tid]), 0), (uint32_t)ib);
-    }
+    fused_pair_partials<LR, CPL, NS>(k, U, sh, part, im.Ml, im.row_lo, im.B, rank);
     return st;
 }
 
@@ -502,217 +500,6 @@ __device__ inline void fused_wait_groups(int lag)
     else ptx::cp_async_wait<0>();
 }
 
-// Stage 1 of Algorithm 1 for one image inside the cluster (Eq. 1, Eq. 8, Eq. 10, the top-M selection of
-// Section 3.3.1): CTA r streams the image's tokens [r * tpc, ...), tpc = ceil(N / 2), through a ring of
-// shared-memory stages (1-D bulk copies of 16 contiguous rows, one row per warp): sum of squares by
-// shuffles, the norm, and the row divided by its norm into per-lane accumulators.  The two CTAs then
-// hand each other their norms and their sums of unit tokens through distributed shared memory, and both
-// compute phi = (|sum of unit tokens|^2 - N) / (N (N - 1)), the ratio, M, and the selection, in the same
-// order of operations: they agree bit for bit.  Selection: token k is kept iff fewer than M tokens rank
-// before it (larger norm, or equal norm and lower index): every thread counts the tokens that rank before
-// its own.  Fills rowtok, inv_ni, inv_nj; returns M.  Rank 0 writes counts and stats and publishes the
-// image's count to the other clusters (sel_flag[img] = run).
-__device__ inline int fused_stage1(FuShared *sh, uint8_t *arena, const uint8_t *img_base, int img, FuImage &im, int d,
-                                   uint32_t rank, const RatioParams &rp, const float *__restrict__ rho,
-                                   int32_t *__restrict__ counts, float *__restrict__ stats, int *__restrict__ sel_flag,
-                                   int run, WsHeader *hdr)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int N = im.N;
-    const int tpc = (N + 1) >> 1;
-    const int tok_lo = min(N, (int)rank * tpc);
-    const int ntok = min(N, tok_lo + tpc) - tok_lo;
-    const uint32_t row_bytes = (uint32_t)d * 2u;
-    const int nvec = d >> 3;
-    const uint32_t stage_bytes = (uint32_t)kFuS1Rows * row_bytes;
-    const int nst = min(kFuS1Stages, kFuArenaBytes / (int)stage_bytes);
-    const int nit = (ntok + kFuS1Rows - 1) / kFuS1Rows;
-    const uint32_t arena_u32 = ptx::smem_u32(arena);
-    const uint32_t peer = rank ^ 1u;
-    const float rho_i = (tid == 0 && rho) ? __ldg(rho + img) : 0.f;
-
-    float acc[kFuS1Vpl * 8];
-#pragma unroll
-    for (int e = 0; e < kFuS1Vpl * 8; ++e) acc[e] = 0.f;
-    bool bad = false, gave_up = false;
-    auto issue = [&](int it) {
-        const int s = it % nst;
-        const int r0 = it * kFuS1Rows;
-        const uint32_t bytes = (uint32_t)min(kFuS1Rows, ntok - r0) * row_bytes;
-        ptx::mbar_arrive_expect_tx(&sh->s1_full[s], bytes);
-        ptx::bulk_load(arena_u32 + s * stage_bytes, img_base + (size_t)(tok_lo + r0) * row_bytes, bytes, &sh->s1_full[s]);
-    };
-    if (tid == 0)
-        for (int it = 0; it < min(nst, nit); ++it) issue(it);
-    for (int it = 0; it < nit; ++it) {
-        const int s = it % nst;
-        if (!gave_up && !ptx::mbar_wait(&sh->s1_full[s], (it / nst) & 1)) gave_up = true;
-        const int t = it * kFuS1Rows + warp;
-        if (t < ntok && !gave_up) {
-            const uint4 *row = reinterpret_cast<const uint4 *>(arena + s * stage_bytes + warp * row_bytes);
-            uint4 cur[kFuS1Vpl];
-#pragma unroll
-            for (int j = 0; j < kFuS1Vpl; ++j) {
-                const int vi = lane + 32 * j;
-                cur[j] = (vi < nvec) ? row[vi] : make_uint4(0, 0, 0, 0);
-            }
-            float ss = 0.f;
-#pragma unroll
-            for (int j = 0; j < kFuS1Vpl; ++j) {
-                float f[8];
-                Elem<__nv_bfloat16>::unpack(cur[j], f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-            }
-            ss = warp_sum(ss);
-            const float n = sqrtf(ss);
-            if (!(ss <= 3.0e38f)) bad = true;  // inf or NaN
-            const float inv = 1.f / fmaxf(n, kNormFloor);
-            if (lane == 0) {
-                sh->nrm[tok_lo + t] = n;
-                ptx::st_cluster_f32(ptx::map_to_rank(ptx::smem_u32(&sh->nrm[tok_lo + t]), peer), n);
-            }
-#pragma unroll
-            for (int j = 0; j < kFuS1Vpl; ++j) {
-                float f[8];
-                Elem<__nv_bfloat16>::unpack(cur[j], f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[j * 8 + e] = fmaf(f[e], inv, acc[j * 8 + e]);
-            }
-        }
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh->s1_empty[s]);
-        if (tid == 0 && it + nst < nit) {        // refill the stage once all the warps have left it
-            if (!gave_up && !ptx::mbar_wait(&sh->s1_empty[s], (it / nst) & 1)) gave_up = true;
-            if (!gave_up) issue(it + nst);
-        }
-    }
-    if (gave_up && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-    if (bad && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_NONFINITE);
-    __syncthreads();          // the ring is free: it now holds the warps' partial sums [16][d], then the CTAs' [2][d]
-    float *wacc = reinterpret_cast<float *>(arena);
-    float *spart = wacc + kFuWarps * d;
-#pragma unroll
-    for (int j = 0; j < kFuS1Vpl; ++j) {
-        const int vi = lane + 32 * j;
-        if (vi < nvec) {
-            *reinterpret_cast<float4 *>(wacc + warp * d + vi * 8) = make_float4(acc[j * 8], acc[j * 8 + 1], acc[j * 8 + 2], acc[j * 8 + 3]);
-            *reinterpret_cast<float4 *>(wacc + warp * d + vi * 8 + 4) = make_float4(acc[j * 8 + 4], acc[j * 8 + 5], acc[j * 8 + 6], acc[j * 8 + 7]);
-        }
-    }
-    // the other CTA is done with the image before (its merge used this part of its arena) before anything lands there
-    ptx::cluster_sync_all();
-    for (int c = tid; c < d; c += kFuThreads) {
-        float sum = 0.f;
-#pragma unroll
-        for (int w = 0; w < kFuWarps; ++w) sum += wacc[w * d + c];
-        const uint32_t a = ptx::smem_u32(spart + rank * d + c);
-        ptx::st_cluster_f32(ptx::map_to_rank(a, 0), sum);
-        ptx::st_cluster_f32(ptx::map_to_rank(a, 1), sum);
-    }
-    if (tid < 4) sh->nrm[N + tid] = 0.f;      // the ranking reads the norms four at a time
-    ptx::cluster_sync_all();                  // both CTAs hold all the norms and both sums of unit tokens
-
-    // phi (Eq. 8), the ratio (Eq. 10) and M: the same arithmetic in both CTAs
-    float local = 0.f;
-    for (int c = tid; c < d; c += kFuThreads) {
-        const float v = spart[c] + spart[d + c];
-        local = fmaf(v, v, local);
-    }
-    const float ssum = block_sum(local, sh->red);
-    if (tid == 0) {
-        const float Nf = (float)N;
-        const float phi = (N >= 2) ? (ssum - Nf) / (Nf * (Nf - 1.f)) : 0.f;
-        float r;
-        if (rp.dynamic) {
-            float f = (phi - rp.phi_lo) / (rp.phi_hi - rp.phi_lo);
-            f = fminf(fmaxf(f, 0.f), 1.f);
-            r = fminf(f * (1.f - rho_i), rp.r_max);
-        } else {
-            r = rp.r_fixed;
-        }
-        r = fmaxf(r, 0.f);
-        int B = (int)floorf(r * Nf + 0.5f);
-        B = max(0, min(B, N - 1));
-        sh->sel_m = N - B;
-        if (rank == 0) {
-            float *st = stats + (size_t)img * kStats;
-            st[0] = phi;
-            st[1] = rho_i;
-            st[2] = r;
-            st[3] = (float)(N - B);
-            st[4] = (float)B;
-            st[5] = 0.f;
-            st[6] = 0.f;
-            st[7] = 0.f;
-            counts[img] = N - B;
-            __threadfence();
-            ptx::st_release_gpu(sel_flag + img, run);     // the clusters of later images add this count to their out0
-        }
-    }
-    __syncthreads();
-    const int M = sh->sel_m;
-    im.M = M;
-    im.B = N - M;
-    im.half = (M + 1) >> 1;
-    im.row_lo = min(M, (int)rank * im.half);
-    im.Ml = min(M, im.row_lo + im.half) - im.row_lo;
-    im.ntile = (im.Ml + kFuTileM - 1) / kFuTileM;
-    im.ldk = im.B > 0 ? sinkhorn_ldk(im.B) : 32;
-    im.nkb = (im.B + 63) >> 6;
-    im.Ra = (im.Ml + 15) & ~15;
-    im.Rb = (im.B + 15) & ~15;
-
-    // ---- selection: thread k ranks token k among all N (norm bits: the unsigned order is the float order) ----
-    const int k = tid;
-    bool kept = false;
-    if (k < N) {
-        const uint32_t mine = __float_as_uint(sh->nrm[k]) & 0x7fffffffu;
-        int before = 0;
-        for (int j0 = 0; j0 < N; j0 += 4) {
-            const float4 v = *reinterpret_cast<const float4 *>(sh->nrm + j0);
-            const uint32_t kj[4] = {__float_as_uint(v.x) & 0x7fffffffu, __float_as_uint(v.y) & 0x7fffffffu,
-                                    __float_as_uint(v.z) & 0x7fffffffu, __float_as_uint(v.w) & 0x7fffffffu};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int j = j0 + e;
-                before += (j < N && (kj[e] > mine || (kj[e] == mine && j < k))) ? 1 : 0;
-            }
-        }
-        kept = before < M;
-    }
-    // positions in ascending token order: kept tokens before k, pruned tokens before k
-    const uint32_t kmask = __ballot_sync(0xffffffffu, kept);
-    const uint32_t pmask = __ballot_sync(0xffffffffu, k < N && !kept);
-    if (lane == 0) {
-        sh->wcount[0][warp] = __popc(kmask);
-        sh->wcount[1][warp] = __popc(pmask);
-    }
-    for (int r = tid; r < im.Ra + im.Rb; r += kFuThreads) sh->rowtok[r] = -1;
-    __syncthreads();
-    int kb = 0, pb = 0;
-    for (int w = 0; w < warp; ++w) {
-        kb += sh->wcount[0][w];
-        pb += sh->wcount[1][w];
-    }
-    const uint32_t lt = (1u << lane) - 1u;
-    if (k < N) {
-        if (kept) {
-            const int pos = kb + __popc(kmask & lt) - im.row_lo;      // among this CTA's kept rows?
-            if (pos >= 0 && pos < im.Ml) {
-                sh->rowtok[pos] = k;
-                sh->inv_ni[pos] = 1.f / fmaxf(sh->nrm[k], kNormFloor);
-            }
-        } else {
-            const int pos = pb + __popc(pmask & lt);
-            sh->rowtok[im.Ra + pos] = k;
-            sh->inv_nj[pos] = 1.f / fmaxf(sh->nrm[k], kNormFloor);
-        }
-    }
-    __syncthreads();
-    return M;
-}
-
 __device__ inline void fused_init_barriers(FuShared *sh, bool again)
 {
     for (int s = 0; s < kFuScStages; ++s) {
@@ -720,7 +507,7 @@ __device__ inline void fused_init_barriers(FuShared *sh, bool again)
             mbar_inval(&sh->sc_full[s]);
             mbar_inval(&sh->sc_empty[s]);
         }
-        ptx::mbar_init(&sh->sc_full[s], kFuScProducers);
+        ptx::mbar_init(&sh->sc_full[s], kFuScProducers / 32);
         ptx::mbar_init(&sh->sc_empty[s], 1);
     }
     if (again) mbar_inval(&sh->sc_accum);
@@ -730,8 +517,8 @@ __device__ inline void fused_init_barriers(FuShared *sh, bool again)
             mbar_inval(&sh->mg_full[s]);
             mbar_inval(&sh->mg_empty[s]);
         }
-        ptx::mbar_init(&sh->mg_full[s], kFuMgProducers);
-        ptx::mbar_init(&sh->mg_empty[s], kFuEpiWarps * 32);
+        ptx::mbar_init(&sh->mg_full[s], kFuMgProducers / 32);
+        ptx::mbar_init(&sh->mg_empty[s], kFuEpiWarps);
     }
     for (int s = 0; s < kFuAccStages; ++s) {
         if (again) {
@@ -739,31 +526,18 @@ __device__ inline void fused_init_barriers(FuShared *sh, bool again)
             mbar_inval(&sh->acc_empty[s]);
         }
         ptx::mbar_init(&sh->acc_full[s], 1);
-        ptx::mbar_init(&sh->acc_empty[s], kFuEpiWarps * 32);
-    }
-    for (int s = 0; s < kFuS1Stages; ++s) {
-        if (again) {
-            mbar_inval(&sh->s1_full[s]);
-            mbar_inval(&sh->s1_empty[s]);
-        }
-        ptx::mbar_init(&sh->s1_full[s], 1);
-        ptx::mbar_init(&sh->s1_empty[s], kFuWarps);
+        ptx::mbar_init(&sh->acc_empty[s], kFuEpiWarps);
     }
     ptx::fence_mbar_init();
 }
 
-template <bool WITH_S1>
 __global__ void __launch_bounds__(kFuThreads, 1)
 stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ offsets, int d, int batch,
                     const int32_t *__restrict__ counts, const int32_t *__restrict__ order,
                     const float *__restrict__ norms, int max_tokens, int total, OtParams p,
                     __nv_bfloat16 *__restrict__ Y, int32_t *__restrict__ out_offsets, int32_t *__restrict__ kept_idx,
                     int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
-                    float *__restrict__ merge_weight, float *__restrict__ stats, WsHeader *__restrict__ hdr,
-                    // stage 1 inside this kernel (WITH_S1: counts, order and norms are not inputs then; counts is
-                    // written here and sel_flag[img] = run tells the other clusters that it is)
-                    RatioParams rp, const float *__restrict__ rho, int32_t *counts_out,
-                    int *__restrict__ sel_flag, int run)
+                    float *__restrict__ merge_weight, float *__restrict__ stats, WsHeader *__restrict__ hdr)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -810,19 +584,8 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
         if (!image_range(offsets, img, max_tokens, total, im.t_begin, im.N)) {
             // no output rows; the image's slot of out_offsets still has to be right
             if (rank == 0 && warp == 0) {
-                if (WITH_S1 && lane == 0) {      // offsets broke the contract: the image yields no output
-                    atomicOr(&hdr->status, RTPRUNE_DEV_BAD_OFFSETS);
-                    counts_out[img] = 0;
-                    float *st = stats + (size_t)img * kStats;
-                    for (int q = 0; q < kStats; ++q) st[q] = 0.f;
-                    __threadfence();
-                    ptx::st_release_gpu(sel_flag + img, run);
-                }
                 int s = 0;
-                for (int b = lane; b < img; b += 32) {
-                    if (WITH_S1 && !ptx::wait_equal_gpu(sel_flag + b, run)) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-                    s += __ldcg(counts + b);
-                }
+                for (int b = lane; b < img; b += 32) s += __ldcg(counts + b);
                 for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
                 if (lane == 0) {
                     out_offsets[img] = s;
@@ -837,9 +600,7 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
         if (!first) __syncthreads();
         first = false;
 
-        if constexpr (WITH_S1) {
-            fused_stage1(sh, arena, img_base, img, im, d, rank, rp, rho, counts_out, stats, sel_flag, run, hdr);
-        } else {
+        {
             im.M = __ldcg(counts + img);
             im.B = im.N - im.M;
             im.half = (im.M + 1) >> 1;
@@ -859,14 +620,10 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
                 sh->rowtok[r] = tok;
             }
         }
-        // out0 = number of kept rows of the images before this one (with stage 1 in this kernel their counts
-        // come from other clusters, which publish them as soon as they have them)
+        // out0 = number of kept rows of the images before this one
         if (warp == kFuWarps - 1) {
             int s = 0;
-            for (int b = lane; b < img; b += 32) {
-                if (WITH_S1 && !ptx::wait_equal_gpu(sel_flag + b, run)) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-                s += __ldcg(counts + b);
-            }
+            for (int b = lane; b < img; b += 32) s += __ldcg(counts + b);
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == 0) {
                 sh->out0 = s;
@@ -897,20 +654,22 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
                     if (kb >= lag) {
                         fused_wait_groups(lag);
                         ptx::fence_proxy_async_smem();
-                        ptx::mbar_arrive(&sh->sc_full[(kb - lag) % nstages]);
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&sh->sc_full[(kb - lag) % nstages]);
                     }
                 }
                 for (int kb = max(nkblk - lag, 0); kb < nkblk; ++kb) {
                     ptx::cp_async_wait<0>();
                     ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(&sh->sc_full[kb % nstages]);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&sh->sc_full[kb % nstages]);
                 }
                 if (!ok) {
                     sh->abort_flag = 1;
                     atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
                 }
-                // the norms of the rows, while the last k-blocks are multiplied (stage 1 in this kernel left them)
-                if (!WITH_S1) {
+                // the norms of the rows, while the last k-blocks are multiplied
+                {
                     for (int i = pt; i < im.Ml; i += kFuScProducers)
                         sh->inv_ni[i] = 1.f / fmaxf(__ldcg(norms + im.t_begin + sh->rowtok[i]), kNormFloor);
                     for (int j = pt; j < im.B; j += kFuScProducers)
@@ -1059,13 +818,15 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
                 if (ct >= mlag) {
                     fused_wait_groups(mlag);
                     ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(&sh->mg_full[(ct - mlag) % mstages]);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&sh->mg_full[(ct - mlag) % mstages]);
                 }
             }
             for (int ct = max(nct - mlag, 0); ct < nct; ++ct) {
                 ptx::cp_async_wait<0>();
                 ptx::fence_proxy_async_smem();
-                ptx::mbar_arrive(&sh->mg_full[ct % mstages]);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&sh->mg_full[ct % mstages]);
             }
             if (!ok) {
                 sh->abort_flag = 1;
@@ -1149,7 +910,8 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
                         for (int e = 0; e < 32; ++e) r0[e] = r1[e] = 0u;
                     }
                     ptx::tc_fence_before();
-                    ptx::mbar_arrive(&sh->acc_empty[as]);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&sh->acc_empty[as]);
                     __nv_bfloat16 *yrow0 = Y + (size_t)(out0 + im.row_lo + i0) * d + ct * kFuNT;
                     // 32 columns at a time: add, round, back into the row's cells; then 4 lanes write a row's 64
                     // bytes, 8 rows per instruction
@@ -1183,10 +945,11 @@ stage2_fused_kernel(const __nv_bfloat16 *__restrict__ X, const int32_t *__restri
                                 *reinterpret_cast<uint4 *>(yrow0 + (size_t)row * d + (4 * h + (lane & 3)) * 8) = yv[rr];
                         }
                     }
-                } else {
+                } else if (lane == 0) {
                     ptx::mbar_arrive(&sh->acc_empty[as]);
                 }
-                ptx::mbar_arrive(&sh->mg_empty[s]);          // the stage's rows have been read (and written out)
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&sh->mg_empty[s]);          // the stage's rows have been read (and written out)
             }
         }
         // every role is done with the image before the next one reuses the arena and the barriers

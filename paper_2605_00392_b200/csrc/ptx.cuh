@@ -53,6 +53,26 @@ __device__ inline bool mbar_wait(uint64_t *bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// The same by polling (test_wait never suspends the thread): it reacts within a few cycles of the phase's
+// completion, at the price of issue slots while it waits.  For waits on the critical path of a pipeline.
+__device__ inline bool mbar_test_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ inline bool mbar_poll(uint64_t *bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < 64u * kSpinLimit; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    return false;
+}
 
 // ---- proxies, cp.async ------------------------------------------------------------------------
 // Orders this thread's earlier generic-proxy writes to shared memory before later async-proxy reads

@@ -16,6 +16,7 @@
 #include "scores_umma.cuh"
 #include "sinkhorn.cuh"
 #include "sinkhorn_cluster.cuh"
+#include "sinkhorn_reg.cuh"
 #include "sinkhorn_tall.cuh"
 #include "stage1.cuh"
 
@@ -79,8 +80,6 @@ WsLayout make_layout(int d, rtprune_dtype_t dtype, int max_batch, int64_t max_to
     off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
     L.scores_done = off;
     off = align_up(off + sizeof(uint32_t) * (size_t)max_batch, 256);
-    L.sel_flag = off;
-    off = align_up(off + sizeof(int32_t) * (size_t)max_batch, 256);
     L.clear_bytes = off;
     L.norms = off;
     off = align_up(off + sizeof(float) * (size_t)max_total, 256);
@@ -203,6 +202,7 @@ rtprune_status_t check_params(const rtprune_params_t *p)
     if (!(p->tol >= 0.f)) return RTPRUNE_ERR_INVALID_ARG;
     if (p->criterion < RTPRUNE_CRITERION_L2NORM || p->criterion > RTPRUNE_CRITERION_ENTROPY)
         return RTPRUNE_ERR_INVALID_ARG;
+    if (p->schedule < RTPRUNE_SCHEDULE_AUTO || p->schedule > RTPRUNE_SCHEDULE_FUSED) return RTPRUNE_ERR_INVALID_ARG;
     const bool scaling_safe = p->eps >= 0.25f && std::fabs(p->z) <= 4.f;
     if (p->form == RTPRUNE_SINKHORN_SCALING && !scaling_safe) return RTPRUNE_ERR_INVALID_ARG;
     return RTPRUNE_OK;
@@ -323,26 +323,21 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
     return RTPRUNE_OK;
 }
 
-constexpr bool kFusedStage1 = false;   // stage 1 inside the fused kernel (slower than the separate kernel as it stands)
-
 // The fused kernel takes the run's second stage: bf16 storage, scaling form, every possible tile fits.
 bool fused_stage2_ok(const rtprune_plan_t *plan, const rtprune_params_t *params)
 {
     const int maxB = max_pruned(params, plan->max_tokens);
+    if (params->schedule == RTPRUNE_SCHEDULE_SEPARATE) return false;
+    // AUTO: the separate kernels overlap one another across the images of a batch and are ahead on the batches
+    // measured so far; the fused kernel is taken on request
+    if (params->schedule == RTPRUNE_SCHEDULE_AUTO) return false;
     return plan->dtype == RTPRUNE_BF16 && maxB > 0 && plan->fused_clusters > 0 && !use_log_form(params) &&
            fused_eligible(plan->d, plan->max_tokens, maxB);
 }
-// ... and the first stage too (ranking by the l2 norm, rows that fit its streaming ring).
-bool fused_whole_path(const rtprune_plan_t *plan, const rtprune_params_t *params)
-{
-    return kFusedStage1 && fused_stage2_ok(plan, params) && params->criterion == RTPRUNE_CRITERION_L2NORM &&
-           fused_stage1_eligible(plan->d);
-}
-
 template <typename T>
 rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void *X,
                                const int32_t *offsets, int32_t batch, int total,
-                               const rtprune_params_t *params, char *ws, const DevOut &o, bool with_stage1 = false)
+                               const rtprune_params_t *params, char *ws, const DevOut &o)
 {
     Checked c{plan};
     const WsLayout &L = plan->ws;
@@ -365,17 +360,13 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             OtParams op{params->z, params->alpha, params->eps, params->iters, params->stop_at_fixed_point,
                         params->tol};
             const int clusters = std::min(batch, plan->fused_clusters);
-            RatioParams rp{params->dynamic, params->r_fixed, params->phi_lo, params->phi_hi, params->r_max,
-                           params->criterion};
-            auto kern = with_stage1 ? stage2_fused_kernel<true> : stage2_fused_kernel<false>;
-            if (!c.ok(launch_pdl(kern, dim3((unsigned)(2 * clusters)), dim3(kFuThreads),
+            if (!c.ok(launch_pdl(stage2_fused_kernel, dim3((unsigned)(2 * clusters)), dim3(kFuThreads),
                                  (size_t)kFuSmemBytes, st, 2u, (const __nv_bfloat16 *)X, offsets, plan->d, batch,
                                  (const int32_t *)o.counts, (const int32_t *)order, (const float *)norms, maxN, total, op,
                                  (__nv_bfloat16 *)o.Y, o.out_offsets, o.kept_idx, o.merged_idx, o.merge_partner,
-                                 o.merge_weight, o.stats, (WsHeader *)(ws + L.header), rp,
-                                 params->rho, o.counts, (int *)(ws + L.sel_flag), plan->run)))
+                                 o.merge_weight, o.stats, (WsHeader *)(ws + L.header))))
                 return RTPRUNE_ERR_CUDA;
-            launched(plan, st, with_stage1 ? "fused" : "stage2_fused");
+            launched(plan, st, "stage2_fused");
             return RTPRUNE_OK;
         }
     }
@@ -428,7 +419,23 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         int fast_c = 0;
         const int fast_floats = plan->fast_smem_bytes / (int)sizeof(float);
         bool all_fast = false;
-        if (!use_log_form(params)) {
+        // Scaling form, every possible tile small enough for a thread's K values to stay in registers: clusters
+        // of two CTAs per image, in one wave when the batch allows (else the cluster kernels below)
+        const bool use_reg = kTensor && !use_log_form(params) && plan->fused_clusters > 0 &&
+                             sinkhorn_reg_eligible(maxN, maxB) && batch <= plan->fused_clusters;
+        if (use_reg) {
+            ready_list = (int32_t *)(ws + L.ready_list);
+            if (!c.ok(launch_pdl(sinkhorn_reg_kernel, dim3((unsigned)(2 * batch)), dim3(kFuThreads), (size_t)kFuSmemBytes,
+                                 st, 2u, offsets, (const int32_t *)o.counts, (const int32_t *)o.out_offsets,
+                                 (const int32_t *)order, (const float *)kmat, L.kmat_stride, maxN, total, op, pbuf,
+                                 pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats,
+                                 (uint32_t *)(ws + L.sink_done), ready_list, (WsHeader *)(ws + L.header),
+                                 (const uint32_t *)scores_done, plan->run)))
+                return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "sinkhorn_reg");
+            all_fast = true;
+        }
+        if (!use_log_form(params) && !use_reg) {
             // CTAs per image: as many as keep the whole batch on the chip at once, and more if the largest
             // possible tile needs them to keep K in their shared memory; 8 at most (tiles larger than the
             // cluster's shared memory iterate on K in the workspace)
@@ -559,10 +566,6 @@ rtprune_status_t run_device(rtprune_plan_t *plan, cudaStream_t st, const void *X
         return RTPRUNE_OK;
     }
     prof_begin(plan, st);
-    // One kernel for the whole path when every image the run can hold fits the fused kernel and stage 1 ranks by
-    // the l2 norm: the clusters stream their images themselves.
-    if (fused_whole_path(plan, params))
-        return launch_stage2<__nv_bfloat16>(plan, st, X, offsets, batch, total, params, ws, o, true);
     // with bf16 storage and anything to prune, the kernel that copies the pruned rows also turns the counts
     // into out_offsets, so that stage 1 ends with the last image's selection
     const bool scan_later = plan->dtype == RTPRUNE_BF16 && max_pruned(params, plan->max_tokens) > 0;
@@ -629,6 +632,7 @@ rtprune_status_t rtprune_default_params(rtprune_params_t *p)
     p->stop_at_fixed_point = 1;
     p->tol = 0.f;
     p->criterion = RTPRUNE_CRITERION_L2NORM;
+    p->schedule = RTPRUNE_SCHEDULE_AUTO;
     return RTPRUNE_OK;
 }
 
@@ -739,9 +743,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     // device runs at once is what a run's grid is capped at (its clusters then loop over the images).
     p->fused_clusters = 0;
     if (dtype == RTPRUNE_BF16 &&
-        cudaFuncSetAttribute(stage2_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
-            cudaSuccess &&
-        cudaFuncSetAttribute(stage2_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
+        cudaFuncSetAttribute(stage2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) ==
             cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2);
@@ -755,9 +757,12 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, stage2_fused_kernel<false>, &cfg) == cudaSuccess && nclusters > 0)
+        if (cudaOccupancyMaxActiveClusters(&nclusters, stage2_fused_kernel, &cfg) == cudaSuccess && nclusters > 0)
             p->fused_clusters = nclusters;
     }
+    (void)cudaGetLastError();
+    if (dtype == RTPRUNE_BF16)
+        (void)cudaFuncSetAttribute(sinkhorn_reg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes);
     (void)cudaGetLastError();
     // Clusters of 16 CTAs (beyond the portable size) for the wide-tile Sinkhorn kernel: ask the device how
     // many it can run at once; a run uses them only if all its images fit that number.

@@ -94,7 +94,7 @@ def run_gpu(w: synth.Workload, *, overrides: Optional[Dict[str, float]] = None,
         plan = binding.Plan(w.d, w.X.dtype, max(w.batch, 1), max(w.total_tokens, 1),
                             max(w.max_tokens, 1), device=dev)
     rho_dev = torch.from_numpy(w.rho.copy()).to(dev) if w.batch else None
-    fields = {k: (int(v) if k in ("dynamic", "iters", "form", "stop_at_fixed_point", "criterion") else float(v))
+    fields = {k: (int(v) if k in ("dynamic", "iters", "form", "stop_at_fixed_point", "criterion", "schedule") else float(v))
               for k, v in p.items()}
     if host_path:
         params = binding.make_params(None, **fields)
