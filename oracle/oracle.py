@@ -147,6 +147,39 @@ def sinkhorn(S, *, z: float = 0.2, eps: float = 1.0, iters: int = 100):
     return u, v, Pbar
 
 
+def exact_matching(S, *, z: float = 0.2):
+    """Eq. 2-6 solved exactly: the maximum-weight partial matching with gains S_ij - z.
+    Returns (match_prop [B] kept position or -1, objective, dual_kept [M], dual_prop [B])."""
+    S = _f64(S)
+    M, B = S.shape
+    match = np.empty(max(B, 1), dtype=np.int32)
+    obj = ctypes.c_double()
+    du = np.empty(max(M, 1))
+    dv = np.empty(max(B, 1))
+    lib().rtp_oracle_exact_matching(_dp(S), ctypes.c_int(M), ctypes.c_int(B), ctypes.c_double(z), _ip(match),
+                                    ctypes.byref(obj), _dp(du), _dp(dv))
+    return match[:B].copy(), obj.value, du[:M].copy(), dv[:B].copy()
+
+
+def matching_plan(match_prop, M: int) -> np.ndarray:
+    """The vertex of the LP that a matching stands for: P-bar [(M+1) x (B+1)] of zeros and ones plus the
+    dustbin cells (marginals a = [1_M, B], b = [1_B, M])."""
+    B = len(match_prop)
+    Pbar = np.zeros((M + 1, B + 1))
+    pairs = 0
+    for j, i in enumerate(match_prop):
+        if i >= 0:
+            Pbar[i, j] = 1.0
+            pairs += 1
+        else:
+            Pbar[M, j] = 1.0           # pruned token j goes to the dustbin row
+    for i in range(M):
+        if Pbar[i, :B].sum() == 0:
+            Pbar[i, B] = 1.0           # kept token i goes to the dustbin column
+    Pbar[M, B] = pairs
+    return Pbar
+
+
 def merge(T, kept, prop, Pbar, *, alpha: float = 0.1) -> np.ndarray:
     """Eq. 7.  Returns Y [M x D] fp64 (not rounded)."""
     T = _f64(T)
@@ -188,6 +221,7 @@ class Params:
     eps: float = 1.0
     iters: int = 100
     criterion: int = 0      # ranking of stage 1: 0 l2 norm (Eq. 1), 1 variance, 2 entropy (selection-metric ablation)
+    exact: bool = False     # solve the linear program of Eq. 2-6 exactly instead of running Sinkhorn iterations
 
 
 @dataclass
@@ -208,10 +242,38 @@ class ImageResult:
     u: Optional[np.ndarray] = None
     v: Optional[np.ndarray] = None
     Pbar: Optional[np.ndarray] = None
+    S: Optional[np.ndarray] = None          # exact mode: the score matrix the matching was solved on
+    objective: Optional[float] = None       # exact mode: value of the linear program
+
+
+def run_image_exact(T, p: Params, rho: float = 0.0) -> ImageResult:
+    """Algorithm 1 with the transport problem of Eq. 2-6 solved exactly: the steps of run_image strung
+    together from the step functions, the matching in place of the Sinkhorn iterations, hard pairs in Eq. 7."""
+    T = _f64(T)
+    N = T.shape[0]
+    C = norms(T)
+    ph = phi(T, C) if N >= 2 else 0.0
+    r, B, M = ratio(ph, rho, N, dynamic=p.dynamic, r_fixed=p.r_fixed, phi_lo=p.phi_lo, phi_hi=p.phi_hi,
+                    r_max=p.r_max)
+    kept, prop = select(criterion(T, p.criterion) if p.criterion else C, M)
+    if B == 0:
+        return ImageResult(N=N, M=M, B=0, C=C, phi=ph, rho=rho, r=r, kept=kept, prop=prop,
+                           partner=np.zeros(0, np.int32), weight=np.zeros(0), gap=np.zeros(0), Y=T[kept].copy())
+    S = scores(T, C, kept, prop)
+    match, obj, _, _ = exact_matching(S, z=p.z)
+    Pbar = matching_plan(match, M)
+    Y = merge(T, kept, prop, Pbar, alpha=p.alpha)
+    res = ImageResult(N=N, M=M, B=B, C=C, phi=ph, rho=rho, r=r, kept=kept, prop=prop, partner=match,
+                      weight=(match >= 0).astype(np.float64), gap=np.full(B, np.inf), Y=Y, Pbar=Pbar)
+    res.S = S
+    res.objective = obj
+    return res
 
 
 def run_image(T, p: Params, rho: float = 0.0, *, want_plan: bool = False,
               compute_phi: bool = True) -> ImageResult:
+    if p.exact:
+        return run_image_exact(T, p, rho)
     T = _f64(T)
     N, D = T.shape
     C = np.empty(N)

@@ -230,6 +230,109 @@ void rtp_oracle_sinkhorn(const double *S, int M, int B, double z, double eps, in
 }
 
 /*
+ * Eq. 2-6 solved EXACTLY (no entropic regularisation): the linear program
+ *     max sum_ij S-bar_ij P-bar_ij   s.t.  P-bar 1 = a = [1_M, B],  P-bar^T 1 = b = [1_B, M],  P-bar >= 0
+ * over the dustbin-augmented (M+1) x (B+1) plan.  Its constraint matrix is that of a transportation
+ * problem, so an optimal vertex is integral: every kept token i is either paired with one pruned token j
+ * (P_ij = 1) or sent to the dustbin column, every pruned token is either paired or sent to the dustbin
+ * row, and the dustbin-dustbin cell takes the rest.  With m pairs the objective is
+ *     sum_{pairs} S_ij + z (M - m) + z (B - m) + z m = sum_{pairs} (S_ij - z) + z N,
+ * so the optimum is a maximum-weight partial matching with gains g_ij = S_ij - z (pairs of non-positive
+ * gain are never needed).  Solved as an assignment problem on the clipped gains max(g_ij, 0): the smaller
+ * side is assigned, one by one, along shortest augmenting paths with dual potentials (the Hungarian
+ * method, O(n^2 m)); an assignment of clipped gain 0 means "unpaired".
+ *
+ * Outputs: match_prop[j] = kept position paired with pruned token j, or -1; objective = the LP value
+ * sum S-bar P-bar; dual_kept[M], dual_prop[B]: an optimal dual of the clipped assignment problem in
+ * max form (dual_kept_i + dual_prop_j >= max(g_ij, 0), duals of the unassigned side >= 0, and their sum
+ * equal to the clipped gain collected): a certificate of optimality a test can check by itself.
+ * Returns the number of pairs.  Ties between optimal matchings are broken by the order of the search.
+ */
+int rtp_oracle_exact_matching(const double *S, int M, int B, double z, int32_t *match_prop,
+                              double *objective, double *dual_kept, double *dual_prop)
+{
+    const int transposed = B > M;            /* rows of the assignment = the smaller side */
+    const int n = transposed ? M : B, m = transposed ? B : M;
+    /* cost[r][c] = -max(g, 0); 1-based arrays as in the classical formulation */
+    double *u = (double *)calloc((size_t)n + 1, sizeof(double));
+    double *v = (double *)calloc((size_t)m + 1, sizeof(double));
+    double *minv = (double *)malloc(((size_t)m + 1) * sizeof(double));
+    int *p = (int *)calloc((size_t)m + 1, sizeof(int));       /* p[c] = row assigned to column c (0: none) */
+    int *way = (int *)calloc((size_t)m + 1, sizeof(int));
+    char *used = (char *)malloc((size_t)m + 1);
+#define RTP_GAIN(r, c)                                                                           \
+    (transposed ? fmax(S[(size_t)((r) - 1) * B + ((c) - 1)] - z, 0.0)                            \
+                : fmax(S[(size_t)((c) - 1) * B + ((r) - 1)] - z, 0.0))
+    for (int i = 1; i <= n; ++i) {
+        p[0] = i;
+        int j0 = 0;
+        for (int j = 0; j <= m; ++j) {
+            minv[j] = INFINITY;
+            used[j] = 0;
+        }
+        do {
+            used[j0] = 1;
+            const int i0 = p[j0];
+            double delta = INFINITY;
+            int j1 = 0;
+            for (int j = 1; j <= m; ++j) {
+                if (used[j]) continue;
+                const double cur = -RTP_GAIN(i0, j) - u[i0] - v[j];
+                if (cur < minv[j]) {
+                    minv[j] = cur;
+                    way[j] = j0;
+                }
+                if (minv[j] < delta) {
+                    delta = minv[j];
+                    j1 = j;
+                }
+            }
+            for (int j = 0; j <= m; ++j) {
+                if (used[j]) {
+                    u[p[j]] += delta;
+                    v[j] -= delta;
+                } else {
+                    minv[j] -= delta;
+                }
+            }
+            j0 = j1;
+        } while (p[j0] != 0);
+        do {
+            const int j1 = way[j0];
+            p[j0] = p[j1];
+            j0 = j1;
+        } while (j0);
+    }
+    for (int j = 0; j < B; ++j) match_prop[j] = -1;
+    int pairs = 0;
+    double value = z * (double)(M + B);
+    for (int c = 1; c <= m; ++c) {
+        const int r = p[c];
+        if (r == 0) continue;
+        const int kept_i = transposed ? r - 1 : c - 1, prop_j = transposed ? c - 1 : r - 1;
+        const double g = S[(size_t)kept_i * B + prop_j] - z;
+        if (g > 0.0) {                       /* clipped gain 0: the two stay unpaired */
+            match_prop[prop_j] = kept_i;
+            value += g;
+            ++pairs;
+        }
+    }
+    *objective = value;
+    if (dual_kept && dual_prop) {            /* max form: minus the potentials of the min-cost form */
+        for (int r = 1; r <= n; ++r) (transposed ? dual_kept : dual_prop)[r - 1] = -u[r];
+        for (int c = 1; c <= m; ++c) (transposed ? dual_prop : dual_kept)[c - 1] = -v[c];
+    }
+#undef RTP_GAIN
+    free(u);
+    free(v);
+    free(minv);
+    free(p);
+    free(way);
+    free(used);
+    return pairs;
+}
+
+/*
  * Eq. 7 / Appendix C (merge equation): T_k^i <- T_k^i + alpha * sum_j P_ij T_p^j, with P the
  * non-dustbin block of P-bar (row stride B+1).  No renormalisation.  Y is M x D, rows in the order
  * of `kept`.
