@@ -56,9 +56,22 @@ typedef enum { RTPRUNE_BF16 = 0, RTPRUNE_FP32 = 1 } rtprune_dtype_t;
  *   LOG     u, v are the log-domain duals and every sweep is a max-shifted log-sum-exp, as printed.
  *   SCALING the duals are carried as e^u, e^v against the kernel K = exp((S-bar - c)/eps): every
  *           sweep is a matrix-vector product.  Used only when eps >= 0.25, where K cannot underflow.
- *   AUTO    SCALING when eps >= 0.25, else LOG. */
-typedef enum { RTPRUNE_SINKHORN_AUTO = 0, RTPRUNE_SINKHORN_LOG = 1, RTPRUNE_SINKHORN_SCALING = 2 }
-    rtprune_sinkhorn_form_t;
+ *   AUTO    SCALING when eps >= 0.25, else LOG.
+ *   EXACT   no iterations: the linear program of Eq. 2-6 itself is solved (the limit eps -> 0 of the
+ *           entropic problem).  With the dustbins of Eq. 5 it is a maximum-weight partial matching in
+ *           which pairing kept token i with pruned token j gains S_ij - z over leaving both in the
+ *           dustbins; the solver finds a vertex by shortest augmenting paths in fp32.  The plan then
+ *           holds ones at the pairs and zeros elsewhere, Eq. 7 adds alpha T_p^j to the partner of every
+ *           paired token, merge_partner is the kept position or -1 (unpaired: the token is dropped),
+ *           merge_weight is 1 or 0, stats[5] counts path-search steps and stats[6] is 0.  eps, iters,
+ *           stop_at_fixed_point, tol and schedule are ignored.  Where several matchings reach the optimum
+ *           any one of them may be returned. */
+typedef enum {
+    RTPRUNE_SINKHORN_AUTO = 0,
+    RTPRUNE_SINKHORN_LOG = 1,
+    RTPRUNE_SINKHORN_SCALING = 2,
+    RTPRUNE_SINKHORN_EXACT = 3
+} rtprune_sinkhorn_form_t;
 
 /* Criterion C_k by which stage 1 ranks the tokens of an image (the M largest are kept).  The paper's
  * method uses the l2 norm (Eq. 1); its ablation on the selection metric also ranks by variance and by
@@ -197,24 +210,36 @@ rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const v
  * library holds it until the process exits).  It calls no cudaMalloc / cudaFree and no allocating
  * library routine; inputs and outputs are still the caller's buffers.
  *
- *   - Limit: the plan's stage-1 scratch (norms, unit-token partial sums, selection lists; it grows
- *     with max_total_tokens and with max_batch * max_tokens_per_image * d) must fit the array, else
- *     RTPRUNE_ERR_WORKSPACE is returned and nothing is launched.  A 64-image x 400-token x 1280
- *     plan needs about 2.6 MiB.
+ *   - Limit: the plan's stage-1 scratch must fit the array, else RTPRUNE_ERR_WORKSPACE is returned and
+ *     nothing is launched.  rtprune_static_scratch_needed reports it for a plan; with a(x) = x rounded
+ *     up to a multiple of 256 it is
+ *         256 + 4 a(4 max_batch) + 4 a(4 max_total_tokens)
+ *             + a(4 max_batch ceil(max_tokens_per_image / 32) d)   bytes,
+ *     the last term (partial sums of the unit tokens, Eq. 8) being the large one: a 64-image x 400-token
+ *     x 1280 plan needs 4,670,720 bytes (4.45 MiB), and 114 such images are the most the array holds.
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside any stream capture.
  *   - Every call on a device shares the one array, which keeps the previous call's contents; the
  *     call clears the words that must start at zero itself.  Two calls that overlap on the same
  *     GPU (different streams, or threads) race on it: serialise them.
- *   - The device status word lives in the array too and cannot be read with rtprune_query_status;
- *     a batch that breaks the offsets contract yields counts of 0 for the offending image.
+ *   - The device status word lives in the array too: read it with rtprune_query_status_static (a
+ *     non-finite token norm, an image outside the offsets contract, whose count is then 0).
  */
-#define RTPRUNE_STATIC_SCRATCH_BYTES (4u << 20)
+#define RTPRUNE_STATIC_SCRATCH_BYTES (8u << 20)
 rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, const void *X,
                                        const int32_t *offsets, int32_t batch, int64_t total_tokens,
                                        const rtprune_params_t *params, int32_t *out_offsets,
                                        int32_t *counts, float *stats, float *norms_out,
                                        int32_t *order_out);
+
+/* Bytes of the built-in array rtprune_select_static uses for this plan (it runs iff they are at most
+ * RTPRUNE_STATIC_SCRATCH_BYTES).  HOST pointers. */
+rtprune_status_t rtprune_static_scratch_needed(const rtprune_plan_t *plan, size_t *bytes);
+
+/* rtprune_query_status for the built-in array of the current device: synchronises the stream, reads the
+ * status word the last rtprune_select_static call on this device left there and clears it.  Allocates
+ * nothing.  Before any rtprune_select_static call on the device it reports RTPRUNE_OK and no bits. */
+rtprune_status_t rtprune_query_status_static(rtprune_plan_t *plan, void *cuda_stream, uint32_t *flags_out);
 
 /*
  * The same run, from and to HOST buffers (pinned memory recommended): copies X, offsets and rho to
@@ -275,6 +300,19 @@ rtprune_status_t rtprune_profile_read(rtprune_plan_t *plan, int32_t *n, float *m
 rtprune_status_t rtprune_density(void *cuda_stream, const uint8_t *images, int32_t batch, int32_t height,
                                  int32_t width, int32_t patch, float tau, float *rho,
                                  uint32_t *image_counts, int32_t *edge_counts);
+
+/*
+ * Test aid: makes the library's bounded device-side waits run out without any fault.  Launches one small
+ * kernel on the stream that waits, with the same wait routines the kernels of a run use but only
+ * `poll_limit` polls (1 .. 65536), first for a run number that no run ever has (the flag in the workspace
+ * header the second-stage kernels wait on) and then on a shared-memory barrier nobody arrives at.  Each wait
+ * that gives up sets RTPRUNE_DEV_TIMEOUT in the workspace's status word, exactly as a kernel of a run does;
+ * the kernel then returns normally, so the context and the workspace stay usable and the next
+ * rtprune_query_status reports RTPRUNE_ERR_TIMEOUT.  `expired_out` (DEVICE int32, may be NULL) receives the
+ * number of waits that gave up (2).  The workspace must have been initialised.
+ */
+rtprune_status_t rtprune_test_expire_waits(rtprune_plan_t *plan, void *cuda_stream, void *workspace,
+                                           size_t workspace_bytes, uint32_t poll_limit, int32_t *expired_out);
 
 /* Kernels launched by the most recent run / select / run_host call on this plan. */
 int32_t rtprune_last_launch_count(const rtprune_plan_t *plan);

@@ -17,7 +17,7 @@ from . import build as _build
 
 STATS_STRIDE = 8
 BF16, FP32 = 0, 1
-SINKHORN_AUTO, SINKHORN_LOG, SINKHORN_SCALING = 0, 1, 2
+SINKHORN_AUTO, SINKHORN_LOG, SINKHORN_SCALING, SINKHORN_EXACT = 0, 1, 2, 3
 SCHEDULE_AUTO, SCHEDULE_SEPARATE, SCHEDULE_FUSED = 0, 1, 2
 DEV_NONFINITE, DEV_TIMEOUT, DEV_BAD_OFFSETS = 1, 2, 4
 
@@ -65,6 +65,9 @@ def lib() -> ctypes.CDLL:
     L.rtprune_workspace_init.argtypes = [vp, vp, vp, sz]
     L.rtprune_select.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, sz, vp, vp, vp, vp, vp]
     L.rtprune_select_static.argtypes = [vp, vp, vp, vp, i32, i64, pp, vp, vp, vp, vp, vp]
+    L.rtprune_static_scratch_needed.argtypes = [vp, ctypes.POINTER(sz)]
+    L.rtprune_query_status_static.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.rtprune_test_expire_waits.argtypes = [vp, vp, vp, sz, ctypes.c_uint32, vp]
     L.rtprune_run_host.argtypes = [vp, vp, vp, vp, vp, i32, i64, pp, vp, sz,
                                    vp, vp, vp, vp, vp, vp, vp, vp]
     L.rtprune_host_arena_bytes.argtypes = [vp, ctypes.POINTER(sz)]
@@ -209,6 +212,27 @@ class Plan:
                                            out.counts.data_ptr(), out.stats.data_ptr(),
                                            _ptr(norms_out), _ptr(order_out)),
                "rtprune_select_static")
+
+    # -- rtprune_static_scratch_needed / rtprune_query_status_static
+    def static_scratch_needed(self) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().rtprune_static_scratch_needed(self.handle, ctypes.byref(n)), "rtprune_static_scratch_needed")
+        return n.value
+
+    def query_status_static(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """Synchronises, returns the status bits the last select_static call left (0 = clean), clears them."""
+        flags = ctypes.c_uint32()
+        lib().rtprune_query_status_static(self.handle, _stream_handle(stream), ctypes.byref(flags))
+        return flags.value
+
+    # -- rtprune_test_expire_waits
+    def expire_waits(self, poll_limit: int, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """Test aid: lets two bounded device-side waits run out on this plan's workspace; returns how many did."""
+        expired = torch.zeros(1, dtype=torch.int32, device=self.device)
+        _check(lib().rtprune_test_expire_waits(self.handle, _stream_handle(stream), self.workspace.data_ptr(),
+                                               self.workspace.numel(), int(poll_limit), expired.data_ptr()),
+               "rtprune_test_expire_waits")
+        return int(expired.item())
 
     # -- rtprune_host_arena_bytes / rtprune_run_host
     def host_arena_bytes(self) -> int:

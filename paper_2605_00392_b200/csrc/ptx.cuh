@@ -46,10 +46,10 @@ __device__ inline bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.  false = gave up.
-__device__ inline bool mbar_wait(uint64_t *bar, uint32_t parity)
+// Bounded wait for the phase with the given parity to complete.  false = gave up after `limit` polls.
+__device__ inline bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit = kSpinLimit)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -94,10 +94,10 @@ __device__ inline void st_release_gpu(int *p, int v)
 {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-// Bounded wait until *p == want (acquire).  false = gave up.
-__device__ inline bool wait_equal_gpu(const int *p, int want)
+// Bounded wait until *p == want (acquire).  false = gave up after `limit` polls.
+__device__ inline bool wait_equal_gpu(const int *p, int want, uint32_t limit = kSpinLimit)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (ld_acquire_gpu(p) == want) return true;
         __nanosleep(200);
     }

@@ -10,6 +10,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "exact.cuh"
 #include "fused.cuh"
 #include "gemm_simt.cuh"
 #include "merge_umma.cuh"
@@ -47,6 +48,7 @@ struct rtprune_plan_s {
     int run;       // number of the most recent run's second stage, unique in the process: what the kernels
                    // that share counters through the workspace wait for before they read them
     int fused_clusters;     // clusters of 2 CTAs of the fused stage-2 kernel the device runs at once (0: none)
+    int exact_smem_bytes;   // dynamic shared memory of the exact-pairing kernel
 };
 
 // Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
@@ -159,6 +161,26 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Test aid (rtprune_test_expire_waits): two waits that nothing ends, with a short poll limit.
+__global__ void expire_waits_kernel(WsHeader *hdr, uint32_t poll_limit, int32_t *expired_out)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x != 0) return;
+    int expired = 0;
+    // run numbers count up from 1: -1 is not stored before a process has made 2^32 - 1 runs
+    if (!ptx::wait_equal_gpu(&hdr->run_tag, -1, poll_limit)) {
+        atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+        ++expired;
+    }
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+    if (!ptx::mbar_wait(&bar, 0, poll_limit)) {     // phase 0 never completes: nobody arrives
+        atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+        ++expired;
+    }
+    if (expired_out) *expired_out = expired;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -197,7 +219,7 @@ rtprune_status_t check_params(const rtprune_params_t *p)
     if (!(p->eps > 0.f) || !std::isfinite(p->eps)) return RTPRUNE_ERR_INVALID_ARG;
     if (!std::isfinite(p->z) || !std::isfinite(p->alpha)) return RTPRUNE_ERR_INVALID_ARG;
     if (p->iters < 0) return RTPRUNE_ERR_INVALID_ARG;
-    if (p->form < RTPRUNE_SINKHORN_AUTO || p->form > RTPRUNE_SINKHORN_SCALING)
+    if (p->form < RTPRUNE_SINKHORN_AUTO || p->form > RTPRUNE_SINKHORN_EXACT)
         return RTPRUNE_ERR_INVALID_ARG;
     if (!(p->tol >= 0.f)) return RTPRUNE_ERR_INVALID_ARG;
     if (p->criterion < RTPRUNE_CRITERION_L2NORM || p->criterion > RTPRUNE_CRITERION_ENTROPY)
@@ -327,7 +349,7 @@ rtprune_status_t launch_stage1(rtprune_plan_t *plan, cudaStream_t st, const void
 bool fused_stage2_ok(const rtprune_plan_t *plan, const rtprune_params_t *params)
 {
     const int maxB = max_pruned(params, plan->max_tokens);
-    if (params->schedule == RTPRUNE_SCHEDULE_SEPARATE) return false;
+    if (params->schedule == RTPRUNE_SCHEDULE_SEPARATE || params->form == RTPRUNE_SINKHORN_EXACT) return false;
     // AUTO: the separate kernels overlap one another across the images of a batch and are ahead on the batches
     // measured so far; the fused kernel is taken on request
     if (params->schedule == RTPRUNE_SCHEDULE_AUTO) return false;
@@ -353,6 +375,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     int32_t *ready_list = nullptr;   // images in the order their plans are finished, when the merge follows it
     do plan->run = ++g_run_count; while (plan->run == 0);   // 0 is what a fresh workspace holds
     uint32_t *scores_done = nullptr; // per-image counts of finished score tiles, when the scores kernel keeps them
+    const bool iterate = params->form != RTPRUNE_SINKHORN_EXACT;   // Sinkhorn iterations, else the exact pairing
 
     if constexpr (kTensor) {
         // One kernel for the whole second stage when every image the run can hold fits it
@@ -396,7 +419,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             // costs each scores CTA a release (its stores made visible before it counts itself), which
             // pays when the grid is one wave of CTAs and its end is a tail of a few slow CTAs, not when
             // CTAs queue for the SMs.
-            if ((long long)grid.x * grid.y <= 2LL * plan->sm_count) scores_done = (uint32_t *)(ws + L.scores_done);
+            if (iterate && (long long)grid.x * grid.y <= 2LL * plan->sm_count)
+                scores_done = (uint32_t *)(ws + L.scores_done);
             if (!c.ok(launch_pdl(scores_umma_kernel, grid, dim3(kScThreads), kScSmemBytes, st, 1u, tmapX, tmapXp,
                                  offsets, plan->d, o.counts, order, (const int32_t *)(ws + L.kpos), norms, kmat,
                                  L.kmat_stride, maxN, total, (WsHeader *)(ws + L.header), scores_done)))
@@ -421,7 +445,16 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         bool all_fast = false;
         // Scaling form, every possible tile small enough for a thread's K values to stay in registers: clusters
         // of two CTAs per image, in one wave when the batch allows (else the cluster kernels below)
-        const bool use_reg = kTensor && !use_log_form(params) && plan->fused_clusters > 0 &&
+        if (!iterate) {
+            // Eq. 2-6 solved exactly, one CTA per image (an ordinary launch: it starts when the scores are complete)
+            exact_pairing_kernel<<<batch, kExThreads, plan->exact_smem_bytes, st>>>(
+                offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
+                plan->exact_smem_bytes / (int)sizeof(float), pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
+                o.merge_weight, o.stats, (WsHeader *)(ws + L.header));
+            if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+            launched(plan, st, "exact_pairing");
+        }
+        const bool use_reg = iterate && kTensor && !use_log_form(params) && plan->fused_clusters > 0 &&
                              sinkhorn_reg_eligible(maxN, maxB) && batch <= plan->fused_clusters;
         if (use_reg) {
             ready_list = (int32_t *)(ws + L.ready_list);
@@ -435,7 +468,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             launched(plan, st, "sinkhorn_reg");
             all_fast = true;
         }
-        if (!use_log_form(params) && !use_reg) {
+        if (iterate && !use_log_form(params) && !use_reg) {
             // CTAs per image: as many as keep the whole batch on the chip at once, and more if the largest
             // possible tile needs them to keep K in their shared memory; 8 at most (tiles larger than the
             // cluster's shared memory iterate on K in the workspace)
@@ -489,7 +522,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         // CTAs iterate on K in the workspace tile; the general kernel keeps only what is wider still.
         // It takes all the shared memory a CTA can have: what its fixed regions leave is the ring of row blocks.
         const size_t tall_smem = (size_t)std::max(plan->smem_optin - 1024, 0);
-        const bool tall = !use_log_form(params) && !all_fast &&
+        const bool tall = iterate && !use_log_form(params) && !all_fast &&
                           sizeof(float) * (sinkhorn_tall_smem_floats(std::min(maxB, kTallMaxB), maxN) +
                                            kTallStageFloatsMax) <= tall_smem;
         if (tall) {      // (rtprune_plan gave the kernel its shared memory)
@@ -511,7 +544,8 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
             launched(plan, st, "sinkhorn_tall");
             if (maxB <= kTallMaxB) all_fast = true;       // nothing is left for the general kernel
         }
-        if (use_log_form(params))
+        if (!iterate) {
+        } else if (use_log_form(params))
             sinkhorn_kernel<true><<<batch, kSinkThreads, plan->sink_smem_bytes, st>>>(
                 offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
@@ -522,7 +556,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 smem_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
                 o.stats, fast_c, fast_floats, tall ? kTallMaxB : 0);
         if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
-        if (use_log_form(params) || !all_fast) launched(plan, st, "sinkhorn");
+        if (iterate && (use_log_form(params) || !all_fast)) launched(plan, st, "sinkhorn");
     }
 
     if constexpr (kTensor) {
@@ -710,6 +744,14 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         }
     }
     p->fast_smem_bytes = (int)(cap / 16 * 16);
+    p->exact_smem_bytes = (int)(exact_smem_bytes(max_tokens_per_image, (size_t)std::max(optin - 4096, 0)) / 16 * 16);
+    if (4 * exact_array_words(max_tokens_per_image) > (size_t)p->exact_smem_bytes ||
+        !c.ok(cudaFuncSetAttribute(exact_pairing_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   std::max(optin - 4096, 0)))) {
+        if (!p->last_cuda_error) p->last_cuda_error = (int)cudaErrorInvalidValue;
+        delete p;
+        return RTPRUNE_ERR_CUDA;
+    }
     if (!c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    p->fast_smem_bytes)) ||
         !c.ok(cudaFuncSetAttribute(sinkhorn_cluster_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -896,6 +938,55 @@ rtprune_status_t rtprune_select_static(rtprune_plan_t *plan, void *cuda_stream, 
     prof_begin(plan, st);
     return launch_stage1(plan, st, X, offsets, batch, (int)total_tokens, params, scratch, out_offsets,
                          counts, stats, norms_out, order_out, true);
+}
+
+rtprune_status_t rtprune_static_scratch_needed(const rtprune_plan_t *plan, size_t *bytes)
+{
+    if (!plan || !bytes) return RTPRUNE_ERR_INVALID_ARG;
+    *bytes = plan->ws.kmat;      // stage 1 uses the workspace regions that precede the score tiles
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_query_status_static(rtprune_plan_t *plan, void *cuda_stream, uint32_t *flags_out)
+{
+    if (!plan) return RTPRUNE_ERR_INVALID_ARG;
+    if (!on_plan_device(plan)) return RTPRUNE_ERR_INVALID_ARG;
+    Checked c{plan};
+    int dev = -1;
+    if (!c.ok(cudaGetDevice(&dev))) return RTPRUNE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return RTPRUNE_ERR_UNSUPPORTED;
+    char *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        scratch = (char *)g_static_scratch_addr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint32_t flags = 0;
+    if (scratch) {
+        WsHeader *hdr = (WsHeader *)(scratch + plan->ws.header);
+        if (!c.ok(cudaMemcpyAsync(&flags, &hdr->status, sizeof(flags), cudaMemcpyDeviceToHost, st)) ||
+            !c.ok(cudaMemsetAsync(&hdr->status, 0, sizeof(uint32_t), st)) || !c.ok(cudaStreamSynchronize(st)))
+            return RTPRUNE_ERR_CUDA;
+    }
+    if (flags_out) *flags_out = flags;
+    if (flags & RTPRUNE_DEV_NONFINITE) return RTPRUNE_ERR_NONFINITE;
+    if (flags & RTPRUNE_DEV_BAD_OFFSETS) return RTPRUNE_ERR_BAD_OFFSETS;
+    if (flags & RTPRUNE_DEV_TIMEOUT) return RTPRUNE_ERR_TIMEOUT;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_test_expire_waits(rtprune_plan_t *plan, void *cuda_stream, void *workspace,
+                                           size_t workspace_bytes, uint32_t poll_limit, int32_t *expired_out)
+{
+    if (!plan || !workspace || ((uintptr_t)workspace & 255u)) return RTPRUNE_ERR_INVALID_ARG;
+    if (!on_plan_device(plan)) return RTPRUNE_ERR_INVALID_ARG;
+    if (workspace_bytes < plan->ws.total) return RTPRUNE_ERR_WORKSPACE;
+    if (poll_limit < 1 || poll_limit > 65536) return RTPRUNE_ERR_INVALID_ARG;
+    Checked c{plan};
+    expire_waits_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>((WsHeader *)((char *)workspace + plan->ws.header),
+                                                                 poll_limit, expired_out);
+    if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+    return RTPRUNE_OK;
 }
 
 rtprune_status_t rtprune_host_arena_bytes(const rtprune_plan_t *plan, size_t *arena_bytes)

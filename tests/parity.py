@@ -39,6 +39,7 @@ MERGE_ROW_GAIN_TOL = {torch.float32: 1e-3}    # per row with a visible term
 BF16_MODEL_MISMATCH = 0.01      # share of a bf16 image's elements that may differ from the reference
 ROUND_MARGIN = 1e-3
 ORACLE_CHUNK = 64          # images per oracle call: bounds the fp64 copies held at once
+EXACT_OBJECTIVE_RTOL = 1e-5     # exact pairing: the device's matching reaches the oracle's optimum to this
 
 
 def oracle_params(p: Dict[str, float]) -> oracle.Params:
@@ -261,6 +262,85 @@ def check_workload(w: synth.Workload, *, images: Optional[Sequence[int]] = None,
                                               report.get("max_partner_regret", 0.0), report.get("max_feature_err", 0.0),
                                               report.get("max_merge_gain_err", 0.0),
                                               report.get("max_merge_row_gain_err", 0.0)))
+    return report
+
+
+def check_exact(w: synth.Workload, *, overrides: Optional[Dict[str, float]] = None,
+                images: Optional[Sequence[int]] = None, plan: Optional[binding.Plan] = None) -> Dict[str, float]:
+    """Exact pairing (Eq. 2-6 as a linear program) against the oracle's exact solver.  Several matchings can
+    be optimal, so what is unique is compared and the rest is checked for validity:
+      * selection outputs, phi, r: as in compare_image (bit-exact / same tolerances);
+      * the device's matching is valid: partners in [-1, M), no kept token paired twice, every pair's gain
+        S_ij - z positive on the oracle's fp64 scores (to 1e-6: the device decides it in fp32);
+      * its objective, evaluated on the oracle's fp64 scores, reaches the oracle's optimum within
+        EXACT_OBJECTIVE_RTOL (and cannot exceed it by more than rounding);
+      * merge_weight is 1 at the pairs and 0 elsewhere;
+      * Y equals Eq. 7 evaluated by the oracle on the device's own matching, within FEATURE_TOL."""
+    imgs = list(range(w.batch)) if images is None else list(images)
+    if overrides:
+        w.params.update(overrides)
+    settle_rho(w, imgs)
+    res = run_gpu(w, overrides={"form": binding.SINKHORN_EXACT}, plan=plan)
+    assert res.status_bits == 0, res.status_bits
+    g = res.out
+    p = oracle_params(w.params)
+    report: Dict[str, float] = {"launches": res.launches, "images_compared": len(imgs), "pairs": 0, "pruned": 0}
+    tol = FEATURE_TOL[w.X.dtype]
+    with ThreadPoolExecutor(max_workers=cpu_threads()) as ex:
+        refs = list(ex.map(lambda i: oracle.run_image_exact(w.image_f64(i), p, float(w.rho[i])), imgs))
+    for i, ref in zip(imgs, refs):
+        tag = "%s image %d (exact)" % (w.name, i)
+        o0, o1 = int(g.out_offsets[i]), int(g.out_offsets[i + 1])
+        assert int(g.counts[i]) == ref.M and o1 - o0 == ref.M, (tag, int(g.counts[i]), ref.M)
+        st = g.stats[i].numpy()
+        assert abs(st[0] - ref.phi) <= 2e-5 and abs(st[2] - ref.r) <= 1e-5, tag
+        np.testing.assert_array_equal(g.kept_idx[o0:o1].numpy(), ref.kept, err_msg=tag)
+        seg = int(w.offsets[i]) - o0
+        np.testing.assert_array_equal(g.merged_idx[seg:seg + ref.B].numpy(), ref.prop, err_msg=tag)
+        y = g.Y[o0:o1].to(torch.float64).numpy()
+        if ref.B == 0:
+            assert torch.equal(g.Y[o0:o1], w.X[int(w.offsets[i]):int(w.offsets[i + 1])]), tag
+            continue
+        gp = g.merge_partner[seg:seg + ref.B].numpy()
+        gw = g.merge_weight[seg:seg + ref.B].numpy()
+        assert np.all((gp >= -1) & (gp < ref.M)), tag
+        paired = gp >= 0
+        assert len(np.unique(gp[paired])) == int(paired.sum()), (tag, "a kept token is paired twice")
+        np.testing.assert_array_equal(gw, paired.astype(np.float32), err_msg=tag)
+        z = float(np.float32(w.params["z"]))
+        gains = ref.S[gp[paired], np.nonzero(paired)[0]] - z
+        assert np.all(gains > -1e-6), (tag, float(gains.min()))
+        objective = z * (ref.M + ref.B) + float(gains.sum())
+        gap = (ref.objective - objective) / max(abs(ref.objective), 1e-30)
+        report["max_objective_gap"] = max(report.get("max_objective_gap", 0.0), gap)
+        assert -1e-6 * ref.B <= gap <= EXACT_OBJECTIVE_RTOL, (tag, objective, ref.objective)
+        report["pairs"] += int(paired.sum())
+        report["pruned"] += ref.B
+        report["same_as_oracle"] = report.get("same_as_oracle", 0) + int((gp == ref.partner).sum())
+        assert st[5] >= min(ref.M, ref.B), (tag, st[5])
+        # Eq. 7 on the device's own matching
+        a0 = int(w.offsets[i])
+        Ti = w.X[a0:a0 + ref.N].to(torch.float64).numpy()
+        ystar = oracle.merge(Ti, ref.kept, ref.prop, oracle.matching_plan(gp, ref.M), alpha=p.alpha)
+        rms = np.sqrt(np.mean(ystar * ystar, axis=1, keepdims=True))
+        denom = np.maximum(np.abs(ystar), rms)
+        err = np.abs(y - ystar) / np.where(denom > 0, denom, 1.0)
+        worst = float(err.max())
+        report["max_feature_err"] = max(report.get("max_feature_err", 0.0), worst)
+        assert worst <= tol, (tag, worst, tol)
+        # the term itself: rows that received a token differ from T_k, rows that did not are T_k bit for bit
+        got_rows = np.zeros(ref.M, dtype=bool)
+        got_rows[gp[paired]] = True
+        xk = w.X[a0:a0 + ref.N][torch.from_numpy(ref.kept.astype(np.int64))]
+        assert torch.equal(g.Y[o0:o1][torch.from_numpy(~got_rows)], xk[torch.from_numpy(~got_rows)]), tag
+        if w.X.dtype == torch.float32 and p.alpha != 0.0 and got_rows.any():
+            term = ystar[got_rows] - Ti[ref.kept][got_rows]
+            got = y[got_rows] - Ti[ref.kept][got_rows]
+            gain = float((got * term).sum() / (term * term).sum())
+            assert abs(gain - 1.0) <= MERGE_GAIN_TOL[torch.float32], (tag, "merge-term gain", gain)
+    print("exact parity %s: %d images, %d of %d pruned tokens paired, %d pairs as the oracle's, objective gap %.2e, "
+          "max feature err %.2e" % (w.name, len(imgs), report["pairs"], report["pruned"], report.get("same_as_oracle", 0),
+                                    report.get("max_objective_gap", 0.0), report.get("max_feature_err", 0.0)))
     return report
 
 
