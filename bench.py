@@ -5,10 +5,11 @@ A step is one pass of the whole path (norms + statistics -> ratio -> top-M -> co
 Sinkhorn -> merge + pack) over one synthetic DeepSeek-OCR-Large-shaped batch: 64 images x 400 tokens
 x 1280 bf16, dynamic ratio with mean retention ~0.84.  Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--repeats R] [--impl reference]
 
-N > 1 is launched by torch.distributed.run (one rank per GPU); images are independent, so every rank
-prunes its own batch and there is no data-path collective (weak scaling).
+N > 1 runs one rank per GPU under torch.distributed.run (started by the caller, or by bench.py itself when
+it is run plainly with --gpus N); images are independent, so every rank prunes its own batch and there is no
+data-path collective (weak scaling).  The K-step region is timed R times; `value` is the median region.
 --impl reference times the fp64 CPU oracle on the host cores instead (a deliberately slow program).
 """
 from __future__ import annotations
@@ -32,8 +33,9 @@ WORKLOAD = "large"
 WORKLOAD_DESC = "large: 64 images x 400 tokens x 1280 bf16, dynamic ratio (mean retention 0.84), T=100"
 ROTATE = 4                 # input/output buffer sets cycled so that no step finds its input in L2
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
-REFERENCE_SAMPLE = 8       # images per step of the --impl reference arm
+REFERENCE_SAMPLE = 64      # images per step of the --impl reference arm: the whole Large batch, as cpu_baseline
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
+# (kernels changed since their capture, or never captured, have no entry and report null)
 NCU_TRAFFIC_BYTES = {"stage1": 66109952, "gather": 10354432, "scores": 85585408,
                      "sinkhorn_cluster": 4840960, "merge": 119804416, "density_tile": 318402048}
 
@@ -130,7 +132,7 @@ def run_reference(args, rank: int) -> None:
         t += time_oracle(w, images, threads)
     ms = 1e3 * t / max(args.steps, 1)
     value = REFERENCE_SAMPLE / (ms / 1e3)
-    sample = "first %d images of the Large batch per step, all host cores" % REFERENCE_SAMPLE
+    sample = "all %d images of the Large batch per step, all host cores" % REFERENCE_SAMPLE
     line = {"impl": "reference", "metric": "pruned images/sec", "value": value, "unit": "images/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
@@ -147,6 +149,10 @@ def run_reference(args, rank: int) -> None:
 def run_density(args) -> None:
     """`--step density`: the textual-density kernel (Eq. 9) alone, on the pages of one Large batch (64
     pages of 1280 x 1280 RGB, 8 bits per channel).  One GPU; prints one JSON line of its own."""
+    print(json.dumps(density_line(args)))
+
+
+def density_line(args) -> dict:
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device")
     from paper_2605_00392_b200 import binding, synth
@@ -205,7 +211,7 @@ def run_density(args) -> None:
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": len(sample) / dt, "unit": "images/s", "cores": 1, "kind": "oracle",
                                 "sample": "4 pages of the batch, numpy fp64, one thread"}
-    print(json.dumps(line))
+    return line
 
 
 LARGE_N = {   # token counts before -> after pruning of the OCR models with large visual token sets (the paper's
@@ -219,6 +225,10 @@ def run_large_n(args) -> None:
     """`--step largen`: the whole path on images of thousands of tokens (score tiles of 4 to 19 MB that
     no cluster's shared memory holds: the Sinkhorn kernel for wide tiles).  One GPU; one JSON line with
     one entry per shape."""
+    print(json.dumps(large_n_line(args)), flush=True)
+
+
+def large_n_line(args) -> dict:
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the pruning path has no CPU fallback")
     from paper_2605_00392_b200 import binding, synth
@@ -277,10 +287,98 @@ def run_large_n(args) -> None:
             shapes[name]["cpu_baseline"] = {"value": batch / sec, "unit": "images/s", "cores": threads, "kind": "oracle",
                                             "sample": "all %d images of this batch, once" % batch}
         plan.close()
-    print(json.dumps({"metric": "pruned images/sec", "unit": "images/s", "n_gpus": 1, "steps": steps, "warmup": warm,
-                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
-                      "timing": "sum of the kernels' CUDA-event times per step, L2 flushed between steps",
-                      "shapes": shapes}), flush=True)
+    return {"metric": "pruned images/sec", "unit": "images/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+            "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "timing": "sum of the kernels' CUDA-event times per step, L2 flushed between steps",
+            "shapes": shapes}
+
+
+def sweep_line(w0, steps: int, warm: int) -> dict:
+    """1024 images x 400 tokens (the Large batch tiled 16 times on the device: 1.05 GB of tokens, far beyond L2):
+    the batch on which the path's HBM bound can be approached.  One GPU."""
+    from paper_2605_00392_b200 import binding
+    dev = torch.device("cuda", 0)
+    reps = 16
+    batch, total, d = w0.batch * reps, w0.total_tokens * reps, w0.d
+    X = w0.X.to(dev).repeat(reps, 1)
+    lens = np.tile(np.diff(w0.offsets.astype(np.int64)), reps)
+    offs = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).to(dev)
+    rho = torch.from_numpy(np.tile(w0.rho, reps)).to(dev)
+    fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
+    params = binding.make_params(rho, **fields)
+    plan = binding.Plan(d, torch.bfloat16, batch, total, w0.max_tokens, device=dev)
+    out = binding.Outputs.allocate(total, batch, d, torch.bfloat16, dev)
+    for _ in range(warm):
+        plan.run(X, offs, params, out)
+    torch.cuda.synchronize()
+    assert plan.query_status() == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        plan.run(X, offs, params, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    kept = int(out.out_offsets[batch])
+    launches = plan.last_launch_count
+    plan.close()
+    hbm_peak, _, peak_kind = measured_peaks()
+    path_bytes = total * d * 2 + kept * d * 2 + 12 * total
+    return {"workload": "sweep: %d images x 400 tokens x %d bf16 (the Large batch tiled %d times), dynamic ratio, T=100"
+                        % (batch, d, reps),
+            "ms_per_step": ms, "images_per_s": batch / (ms / 1e3), "steps": steps, "gpu_launches": launches * steps,
+            "path_roofline": {"bound": "hbm", "algorithmic_bytes": path_bytes, "achieved": path_bytes / (ms / 1e3) / 1e9,
+                              "peak": hbm_peak, "unit": "GB/s", "frac": path_bytes / (ms / 1e3) / 1e9 / hbm_peak,
+                              "peak_source": peak_kind}}
+
+
+def accuracy_against_oracle(w, out, threads: int) -> dict:
+    """Part of the cpu_baseline leg: the oracle's results for the timed batch against the device's (set 0 of the
+    rotation), as the figures the parity tests bound: largest feature error |y - y*| / max(|y*|, rms(y* row)), largest
+    regret of a chosen partner in log P below the oracle's column maximum, and whether every index output agrees."""
+    from oracle import oracle
+    p = w.params
+    op = oracle.Params(dynamic=bool(p["dynamic"]), r_fixed=p["r_fixed"], phi_lo=p["phi_lo"], phi_hi=p["phi_hi"],
+                       r_max=p["r_max"], z=p["z"], alpha=p["alpha"], eps=p["eps"], iters=int(p["iters"]))
+    refs = oracle.run_batch(w.X_f64(), w.offsets, op, w.rho, threads=threads, want_plan=True).images
+    Y = out.Y.cpu().to(torch.float64).numpy()
+    oo = out.out_offsets.cpu().numpy()
+    kept_idx, merged_idx = out.kept_idx.cpu().numpy(), out.merged_idx.cpu().numpy()
+    partner = out.merge_partner.cpu().numpy()
+    worst_feature, worst_regret, indices_equal = 0.0, 0.0, True
+    for i, ref in enumerate(refs):
+        o0, o1 = int(oo[i]), int(oo[i + 1])
+        seg = int(w.offsets[i]) - o0
+        indices_equal &= (o1 - o0 == ref.M and np.array_equal(kept_idx[o0:o1], ref.kept)
+                          and np.array_equal(merged_idx[seg:seg + ref.B], ref.prop))
+        if o1 - o0 != ref.M:
+            continue
+        rms = np.sqrt(np.mean(ref.Y * ref.Y, axis=1, keepdims=True))
+        denom = np.maximum(np.abs(ref.Y), rms)
+        worst_feature = max(worst_feature, float((np.abs(Y[o0:o1] - ref.Y) / np.where(denom > 0, denom, 1.0)).max()))
+        if ref.B:
+            logP = np.log(ref.Pbar[:-1, :-1])
+            gp = np.clip(partner[seg:seg + ref.B], 0, ref.M - 1)
+            worst_regret = max(worst_regret, float((logP.max(axis=0) - logP[gp, np.arange(ref.B)]).max()))
+    return {"images": len(refs), "indices_equal": bool(indices_equal), "max_feature_err": worst_feature,
+            "max_partner_regret": worst_regret}
+
+
+def self_launch(args) -> None:
+    """`python bench.py --gpus N` outside torch.distributed.run: start the N ranks (one per GPU) on this node."""
+    import socket
+    import tempfile
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    if "NCCL_DEBUG" not in env:      # the communicator's log (transports, NVLS) goes to a file, not into the JSON line
+        env["NCCL_DEBUG"] = "INFO"
+        env["NCCL_DEBUG_FILE"] = os.path.join(tempfile.gettempdir(), "rtprune_bench_nccl_%h_%p.log")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.stdout.flush()
+    os.execve(sys.executable, cmd, env)
 
 
 def main() -> None:
@@ -294,7 +392,12 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--repeats", type=int, default=10, help="how many times the K-step region is timed")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the one-shot summaries of the other workloads (density, large N, 1024 images)")
     args = ap.parse_args()
+    if args.gpus > 1 and args.impl == "ours" and args.step == "prune" and "WORLD_SIZE" not in os.environ:
+        self_launch(args)
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -359,17 +462,47 @@ def main() -> None:
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    # ---- timed region: K steps back to back, CUDA events on the launching stream ------------------
+    # ---- timed region: K steps back to back, CUDA events on the launching stream; R such regions --
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    repeats = max(1, args.repeats)
+    region_ms = []
+    for _ in range(repeats):
+        barrier()
+        torch.cuda._sleep(2000000)     # about 1 ms: the host is ahead of the device when the timed region starts
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+        region_ms.append(e0.elapsed_time(e1))
+    launches = plan.last_launch_count * args.steps
+
+    # ---- host time of a call: the library's own clock around rtprune_run, and the binding's on top ----
     barrier()
-    torch.cuda._sleep(2000000)     # about 1 ms: the host is ahead of the device when the timed region starts
+    host_ns = []
+    t_host = time.perf_counter()
+    for i in range(50):
+        step(i)
+        host_ns.append(plan.last_host_ns)
+    t_host = (time.perf_counter() - t_host) / 50
+    barrier()
+
+    # ---- the same K steps with every image running all T iterations (no exit at the fixed point) --
+    for s_ in dev_sets:
+        s_["params_all"] = binding.make_params(s_["rho"], **dict(fields, stop_at_fixed_point=0))
+    for i in range(3):
+        plan.run(dev_sets[i % ROTATE]["X"], dev_sets[i % ROTATE]["offs"], dev_sets[i % ROTATE]["params_all"],
+                 dev_sets[i % ROTATE]["out"])
+    barrier()
     e0.record(stream)
     for i in range(args.steps):
-        step(i)
+        s_ = dev_sets[i % ROTATE]
+        plan.run(s_["X"], s_["offs"], s_["params_all"], s_["out"])
     e1.record(stream)
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    launches = plan.last_launch_count * args.steps
+    ms_all_iters = e0.elapsed_time(e1) / args.steps
+    step(0)                            # set 0 holds the default run's outputs again (read below)
+    barrier()
 
     # ---- same steps again with per-kernel events (feeds the roofline of the dominant kernel) -----
     plan.profile_enable(True)
@@ -454,10 +587,12 @@ def main() -> None:
     d2h = total * d * esz + (batch + 1) * 4 + batch * 4 + 4 * total * 4 + batch * 8 * 4
 
     # ---- max over ranks ---------------------------------------------------------------------------
-    t = torch.tensor([ms_total, ms_e2e, ms_two], dtype=torch.float64, device=dev)
+    t = torch.tensor([ms_e2e, ms_two, ms_all_iters] + region_ms, dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, ms_two = float(t[0]), float(t[1]), float(t[2])
+    ms_e2e, ms_two, ms_all_iters = float(t[0]), float(t[1]), float(t[2])
+    region_ms = sorted(float(x) for x in t[3:])
+    ms_total = float(np.median(region_ms))           # `value` is the median region (max over ranks of each)
     ms_step = ms_total / args.steps
     images_s = world * batch / (ms_step / 1e3)
     e2e_images_s = world * batch / (ms_e2e / 1e3)
@@ -510,6 +645,13 @@ def main() -> None:
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "tokens_per_s": images_s * total / batch,
+            "repeats": {"n": repeats, "steps_each": args.steps, "value_is": "median",
+                        "ms_per_step": {"median": ms_step, "min": region_ms[0] / args.steps,
+                                        "max": region_ms[-1] / args.steps}},
+            "all_iterations": {"ms_per_step": ms_all_iters, "value": world * batch / (ms_all_iters / 1e3),
+                               "unit": "images/s", "note": "stop_at_fixed_point = 0: every image runs T = 100 iterations"},
+            "host_call": {"library_us": float(np.median(host_ns)) / 1e3, "with_binding_us": t_host * 1e6,
+                          "note": "host time of one rtprune_run call (5 launches), device busy"},
             "config": {"workload": WORKLOAD_DESC, "global_batch": world * batch,
                        "accumulate": "fp32", "sinkhorn": "T=100 with exit at the fixed point (no dual moves by more than 1 ulp)",
                        "mean_iterations_run": float(iters_run.mean()),
@@ -541,6 +683,19 @@ def main() -> None:
             line["cpu_baseline"] = {"value": batch / sec, "unit": "images/s", "cores": threads,
                                     "kind": "oracle",
                                     "sample": "all %d images of the Large batch, once" % batch}
+            line["accuracy"] = accuracy_against_oracle(w0, dev_sets[0]["out"], threads)
+        if world == 1 and not args.no_extras:
+            # one-shot records of the other workloads (each has a --step of its own for the full figures)
+            sub = argparse.Namespace(steps=20, warmup=3, no_cpu_baseline=True)
+            dl = density_line(sub)
+            ln = large_n_line(argparse.Namespace(steps=5, warmup=3, no_cpu_baseline=True))
+            line["also"] = {
+                "density": {"workload": dl["config"]["workload"], "ms_per_step": dl["ms_per_step"],
+                            "roofline_frac": dl["roofline"]["frac"]},
+                "largen": {k: {"workload": v["workload"], "ms_per_step": v["ms_per_step"],
+                               "path_roofline_frac": v["path_roofline"]["frac"]} for k, v in ln["shapes"].items()},
+                "sweep1024": sweep_line(w0, steps=10, warm=3),
+            }
         print(json.dumps(line), flush=True)
     plan.close()
     if world > 1:

@@ -54,9 +54,12 @@ typedef enum { RTPRUNE_BF16 = 0, RTPRUNE_FP32 = 1 } rtprune_dtype_t;
  * (u from v, then v from u, `iters` times, starting from u = v = 0 in the log domain) and give the
  * same plan up to rounding.
  *   LOG     u, v are the log-domain duals and every sweep is a max-shifted log-sum-exp, as printed.
- *   SCALING the duals are carried as e^u, e^v against the kernel K = exp((S-bar - c)/eps): every
- *           sweep is a matrix-vector product.  Used only when eps >= 0.25, where K cannot underflow.
- *   AUTO    SCALING when eps >= 0.25, else LOG.
+ *   SCALING the duals are carried as e^u, e^v against the kernel K = exp((S-bar - c)/eps), c = max(1, z):
+ *           every sweep is a matrix-vector product and nothing is subtracted, so the plan is as accurate in
+ *           fp32 as the log form's (more so at small eps).  Allowed while every factor stays inside fp32's
+ *           range: (2 max(1, z) - min(-1, z)) / eps <= 62, i.e. eps >= 0.05 at z = 0.2 and eps >= 0.25 for
+ *           any |z| <= 4; otherwise RTPRUNE_ERR_INVALID_ARG.
+ *   AUTO    SCALING when that condition holds, else LOG.
  *   EXACT   no iterations: the linear program of Eq. 2-6 itself is solved (the limit eps -> 0 of the
  *           entropic problem).  With the dustbins of Eq. 5 it is a maximum-weight partial matching in
  *           which pairing kept token i with pruned token j gains S_ij - z over leaving both in the
@@ -245,7 +248,9 @@ rtprune_status_t rtprune_query_status_static(rtprune_plan_t *plan, void *cuda_st
  * The same run, from and to HOST buffers (pinned memory recommended): copies X, offsets and rho to
  * the device arena, runs, and copies every output back, all asynchronously on the stream; the
  * caller synchronises the stream before reading.  `rho_host` may be NULL (params->rho is ignored
- * here).  Y_host receives total_tokens rows (only the first out_offsets[batch] are meaningful).
+ * here).  Y_host has room for total_tokens rows; the first out_offsets[batch] are written when the ratio is
+ * fixed (the kept counts are then known on the host before the launch), all total_tokens rows when it is
+ * dynamic (only the first out_offsets[batch] are meaningful).
  * `arena` is DEVICE memory, 256-byte aligned, of at least rtprune_host_arena_bytes bytes; it holds
  * the device copies and the workspace (initialised by this call).
  */
@@ -316,6 +321,10 @@ rtprune_status_t rtprune_test_expire_waits(rtprune_plan_t *plan, void *cuda_stre
 
 /* Kernels launched by the most recent run / select / run_host call on this plan. */
 int32_t rtprune_last_launch_count(const rtprune_plan_t *plan);
+
+/* Host time, in nanoseconds, that the most recent rtprune_run call on this plan spent launching (argument
+ * checks excluded; measurement aid). */
+int64_t rtprune_last_host_ns(const rtprune_plan_t *plan);
 
 /* cudaError_t value of the most recent failed CUDA call on this plan (0 if none). */
 int32_t rtprune_last_cuda_error(const rtprune_plan_t *plan);

@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(ctypes.c_char_p)]
     L.rtprune_last_launch_count.argtypes = [vp]
     L.rtprune_last_cuda_error.argtypes = [vp]
+    L.rtprune_last_host_ns.argtypes = [vp]
+    L.rtprune_last_host_ns.restype = ctypes.c_int64
     L.rtprune_destroy.argtypes = [vp]
     L.rtprune_destroy.restype = None
     L.rtprune_status_string.argtypes = [ctypes.c_int]
@@ -281,6 +283,10 @@ class Plan:
     @property
     def last_launch_count(self) -> int:
         return lib().rtprune_last_launch_count(self.handle)
+
+    @property
+    def last_host_ns(self) -> int:
+        return lib().rtprune_last_host_ns(self.handle)
 
     @property
     def last_cuda_error(self) -> int:

@@ -2,6 +2,7 @@
 // Every step of the path runs in the kernels included below; this file only marshals.
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -49,6 +50,19 @@ struct rtprune_plan_s {
                    // that share counters through the workspace wait for before they read them
     int fused_clusters;     // clusters of 2 CTAs of the fused stage-2 kernel the device runs at once (0: none)
     int exact_smem_bytes;   // dynamic shared memory of the exact-pairing kernel
+    // Tensor maps of the tensor-core kernels, kept from run to run: a map depends only on the buffers' addresses
+    // and extents, which a caller cycling over a few buffer sets repeats.
+    struct MapSet {
+        const void *X;
+        const void *ws;
+        int total, batch, pbuf_pitch;
+        bool valid;
+        CUtensorMap scX, scXp, mgX, mgXp, mgP;
+    };
+    static constexpr int kMapSets = 8;
+    MapSet maps[kMapSets];
+    int map_next;           // entry the next miss replaces
+    int64_t last_host_ns;   // host time the most recent rtprune_run call spent inside the library
 };
 
 // Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
@@ -207,6 +221,46 @@ bool make_tmap_bf16(rtprune_plan_t *plan, CUtensorMap *map, const void *base, ui
     return true;
 }
 
+// The scaling form carries e^u, e^v and K = exp((S-bar - c)/eps), c = max(1, z), in fp32.  With lo = min(-1, z)
+// the exponents of K span (c - lo)/eps, the duals stay within that span plus log N of their start, and V starts
+// at e^{c/eps}: every factor and product stays inside fp32's range while (2c - lo)/eps <= 62 (eps >= 0.05 at the
+// paper's z = 0.2; eps >= 0.25 for any |z| <= 4).
+bool scaling_in_range(const rtprune_params_t *p)
+{
+    const float c = std::fmax(1.f, p->z), lo = std::fmin(-1.f, p->z);
+    return (2.f * c - lo) / p->eps <= 62.f;
+}
+
+// The five tensor maps of a bf16 run over (X, workspace): from the plan's cache, or encoded into it.
+const rtprune_plan_s::MapSet *tensor_maps(rtprune_plan_t *plan, const void *X, char *ws, int total, int batch,
+                                          int pbuf_pitch)
+{
+    for (int i = 0; i < rtprune_plan_s::kMapSets; ++i) {
+        const rtprune_plan_s::MapSet &m = plan->maps[i];
+        if (m.valid && m.X == X && m.ws == ws && m.total == total && m.batch == batch && m.pbuf_pitch == pbuf_pitch)
+            return &m;
+    }
+    rtprune_plan_s::MapSet &m = plan->maps[plan->map_next];
+    plan->map_next = (plan->map_next + 1) % rtprune_plan_s::kMapSets;
+    m.valid = false;
+    const WsLayout &L = plan->ws;
+    const uint64_t d = (uint64_t)plan->d, rows_xp = (uint64_t)total + 64 * (uint64_t)batch;
+    if (!make_tmap_bf16(plan, &m.scX, X, (uint64_t)total, d, d * 2, kScBK, kScTileM) ||
+        !make_tmap_bf16(plan, &m.scXp, ws + L.xp, rows_xp, d, d * 2, kScBK, kScBBoxRows) ||
+        !make_tmap_bf16(plan, &m.mgX, X, (uint64_t)total, d, d * 2, 64, kMgBK) ||
+        !make_tmap_bf16(plan, &m.mgXp, ws + L.xp, rows_xp, d, d * 2, 64, kMgBK) ||
+        !make_tmap_bf16(plan, &m.mgP, ws + L.pbuf, (uint64_t)total, (uint64_t)pbuf_pitch, (uint64_t)pbuf_pitch * 2,
+                        kMgBK, kMgTileM))
+        return nullptr;
+    m.X = X;
+    m.ws = ws;
+    m.total = total;
+    m.batch = batch;
+    m.pbuf_pitch = pbuf_pitch;
+    m.valid = true;
+    return &m;
+}
+
 rtprune_status_t check_params(const rtprune_params_t *p)
 {
     if (!p) return RTPRUNE_ERR_INVALID_ARG;
@@ -225,8 +279,7 @@ rtprune_status_t check_params(const rtprune_params_t *p)
     if (p->criterion < RTPRUNE_CRITERION_L2NORM || p->criterion > RTPRUNE_CRITERION_ENTROPY)
         return RTPRUNE_ERR_INVALID_ARG;
     if (p->schedule < RTPRUNE_SCHEDULE_AUTO || p->schedule > RTPRUNE_SCHEDULE_FUSED) return RTPRUNE_ERR_INVALID_ARG;
-    const bool scaling_safe = p->eps >= 0.25f && std::fabs(p->z) <= 4.f;
-    if (p->form == RTPRUNE_SINKHORN_SCALING && !scaling_safe) return RTPRUNE_ERR_INVALID_ARG;
+    if (p->form == RTPRUNE_SINKHORN_SCALING && !scaling_in_range(p)) return RTPRUNE_ERR_INVALID_ARG;
     return RTPRUNE_OK;
 }
 
@@ -234,7 +287,7 @@ bool use_log_form(const rtprune_params_t *p)
 {
     if (p->form == RTPRUNE_SINKHORN_LOG) return true;
     if (p->form == RTPRUNE_SINKHORN_SCALING) return false;
-    return !(p->eps >= 0.25f && std::fabs(p->z) <= 4.f);
+    return !scaling_in_range(p);
 }
 
 // Largest B any image of at most max_tokens tokens can get under these parameters.
@@ -408,12 +461,9 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                 launched(plan, st, "gather");
             }
             // scores: one CTA per (128 consecutive tokens, image)
-            CUtensorMap tmapX, tmapXp;
-            if (!make_tmap_bf16(plan, &tmapX, X, (uint64_t)total, (uint64_t)plan->d,
-                                (uint64_t)plan->d * 2, kScBK, kScTileM) ||
-                !make_tmap_bf16(plan, &tmapXp, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
-                                (uint64_t)plan->d * 2, kScBK, kScBBoxRows))
-                return RTPRUNE_ERR_CUDA;
+            const rtprune_plan_s::MapSet *ms = tensor_maps(plan, X, ws, total, batch, pbuf_pitch);
+            if (!ms) return RTPRUNE_ERR_CUDA;
+            const CUtensorMap &tmapX = ms->scX, &tmapXp = ms->scXp;
             dim3 grid((maxN + kScTileM - 1) / kScTileM, batch);
             // The Sinkhorn kernel can start on an image as soon as that image's score tiles are in.  That
             // costs each scores CTA a release (its stores made visible before it counts itself), which
@@ -561,14 +611,9 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
 
     if constexpr (kTensor) {
         // every operand by tiled TMA: X rows (token tiles), the compact copy of pruned rows, the plan
-        CUtensorMap tmapXm, tmapXpm, tmapP;
-        if (!make_tmap_bf16(plan, &tmapXm, X, (uint64_t)total, (uint64_t)plan->d, (uint64_t)plan->d * 2,
-                            64, kMgBK) ||
-            !make_tmap_bf16(plan, &tmapXpm, ws + L.xp, (uint64_t)(total + 64 * batch), (uint64_t)plan->d,
-                            (uint64_t)plan->d * 2, 64, kMgBK) ||
-            !make_tmap_bf16(plan, &tmapP, pbuf, (uint64_t)total, (uint64_t)pbuf_pitch,
-                            (uint64_t)pbuf_pitch * 2, kMgBK, kMgTileM))
-            return RTPRUNE_ERR_CUDA;
+        const rtprune_plan_s::MapSet *ms = tensor_maps(plan, X, ws, total, batch, pbuf_pitch);
+        if (!ms) return RTPRUNE_ERR_CUDA;
+        const CUtensorMap &tmapXm = ms->mgX, &tmapXpm = ms->mgXp, &tmapP = ms->mgP;
         const int mtiles_m = (maxN + kMgTileM - 1) / kMgTileM;
         const int nct = (plan->d + kMgTileN - 1) / kMgTileN;
         const long long nunits = (long long)batch * mtiles_m * nct;
@@ -696,6 +741,9 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     p->ws = make_layout(d, dtype, max_batch, max_total_tokens, max_tokens_per_image);
     p->last_launches = 0;
     p->last_cuda_error = 0;
+    for (int i = 0; i < rtprune_plan_s::kMapSets; ++i) p->maps[i].valid = false;
+    p->map_next = 0;
+    p->last_host_ns = 0;
     p->profiling = false;
     p->ev_count = 0;
 
@@ -866,8 +914,11 @@ rtprune_status_t rtprune_run(rtprune_plan_t *plan, void *cuda_stream, const void
     if ((uintptr_t)Y & 15u) return RTPRUNE_ERR_INVALID_ARG;
     plan->last_launches = 0;
     DevOut o{Y, out_offsets, counts, kept_idx, merged_idx, merge_partner, merge_weight, stats};
-    return run_device(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
-                      (char *)workspace, o);
+    const auto t0 = std::chrono::steady_clock::now();
+    s = run_device(plan, (cudaStream_t)cuda_stream, X, offsets, batch, (int)total_tokens, params,
+                   (char *)workspace, o);
+    plan->last_host_ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    return s;
 }
 
 rtprune_status_t rtprune_select(rtprune_plan_t *plan, void *cuda_stream, const void *X,
@@ -1057,6 +1108,19 @@ rtprune_status_t rtprune_run_host(rtprune_plan_t *plan, void *cuda_stream, const
                    (int)total_tokens, &p,
                    base + a.ws, o);
     if (s != RTPRUNE_OK) return s;
+    // Rows of Y to bring back: with a fixed ratio every image's kept count is known here (the expression stage 1
+    // evaluates, in the same arithmetic); a dynamic ratio is decided on the device, so all rows are copied.
+    size_t y_rows = (size_t)total_tokens;
+    if (!p.dynamic) {
+        y_rows = 0;
+        const float r = std::fmax(p.r_fixed, 0.f);
+        for (int i = 0; i < batch; ++i) {
+            const int n = offsets_host[i + 1] - offsets_host[i];
+            int b = (int)std::floor(std::fmaf(r, (float)n, 0.5f));
+            b = std::max(0, std::min(b, n - 1));
+            y_rows += (size_t)(n - b);
+        }
+    }
     const size_t tot4 = (size_t)total_tokens * 4;
     if (!c.ok(cudaMemcpyAsync(out_offsets_host, o.out_offsets, ((size_t)batch + 1) * 4, cudaMemcpyDeviceToHost, st)) ||
         !c.ok(cudaMemcpyAsync(counts_host, o.counts, (size_t)batch * 4, cudaMemcpyDeviceToHost, st)) ||
@@ -1065,7 +1129,7 @@ rtprune_status_t rtprune_run_host(rtprune_plan_t *plan, void *cuda_stream, const
         !c.ok(cudaMemcpyAsync(merge_partner_host, o.merge_partner, tot4, cudaMemcpyDeviceToHost, st)) ||
         !c.ok(cudaMemcpyAsync(merge_weight_host, o.merge_weight, tot4, cudaMemcpyDeviceToHost, st)) ||
         !c.ok(cudaMemcpyAsync(stats_host, o.stats, (size_t)batch * kStats * 4, cudaMemcpyDeviceToHost, st)) ||
-        !c.ok(cudaMemcpyAsync(Y_host, o.Y, (size_t)total_tokens * row, cudaMemcpyDeviceToHost, st)))
+        (y_rows && !c.ok(cudaMemcpyAsync(Y_host, o.Y, y_rows * row, cudaMemcpyDeviceToHost, st))))
         return RTPRUNE_ERR_CUDA;
     return RTPRUNE_OK;
 }
@@ -1128,6 +1192,8 @@ rtprune_status_t rtprune_profile_read(rtprune_plan_t *plan, int32_t *n, float *m
 int32_t rtprune_last_launch_count(const rtprune_plan_t *plan) { return plan ? plan->last_launches : 0; }
 
 int32_t rtprune_last_cuda_error(const rtprune_plan_t *plan) { return plan ? plan->last_cuda_error : 0; }
+
+int64_t rtprune_last_host_ns(const rtprune_plan_t *plan) { return plan ? plan->last_host_ns : 0; }
 
 void rtprune_destroy(rtprune_plan_t *plan)
 {

@@ -172,7 +172,7 @@ __device__ inline void select_image(int img, int t_begin, int N, int d, int chun
             r = rp.r_fixed;
         }
         r = fmaxf(r, 0.f);
-        int B = (int)floorf(r * Nf + 0.5f);
+        int B = (int)floorf(fmaf(r, Nf, 0.5f));     // one rounding: the host evaluates the same expression
         B = max(0, min(B, N - 1));
         s_M = N - B;
         float *st = stats + (size_t)img * kStats;

@@ -66,7 +66,9 @@ def test_alpha_zero_is_plain_pruning(parity, binding):
 
 @pytest.mark.parametrize("over", [dict(form=1), dict(eps=0.1), dict(eps=0.3, z=0.6),
                                   dict(iters=0), dict(iters=1), dict(iters=7, stop_at_fixed_point=0),
-                                  dict(z=1.0), dict(z=0.0, alpha=0.5), dict(eps=0.05, iters=300)])
+                                  dict(z=1.0), dict(z=0.0, alpha=0.5), dict(eps=0.05, iters=300),
+                                  dict(eps=0.1, form=1), dict(eps=0.05, form=2), dict(eps=0.04), dict(eps=0.02, iters=200),
+                                  dict(eps=0.06, z=-1.0), dict(eps=0.25, z=4.0), dict(eps=0.25, z=-4.0)])
 def test_ot_parameter_ranges(parity, over):
     w = synth.ragged([64, 150, 31], params=dict(r_fixed=0.25))
     parity.check_workload(w, overrides=over)
@@ -201,7 +203,7 @@ def test_host_side_argument_errors(binding):
     offs = torch.tensor([0, 50, 100], dtype=torch.int32, device=dev)
     for bad in [dict(r_fixed=1.0), dict(r_fixed=-0.1), dict(eps=0.0), dict(iters=-1), dict(form=7),
                 dict(dynamic=1, phi_lo=0.5, phi_hi=0.5), dict(dynamic=1, r_max=0.0),
-                dict(form=2, eps=0.1), dict(tol=-1.0), dict(z=float("inf"))]:
+                dict(form=2, eps=0.04), dict(form=2, eps=0.1, z=4.0), dict(tol=-1.0), dict(z=float("inf"))]:
         with pytest.raises(binding.RtpruneError) as e:
             plan.run(X, offs, binding.make_params(**bad), out)
         assert e.value.status == 1, bad
