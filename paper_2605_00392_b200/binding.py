@@ -7,6 +7,7 @@ loaded, or no CUDA device is present, the calls raise.
 from __future__ import annotations
 
 import ctypes
+import numpy as np
 import os
 from dataclasses import dataclass
 from typing import Optional
@@ -331,3 +332,33 @@ def shard_images(batch: int, world_size: int, rank: int):
     base, extra = divmod(batch, world_size)
     lo = rank * base + min(rank, extra)
     return lo, lo + base + (1 if rank < extra else 0)
+
+
+def shard_slice(offsets, world_size: int, rank: int):
+    """What `rank` takes of a ragged batch: (lo, hi) its images, (row_lo, row_hi) its rows of X, and its own
+    offsets array, rebased so that it starts at 0 (what rtprune_run expects for the slice)."""
+    offsets = np.asarray(offsets, dtype=np.int64)
+    lo, hi = shard_images(len(offsets) - 1, world_size, rank)
+    row_lo, row_hi = int(offsets[lo]), int(offsets[hi])
+    return (lo, hi), (row_lo, row_hi), (offsets[lo:hi + 1] - row_lo).astype(np.int32)
+
+
+def packed_row_base(kept_rows_of_ranks, rank: int) -> int:
+    """Rows of the packed output that the lower ranks produce: what a rank adds to its local out_offsets to get
+    the positions its images have in the output of the whole batch."""
+    return int(sum(int(c) for c in list(kept_rows_of_ranks)[:rank]))
+
+
+def global_out_offsets(local_out_offsets: torch.Tensor, group=None) -> torch.Tensor:
+    """The rank's out_offsets in the numbering of the whole batch.  The only datum that crosses ranks is each
+    rank's number of kept rows (one all_gather of a scalar; nothing on the data path).  With no process group
+    initialised the local offsets are returned as they are."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return local_out_offsets.clone()
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    mine = local_out_offsets[-1:].to(torch.int64).clone()
+    every = [torch.zeros_like(mine) for _ in range(world)]
+    dist.all_gather(every, mine, group=group)
+    return local_out_offsets + packed_row_base([int(t.item()) for t in every], rank)
+

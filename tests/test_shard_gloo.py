@@ -2,7 +2,8 @@
 the batch and nothing is exchanged on the data path.  Two gloo ranks on CPU check the host-side
 logic: the slices cover the batch, and per-rank results (here from the CPU oracle, standing in for
 the GPU path) concatenate to the single-process result once the packed offsets are shifted by the
-counts of the lower ranks."""
+counts of the lower ranks.  The slicing (`binding.shard_slice`) and the shift (`binding.global_out_offsets`,
+one all_gather of a scalar) are the package's."""
 import os
 import socket
 
@@ -28,16 +29,13 @@ def _worker(rank: int, world: int, port: int, ret):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     from oracle import oracle
     w = synth.ragged([40, 17, 64, 9, 33], d=32, dtype=torch.float32, params=dict(r_fixed=0.25))
-    lo, hi = binding.shard_images(w.batch, world, rank)
-    res = oracle.run_batch(w.X_f64(), w.offsets, oracle.Params(r_fixed=0.25), w.rho,
-                           images=list(range(lo, hi)))
-    counts = torch.tensor([im.M for im in res.images], dtype=torch.int64)
-    # the only cross-rank datum: how many packed rows the lower ranks produce
-    mine = torch.tensor([int(counts.sum())])
-    allc = [torch.zeros(1, dtype=torch.int64) for _ in range(world)]
-    dist.all_gather(allc, mine)
-    base = int(sum(int(c) for c in allc[:rank]))
-    offs = base + np.concatenate([[0], np.cumsum(counts.numpy())])
+    # the rank's slice: its images, its rows of X, its own offsets starting at 0
+    (lo, hi), (row_lo, row_hi), local_offsets = binding.shard_slice(w.offsets, world, rank)
+    assert local_offsets[0] == 0 and local_offsets[-1] == row_hi - row_lo
+    res = oracle.run_batch(w.X_f64()[row_lo:row_hi], local_offsets, oracle.Params(r_fixed=0.25), w.rho[lo:hi])
+    local_out = torch.from_numpy(np.asarray(res.out_offsets, dtype=np.int64))
+    # the only cross-rank datum: how many packed rows the lower ranks produce (the package's helper gathers it)
+    offs = binding.global_out_offsets(local_out)
     ret[rank] = (lo, hi, offs.tolist(), [im.kept.tolist() for im in res.images])
     dist.barrier()
     dist.destroy_process_group()
