@@ -36,8 +36,8 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 f
 REFERENCE_SAMPLE = 64      # images per step of the --impl reference arm: the whole Large batch, as cpu_baseline
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
 # (kernels changed since their capture, or never captured, have no entry and report null)
-NCU_TRAFFIC_BYTES = {"stage1": 66109952, "gather": 10354432, "scores": 85585408,
-                     "sinkhorn_cluster": 4840960, "merge": 119804416, "density_tile": 318402048}
+NCU_TRAFFIC_BYTES = {"stage1": 65958912, "gather": 10358784, "scores": 85945344, "sinkhorn_reg": 4934656,
+                     "sinkhorn_cluster": 4840960, "merge": 118841088, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
@@ -393,6 +393,8 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--repeats", type=int, default=10, help="how many times the K-step region is timed")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "separate", "fused"],
+                    help="which kernels carry out stage 2 (rtprune_schedule_t); auto is the library's choice")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the one-shot summaries of the other workloads (density, large N, 1024 images)")
     args = ap.parse_args()
@@ -436,6 +438,8 @@ def main() -> None:
     batch, total, d = w0.batch, w0.total_tokens, w0.d
     plan = binding.Plan(d, torch.bfloat16, batch, total, w0.max_tokens, device=dev)
     fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
+    fields["schedule"] = {"auto": binding.SCHEDULE_AUTO, "separate": binding.SCHEDULE_SEPARATE,
+                          "fused": binding.SCHEDULE_FUSED}[args.schedule]
     dev_sets = []
     for w in sets:
         rho = torch.from_numpy(w.rho).to(dev)
@@ -658,6 +662,7 @@ def main() -> None:
                        "mean_retention": float(sumM) / total,
                        "l2": "inputs and outputs rotate over %d buffer sets (%.0f MB > L2)"
                              % (ROTATE, ROTATE * (x_bytes + y_bytes) / 1e6),
+                       "schedule": args.schedule,
                        "parallelism": "dp%d (independent images, no collective)" % world},
             "roofline": {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak,
                          "unit": unit, "frac": achieved / peak, "peak_source": peak_kind,
