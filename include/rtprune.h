@@ -150,10 +150,11 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan, int32_t d, rtprune_dtype_t 
 
 /*
  * Runs Algorithm 1 on a ragged batch, asynchronously on `cuda_stream`: no allocation, no host
- * synchronisation.  Inputs are not modified.  Each call gives its kernels a number that no other
- * call of the process has had (they hand images to one another through the workspace and tell this
- * run's entries from the last run's by it): do not capture the call into a CUDA graph that is
- * replayed; call it again instead.  One workspace serves one run at a time.
+ * synchronisation.  Inputs are not modified.  The kernels of a run hand images to one another through
+ * the workspace and tell this run's entries from the last run's by a run number that the first kernel
+ * counts up in the workspace itself, so the call may be captured into a CUDA graph and the graph
+ * replayed (the pointers and sizes of the capture are then fixed; keep per-kernel profiling off while
+ * capturing).  One workspace serves one run at a time.
  *
  *   X        DEVICE [total_tokens, d] row-major, dtype of the plan, 16-byte aligned
  *   offsets  DEVICE int32 [batch+1]: offsets[0] = 0, offsets[batch] = total_tokens, image i owns

@@ -18,8 +18,10 @@ struct WsHeader {
     uint32_t select_done;  // images whose selection has been published
     uint32_t n_ready;      // images whose transport plan has been published (entries of ready_list)
     uint32_t merge_next;   // next unit of the merge kernel when its CTAs draw units from a counter
-    int32_t run_tag;       // number of the run whose counters and lists below are in place (see wait_run_tag)
-    uint32_t pad[59];
+    int32_t run_tag;       // number of the run whose counters and lists below are in place
+    int32_t launch_seq;    // number of the run in flight on this workspace: stage 1 counts it up on the device, so a
+                           // run captured into a CUDA graph gets a new number at every replay
+    uint32_t pad[58];
 };
 
 // Byte offsets of the workspace regions; computed on the host from the plan's maxima.

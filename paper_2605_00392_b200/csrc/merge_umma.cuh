@@ -135,7 +135,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
                   int batch, int mtiles, const int32_t *__restrict__ counts,
                   const int32_t *__restrict__ out_offsets, const int32_t *__restrict__ kpos,
                   int max_tokens, int total, __nv_bfloat16 *__restrict__ Y, int32_t *__restrict__ kept_idx,
-                  WsHeader *__restrict__ hdr, const int32_t *ready_list, int run)
+                  WsHeader *__restrict__ hdr, const int32_t *ready_list)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -268,7 +268,7 @@ merge_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_consta
             };
             // with a list of finished images: not before the run's number is there (until then the list
             // and the unit counter are what the run before left)
-            bool ok = !ready_list || ptx::wait_equal_gpu(&hdr->run_tag, run);
+            bool ok = !ready_list || ptx::wait_equal_gpu(&hdr->run_tag, ptx::ld_acquire_gpu(&hdr->launch_seq));
             while (ok && !bars->abort_flag) {
                 // next unit: from the shared counter when the units follow the list of finished images
                 const int u = ready_list ? (int)atomicAdd(&hdr->merge_next, 1u)

@@ -46,8 +46,6 @@ struct rtprune_plan_s {
     const char *ev_name[RTPRUNE_PROFILE_MAX];
     int ev_count;  // kernels recorded by the most recent run
     int tall_c16_clusters;  // clusters of 16 CTAs of the wide-tile Sinkhorn kernel the device runs at once (0: none)
-    int run;       // number of the most recent run's second stage, unique in the process: what the kernels
-                   // that share counters through the workspace wait for before they read them
     int fused_clusters;     // clusters of 2 CTAs of the fused stage-2 kernel the device runs at once (0: none)
     int exact_smem_bytes;   // dynamic shared memory of the exact-pairing kernel
     // Tensor maps of the tensor-core kernels, kept from run to run: a map depends only on the buffers' addresses
@@ -71,8 +69,6 @@ struct rtprune_plan_s {
 static __device__ __align__(256) unsigned char g_static_scratch[RTPRUNE_STATIC_SCRATCH_BYTES];
 
 namespace {
-
-std::atomic<int> g_run_count{0};   // second-stage launches of the process, over all plans
 
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
@@ -181,7 +177,7 @@ __global__ void expire_waits_kernel(WsHeader *hdr, uint32_t poll_limit, int32_t 
     __shared__ uint64_t bar;
     if (threadIdx.x != 0) return;
     int expired = 0;
-    // run numbers count up from 1: -1 is not stored before a process has made 2^32 - 1 runs
+    // run numbers count up from 1 on every workspace: -1 is not stored before 2^32 - 1 runs on it
     if (!ptx::wait_equal_gpu(&hdr->run_tag, -1, poll_limit)) {
         atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
         ++expired;
@@ -426,7 +422,6 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
     __nv_bfloat16 *pbuf = kTensor ? (__nv_bfloat16 *)(ws + L.pbuf) : nullptr;
     const int pbuf_pitch = (std::max(maxB, 1) + 63) / 64 * 64;   // <= L.pbuf_pitch_max
     int32_t *ready_list = nullptr;   // images in the order their plans are finished, when the merge follows it
-    do plan->run = ++g_run_count; while (plan->run == 0);   // 0 is what a fresh workspace holds
     uint32_t *scores_done = nullptr; // per-image counts of finished score tiles, when the scores kernel keeps them
     const bool iterate = params->form != RTPRUNE_SINKHORN_EXACT;   // Sinkhorn iterations, else the exact pairing
 
@@ -456,7 +451,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                      (const __nv_bfloat16 *)X, offsets, o.counts, order, plan->d, maxN, total,
                                      (__nv_bfloat16 *)(ws + L.xp), (uint32_t *)(ws + L.sink_done),
                                      (int32_t *)(ws + L.ready_list), (WsHeader *)(ws + L.header), batch,
-                                     o.out_offsets, (uint32_t *)(ws + L.scores_done), plan->run)))
+                                     o.out_offsets, (uint32_t *)(ws + L.scores_done))))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "gather");
             }
@@ -513,7 +508,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                  (const int32_t *)order, (const float *)kmat, L.kmat_stride, maxN, total, op, pbuf,
                                  pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight, o.stats,
                                  (uint32_t *)(ws + L.sink_done), ready_list, (WsHeader *)(ws + L.header),
-                                 (const uint32_t *)scores_done, plan->run)))
+                                 (const uint32_t *)scores_done)))
                 return RTPRUNE_ERR_CUDA;
             launched(plan, st, "sinkhorn_reg");
             all_fast = true;
@@ -553,7 +548,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                      o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total, op,
                                      fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner, o.merge_weight,
                                      o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
-                                     (WsHeader *)(ws + L.header), sd, plan->run, 0)))
+                                     (WsHeader *)(ws + L.header), sd, 0)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "sinkhorn_cluster");
             } else {
@@ -563,7 +558,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
                                      offsets, o.counts, o.out_offsets, order, kmat, L.kmat_stride, maxN, total,
                                      op, fast_floats, pbuf, pbuf_pitch, o.merged_idx, o.merge_partner,
                                      o.merge_weight, o.stats, (uint32_t *)(ws + L.sink_done), ready_list,
-                                     (WsHeader *)(ws + L.header), sd, plan->run, 1)))
+                                     (WsHeader *)(ws + L.header), sd, 1)))
                     return RTPRUNE_ERR_CUDA;
                 launched(plan, st, "sinkhorn_wide");
             }
@@ -621,7 +616,7 @@ rtprune_status_t launch_stage2(rtprune_plan_t *plan, cudaStream_t st, const void
         if (!c.ok(launch_pdl(merge_umma_kernel, dim3((unsigned)grid), dim3(kMgThreads), kMgSmemBytes, st, 1u,
                              tmapXm, tmapXpm, tmapP, offsets, plan->d, batch, mtiles_m, o.counts, o.out_offsets,
                              (const int32_t *)(ws + L.kpos), maxN, total, (__nv_bfloat16 *)o.Y, o.kept_idx,
-                             (WsHeader *)(ws + L.header), (const int32_t *)ready_list, plan->run)))
+                             (WsHeader *)(ws + L.header), (const int32_t *)ready_list)))
             return RTPRUNE_ERR_CUDA;
     } else {
         const int dtiles = (plan->d + kSimtTile - 1) / kSimtTile;
@@ -808,7 +803,6 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
         return RTPRUNE_ERR_CUDA;
     }
     p->encode_tiled = nullptr;
-    p->run = 0;
     {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;

@@ -272,7 +272,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
                         int32_t *__restrict__ merged_idx, int32_t *__restrict__ merge_partner,
                         float *__restrict__ merge_weight, float *__restrict__ stats,
                         uint32_t *__restrict__ sink_done, int32_t *__restrict__ ready_list,
-                        WsHeader *__restrict__ hdr, const uint32_t *scores_done, int run, int takes_all)
+                        WsHeader *__restrict__ hdr, const uint32_t *scores_done, int takes_all)
 {
     extern __shared__ __align__(16) float sm[];
     const uint32_t C = ptx::cluster_nctarank(), rank = ptx::cluster_ctarank();
@@ -295,7 +295,7 @@ sinkhorn_cluster_kernel(const int32_t *__restrict__ offsets, const int32_t *__re
         if (tid == 0) {
             const uint32_t want = (uint32_t)((N + 127) / 128);     // the scores kernel's 128-token tiles
             // first the run's number: before it is there the counts are what the run before left
-            const bool tagged = ptx::wait_equal_gpu(&hdr->run_tag, run);
+            const bool tagged = ptx::wait_equal_gpu(&hdr->run_tag, ptx::ld_acquire_gpu(&hdr->launch_seq));
             bool ok = false;
             for (uint32_t i = 0; tagged && i < ptx::kSpinLimit && !ok; ++i) {
                 ok = (uint32_t)ptx::ld_acquire_gpu(reinterpret_cast<const int *>(scores_done + img)) >= want;

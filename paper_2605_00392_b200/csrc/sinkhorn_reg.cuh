@@ -80,7 +80,7 @@ sinkhorn_reg_kernel(const int32_t *__restrict__ offsets, const int32_t *__restri
                     __nv_bfloat16 *__restrict__ pbuf, int pbuf_pitch, int32_t *__restrict__ merged_idx,
                     int32_t *__restrict__ merge_partner, float *__restrict__ merge_weight, float *__restrict__ stats,
                     uint32_t *__restrict__ sink_done, int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr,
-                    const uint32_t *scores_done, int run)
+                    const uint32_t *scores_done)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -110,7 +110,7 @@ sinkhorn_reg_kernel(const int32_t *__restrict__ offsets, const int32_t *__restri
     if (scores_done) {
         if (tid == 0) {
             const uint32_t want = (uint32_t)((N + 127) / 128);     // the scores kernel's 128-token tiles
-            const bool tagged = ptx::wait_equal_gpu(&hdr->run_tag, run);
+            const bool tagged = ptx::wait_equal_gpu(&hdr->run_tag, ptx::ld_acquire_gpu(&hdr->launch_seq));
             bool ok = false;
             for (uint32_t i = 0; tagged && i < ptx::kSpinLimit && !ok; ++i) {
                 ok = (uint32_t)ptx::ld_acquire_gpu(reinterpret_cast<const int *>(scores_done + img)) >= want;

@@ -335,8 +335,24 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
     __shared__ uint64_t s_full[kS1MaxStages], s_empty[kS1MaxStages];
     const int img = blockIdx.y, chunk = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    ptx::grid_dep_launch();
-    ptx::grid_dep_wait();     // the workspace may still be in use by the run ahead in the stream
+    if (blockIdx.x == 0 && blockIdx.y == 0) {
+        // This CTA numbers the run: the kernels behind tell this run's counters and lists in the workspace from
+        // the last run's by the number.  It is counted up here, on the device, after the run ahead in the stream
+        // has ended and BEFORE this CTA lets the dependents go (they are scheduled once every CTA of this grid
+        // has done so), so every kernel of the run reads the new number, also in a replayed CUDA graph.
+        ptx::grid_dep_wait();
+        if (tid == 0) {
+            int seq = hdr->launch_seq + 1;
+            if (seq == 0) seq = 1;         // 0 is what a fresh workspace holds
+            ptx::st_release_gpu(&hdr->launch_seq, seq);
+            __threadfence();
+        }
+        __syncthreads();
+        ptx::grid_dep_launch();
+    } else {
+        ptx::grid_dep_launch();
+        ptx::grid_dep_wait();     // the workspace may still be in use by the run ahead in the stream
+    }
     int t_begin, n_img;
     const bool valid = image_range(offsets, img, max_tokens, total, t_begin, n_img);
     if (!valid) {
@@ -549,7 +565,7 @@ gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restri
                    const int32_t *__restrict__ counts, const int32_t *__restrict__ order, int d,
                    int max_tokens, int total, __nv_bfloat16 *__restrict__ xp, uint32_t *__restrict__ sink_done,
                    int32_t *__restrict__ ready_list, WsHeader *__restrict__ hdr, int batch,
-                   int32_t *__restrict__ out_offsets, uint32_t *__restrict__ scores_done, int run)
+                   int32_t *__restrict__ out_offsets, uint32_t *__restrict__ scores_done)
 {
     __shared__ int s_scan[32];
     const int img = blockIdx.y;
@@ -572,7 +588,7 @@ gather_prop_kernel(const __nv_bfloat16 *__restrict__ Xb, const int32_t *__restri
         }
         __threadfence();
         __syncthreads();
-        if (threadIdx.x == 0) ptx::st_release_gpu(&hdr->run_tag, run);
+        if (threadIdx.x == 0) ptx::st_release_gpu(&hdr->run_tag, ptx::ld_acquire_gpu(&hdr->launch_seq));
         scan_counts<128>(counts, out_offsets, batch, s_scan);
     }
     int t_begin, N;

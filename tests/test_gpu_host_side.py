@@ -106,3 +106,71 @@ def test_two_slices_concatenate_to_the_one_call_result(binding):
     for name in ("merged_idx", "merge_partner"):
         got = torch.cat([getattr(p[2], name)[:n] for p, n in zip(parts, pruned)])
         assert torch.equal(got, getattr(whole, name)[:sum(pruned)]), name
+
+
+@pytest.mark.parametrize("name,batch", [("large", 16), ("base", 32), ("ragged", 6)])
+def test_run_captured_into_a_cuda_graph_replays(binding, name, batch):
+    """rtprune_run captured once into a CUDA graph and replayed on changing inputs (copied into the captured
+    buffers) gives, replay after replay and without a synchronisation in between, what the direct call gives
+    bit for bit: the run number the kernels tell their hand-over lists by is counted on the device, not
+    baked into the launches."""
+    dev = torch.device("cuda", 0)
+    if name == "ragged":      # tiles of up to 578 pruned tokens: the cluster kernel's instance for wide tiles
+        sets = [synth.ragged([456, 1156, 700, 64, 300, 900], seed=40 + s, params=dict(r_fixed=0.5)) for s in range(3)]
+    else:
+        sets = [synth.make(name, seed_offset=s, batch=batch) for s in range(3)]
+    total = max(s.total_tokens for s in sets)
+    w0 = sets[0]
+    fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w0.params.items()}
+    plan = binding.Plan(w0.d, w0.X.dtype, batch, total, max(s.max_tokens for s in sets), device=dev)
+    keys = ("out_offsets", "counts", "kept_idx", "Y", "merged_idx", "merge_partner", "merge_weight")
+    try:
+        # direct calls: the reference of each input set
+        ref = []
+        for w in sets:
+            rho = torch.from_numpy(w.rho.copy()).to(dev)
+            out = binding.Outputs.allocate(total, batch, w.d, w.X.dtype, dev)
+            Xp = torch.zeros((total, w.d), dtype=w.X.dtype, device=dev)
+            Xp[:w.total_tokens] = w.X.to(dev)
+            plan.run(Xp[:w.total_tokens], torch.from_numpy(w.offsets.copy()).to(dev), binding.make_params(rho, **fields), out)
+            torch.cuda.synchronize()
+            ref.append(out)
+        # the captured buffers (the sets of a named batch have the same token counts, so one capture serves all)
+        assert all(s.total_tokens == w0.total_tokens and (s.offsets == w0.offsets).all() for s in sets)
+        Xc = torch.empty((w0.total_tokens, w0.d), dtype=w0.X.dtype, device=dev)
+        offs = torch.from_numpy(w0.offsets.copy()).to(dev)
+        rho_c = torch.empty(batch, dtype=torch.float32, device=dev)
+        params = binding.make_params(rho_c, **fields)
+        out_c = binding.Outputs.allocate(total, batch, w0.d, w0.X.dtype, dev)
+        Xc.copy_(sets[0].X.to(dev))
+        rho_c.copy_(torch.from_numpy(sets[0].rho.copy()).to(dev))
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            plan.run(Xc, offs, params, out_c)                # warm-up on the capture stream
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            plan.run(Xc, offs, params, out_c)
+        dev_in = [(s.X.to(dev), torch.from_numpy(s.rho.copy()).to(dev)) for s in sets]
+        keep = [binding.Outputs.allocate(total, batch, w0.d, w0.X.dtype, dev) for _ in range(9)]
+        for burst in range(4):
+            for j in range(9):                               # nine replays back to back, inputs changing
+                Xc.copy_(dev_in[j % 3][0])
+                rho_c.copy_(dev_in[j % 3][1])
+                graph.replay()
+                for k in keys:
+                    getattr(keep[j], k).copy_(getattr(out_c, k))
+            torch.cuda.synchronize()
+            for j in range(9):
+                rf = ref[j % 3]
+                n = int(rf.out_offsets[batch])
+                nb = w0.total_tokens - n
+                for k in keys:
+                    m = n if k in ("kept_idx", "Y") else (nb if k.startswith("merge") else None)
+                    a, b = getattr(keep[j], k), getattr(rf, k)
+                    assert torch.equal(a[:m] if m is not None else a, b[:m] if m is not None else b), (burst, j, k)
+        assert plan.query_status() == 0
+    finally:
+        plan.close()
