@@ -491,6 +491,35 @@ def main() -> None:
     t_host = (time.perf_counter() - t_host) / 50
     barrier()
 
+    # ---- the same K steps as replays of CUDA graphs (one captured step per buffer set) -------------
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(stream)
+    graphs = []
+    with torch.cuda.stream(side):
+        step(0)
+    stream.wait_stream(side)
+    torch.cuda.synchronize()
+    for k in range(ROTATE):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            step(k)
+        graphs.append(g)
+    for i in range(3):
+        graphs[i % ROTATE].replay()
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        graphs[i % ROTATE].replay()
+    e1.record(stream)
+    barrier()
+    ms_graph = e0.elapsed_time(e1) / args.steps
+    t_host_graph = time.perf_counter()
+    for i in range(50):
+        graphs[i % ROTATE].replay()
+    t_host_graph = (time.perf_counter() - t_host_graph) / 50
+    barrier()
+    assert plan.query_status() == 0
+
     # ---- the same K steps with every image running all T iterations (no exit at the fixed point) --
     for s_ in dev_sets:
         s_["params_all"] = binding.make_params(s_["rho"], **dict(fields, stop_at_fixed_point=0))
@@ -655,7 +684,11 @@ def main() -> None:
             "all_iterations": {"ms_per_step": ms_all_iters, "value": world * batch / (ms_all_iters / 1e3),
                                "unit": "images/s", "note": "stop_at_fixed_point = 0: every image runs T = 100 iterations"},
             "host_call": {"library_us": float(np.median(host_ns)) / 1e3, "with_binding_us": t_host * 1e6,
-                          "note": "host time of one rtprune_run call (5 launches), device busy"},
+                          "graph_replay_us": t_host_graph * 1e6,
+                          "note": "host time of one rtprune_run call (5 launches), device busy; of one replay of the "
+                                  "captured step"},
+            "graph_replay": {"ms_per_step": ms_graph, "value": world * batch / (ms_graph / 1e3), "unit": "images/s",
+                             "note": "the K steps as replays of CUDA graphs, one captured rtprune_run per buffer set"},
             "config": {"workload": WORKLOAD_DESC, "global_batch": world * batch,
                        "accumulate": "fp32", "sinkhorn": "T=100 with exit at the fixed point (no dual moves by more than 1 ulp)",
                        "mean_iterations_run": float(iters_run.mean()),

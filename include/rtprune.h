@@ -44,7 +44,8 @@ typedef enum {
     RTPRUNE_ERR_WORKSPACE = 3,   /* workspace / arena smaller than the plan requires         */
     RTPRUNE_ERR_CUDA = 4,        /* a CUDA runtime call failed; see rtprune_last_cuda_error  */
     RTPRUNE_ERR_NONFINITE = 5,   /* device saw a non-finite token norm (query_status only)   */
-    RTPRUNE_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (query_status only)   */
+    RTPRUNE_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (query_status only); the
+                                    outputs of that run are not to be used                    */
     RTPRUNE_ERR_BAD_OFFSETS = 7  /* device saw offsets outside the contract (query_status only) */
 } rtprune_status_t;
 
@@ -319,6 +320,16 @@ rtprune_status_t rtprune_density(void *cuda_stream, const uint8_t *images, int32
  */
 rtprune_status_t rtprune_test_expire_waits(rtprune_plan_t *plan, void *cuda_stream, void *workspace,
                                            size_t workspace_bytes, uint32_t poll_limit, int32_t *expired_out);
+
+/*
+ * Test aid for the give-up path of stage 1 (Eq. 1 / Eq. 8 pass): sets how many polls its waits on the copies
+ * that stream X into shared memory make before they give up (default 2^20; negative restores the default; 0
+ * makes every wait give up at once although its copy is on its way).  A CTA whose wait gave up reports
+ * RTPRUNE_DEV_TIMEOUT, waits once more, with the default limit, for the copies still in flight into its
+ * shared memory, and marks its image, which then passes through unpruned (M = N, Y rows = X rows): nothing
+ * faults, nothing is read that never arrived, and the next run with the default limit is clean.
+ */
+rtprune_status_t rtprune_test_set_poll_limit(rtprune_plan_t *plan, int64_t polls);
 
 /* Kernels launched by the most recent run / select / run_host call on this plan. */
 int32_t rtprune_last_launch_count(const rtprune_plan_t *plan);

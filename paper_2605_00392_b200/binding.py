@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
     L.rtprune_static_scratch_needed.argtypes = [vp, ctypes.POINTER(sz)]
     L.rtprune_query_status_static.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     L.rtprune_test_expire_waits.argtypes = [vp, vp, vp, sz, ctypes.c_uint32, vp]
+    L.rtprune_test_set_poll_limit.argtypes = [vp, ctypes.c_int64]
     L.rtprune_run_host.argtypes = [vp, vp, vp, vp, vp, i32, i64, pp, vp, sz,
                                    vp, vp, vp, vp, vp, vp, vp, vp]
     L.rtprune_host_arena_bytes.argtypes = [vp, ctypes.POINTER(sz)]
@@ -236,6 +237,10 @@ class Plan:
                                                self.workspace.numel(), int(poll_limit), expired.data_ptr()),
                "rtprune_test_expire_waits")
         return int(expired.item())
+
+    def set_poll_limit(self, polls: int) -> None:
+        """Test aid: polls after which stage 1's waits on its copies give up (negative: the default)."""
+        _check(lib().rtprune_test_set_poll_limit(self.handle, int(polls)), "rtprune_test_set_poll_limit")
 
     # -- rtprune_host_arena_bytes / rtprune_run_host
     def host_arena_bytes(self) -> int:

@@ -61,6 +61,7 @@ struct rtprune_plan_s {
     MapSet maps[kMapSets];
     int map_next;           // entry the next miss replaces
     int64_t last_host_ns;   // host time the most recent rtprune_run call spent inside the library
+    uint32_t poll_limit;    // polls after which stage 1's waits on its copies give up (ptx::kSpinLimit; tests lower it)
 };
 
 // Scratch of rtprune_select_static: lives in the library's device image, so every GPU that loads the
@@ -329,7 +330,7 @@ cudaError_t launch_stage1_kernel(const rtprune_plan_t *pl, cudaStream_t st, cons
             (float *)(ws + L.norms), (float *)(ws + (rp.criterion ? L.crit : L.norms)),          \
             (float *)(ws + L.spart), (uint32_t *)(ws + L.img_done),                              \
             (int32_t *)(ws + L.order), (int32_t *)(ws + L.kpos), counts, out_offsets, stats,     \
-            norms_out, order_out, (WsHeader *)(ws + L.header), scan_here);                       \
+            norms_out, order_out, (WsHeader *)(ws + L.header), scan_here, pl->poll_limit);       \
         if (e != cudaSuccess) return e;                                                          \
         break;                                                                                   \
     }
@@ -739,6 +740,7 @@ rtprune_status_t rtprune_plan(rtprune_plan_t **plan_out, int32_t d, rtprune_dtyp
     for (int i = 0; i < rtprune_plan_s::kMapSets; ++i) p->maps[i].valid = false;
     p->map_next = 0;
     p->last_host_ns = 0;
+    p->poll_limit = ptx::kSpinLimit;
     p->profiling = false;
     p->ev_count = 0;
 
@@ -1031,6 +1033,13 @@ rtprune_status_t rtprune_test_expire_waits(rtprune_plan_t *plan, void *cuda_stre
     expire_waits_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>((WsHeader *)((char *)workspace + plan->ws.header),
                                                                  poll_limit, expired_out);
     if (!c.ok(cudaGetLastError())) return RTPRUNE_ERR_CUDA;
+    return RTPRUNE_OK;
+}
+
+rtprune_status_t rtprune_test_set_poll_limit(rtprune_plan_t *plan, int64_t polls)
+{
+    if (!plan || polls > (int64_t)ptx::kSpinLimit) return RTPRUNE_ERR_INVALID_ARG;
+    plan->poll_limit = polls < 0 ? ptx::kSpinLimit : (uint32_t)polls;
     return RTPRUNE_OK;
 }
 

@@ -326,11 +326,11 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
               float *norms, float *critv, float *spart, uint32_t *img_done, int32_t *__restrict__ order,
               int32_t *__restrict__ kpos, int32_t *counts, int32_t *__restrict__ out_offsets,
               float *__restrict__ stats, float *__restrict__ norms_out, int32_t *__restrict__ order_out,
-              WsHeader *hdr, int scan_here)
+              WsHeader *hdr, int scan_here, uint32_t poll_limit)
 {
     constexpr int EPV = Elem<T>::kPerVec;
     extern __shared__ __align__(16) float s_dyn[];
-    __shared__ bool s_last;
+    __shared__ bool s_last, s_unseen;
     __shared__ int s_scan[32];
     __shared__ uint64_t s_full[kS1MaxStages], s_empty[kS1MaxStages];
     const int img = blockIdx.y, chunk = blockIdx.x;
@@ -387,6 +387,7 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
                 ptx::mbar_init(&s_full[s], 1);
                 ptx::mbar_init(&s_empty[s], kS1Warps);
             }
+            s_unseen = false;
             ptx::fence_mbar_init();
         }
         __syncthreads();
@@ -397,11 +398,15 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
             ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
             ptx::bulk_load(ring_u32 + s * stage_bytes, X + (size_t)r0 * d, bytes, &s_full[s]);
         };
+        int issued = 0;           // thread 0: copies issued so far
         if (tid == 0)
-            for (int it = 0; it < min(nstage, nit); ++it) issue(it);
+            for (int it = 0; it < min(nstage, nit); ++it, ++issued) issue(it);
         for (int it = 0; it < nit; ++it) {
             const int s = it % nstage;
-            if (!gave_up && !ptx::mbar_wait(&s_full[s], (it / nstage) & 1)) gave_up = true;
+            {   // a warp goes on or gives up as one (the row's reductions below are warp-wide)
+                const bool landed = !gave_up && ptx::mbar_wait(&s_full[s], (it / nstage) & 1, poll_limit);
+                if (!__all_sync(0xffffffffu, landed)) gave_up = true;
+            }
             const int t = t0 + it * kS1StageRows + warp;
             if (t < t1 && !gave_up) {
                 const uint4 *row = reinterpret_cast<const uint4 *>(
@@ -494,31 +499,50 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&s_empty[s]);
-            if (tid == 0 && it + nstage < nit) {     // refill the stage once all eight warps have left it
-                if (!gave_up && !ptx::mbar_wait(&s_empty[s], (it / nstage) & 1)) gave_up = true;
-                if (!gave_up) issue(it + nstage);
+            if (tid == 0 && it + nstage < nit && !gave_up) {     // refill the stage once all eight warps have left it
+                if (ptx::mbar_wait(&s_empty[s], (it / nstage) & 1, poll_limit)) {
+                    issue(it + nstage);
+                    ++issued;
+                } else {
+                    s_unseen = true;       // (read after the barrier below; only ever set)
+                }
             }
         }
-        if (gave_up && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
-        __syncthreads();      // the ring is free: it now holds the warps' partial sums
+        // Did any wait of this CTA run out?  Then rows of the chunk were never seen: report it, wait once more
+        // (with the full limit) for the copies still on their way into this CTA's shared memory, which is not
+        // touched until then, and mark the image: it will pass through unpruned.
+        const int unseen = __syncthreads_or((gave_up || (tid == 0 && s_unseen)) ? 1 : 0);
         if (bad && lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_NONFINITE);
-
-        // reduce the 8 warps' accumulators through shared memory
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int vi = lane + 32 * j;
-            if (vi < nvec) {
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) s_dyn[warp * d + vi * EPV + e] = acc[j * EPV + e];
+        if (unseen) {
+            if (tid == 0) {
+                atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                for (int s = 0; s < nstage; ++s) {
+                    // the last copy issued into stage s (an earlier one has completed: its barrier was waited for
+                    // before the stage was refilled)
+                    const int last = issued - 1 - ((issued - 1 - s) % nstage + nstage) % nstage;
+                    if (issued > s && last >= 0) (void)ptx::mbar_wait(&s_full[s], (last / nstage) & 1);
+                }
+                atomicOr(&img_done[img], 0x80000000u);
             }
-        }
-        __syncthreads();
-        float *out = spart + ((size_t)img * chunks + chunk) * d;
-        for (int c = tid; c < d; c += kS1Threads) {
-            float s = 0.f;
+            __syncthreads();
+        } else {
+            // the ring is free: it now holds the warps' partial sums, reduced through shared memory
 #pragma unroll
-            for (int w = 0; w < kS1Warps; ++w) s += s_dyn[w * d + c];
-            out[c] = s;
+            for (int j = 0; j < VPL; ++j) {
+                const int vi = lane + 32 * j;
+                if (vi < nvec) {
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) s_dyn[warp * d + vi * EPV + e] = acc[j * EPV + e];
+                }
+            }
+            __syncthreads();
+            float *out = spart + ((size_t)img * chunks + chunk) * d;
+            for (int c = tid; c < d; c += kS1Threads) {
+                float s = 0.f;
+#pragma unroll
+                for (int w = 0; w < kS1Warps; ++w) s += s_dyn[w * d + c];
+                out[c] = s;
+            }
         }
 
         // the CTA that completes the image selects its tokens
@@ -526,15 +550,33 @@ stage1_kernel(const T *__restrict__ X, const int32_t *__restrict__ offsets, int 
         __syncthreads();
         if (tid == 0) {
             const uint32_t nchunk = (uint32_t)((n_img + chunk_tokens - 1) / chunk_tokens);
-            const uint32_t prev = atomicAdd(&img_done[img], 1u);
-            s_last = (prev == nchunk - 1u);
+            const uint32_t prev = atomicAdd(&img_done[img], 1u);      // (after this CTA's own mark, if it set one)
+            s_last = ((prev & 0x7fffffffu) == nchunk - 1u);
+            s_unseen = (prev & 0x80000000u) != 0u;
             if (s_last) img_done[img] = 0;       // ready for the next run
         }
         __syncthreads();
         if (!s_last) return;
         __threadfence();
-        select_image(img, t_begin, n_img, d, chunks, chunk_tokens, rp, rho, critv, spart, order, kpos, counts, stats,
-                     norms_out, order_out, reinterpret_cast<uint32_t *>(s_dyn));
+        if (s_unseen) {
+            // some chunk of the image was never read (reported above): the image passes through unpruned
+            for (int k = tid; k < n_img; k += kS1Threads) {
+                order[t_begin + k] = k;
+                kpos[t_begin + k] = k;
+                if (order_out) order_out[t_begin + k] = k;
+                if (norms_out) norms_out[t_begin + k] = 0.f;
+            }
+            if (tid == 0) {
+                counts[img] = n_img;
+                float *st = stats + (size_t)img * kStats;
+                for (int q = 0; q < kStats; ++q) st[q] = 0.f;
+                st[3] = (float)n_img;
+            }
+            __syncthreads();
+        } else {
+            select_image(img, t_begin, n_img, d, chunks, chunk_tokens, rp, rho, critv, spart, order, kpos, counts, stats,
+                         norms_out, order_out, reinterpret_cast<uint32_t *>(s_dyn));
+        }
     }
 
     // the CTA that completes the batch: out_offsets = exclusive prefix sum of counts (unless a kernel

@@ -174,3 +174,32 @@ def test_run_captured_into_a_cuda_graph_replays(binding, name, batch):
         assert plan.query_status() == 0
     finally:
         plan.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_stage1_gives_up_cleanly_and_recovers(parity, binding, dtype):
+    """Stage 1's waits on the copies that stream X are given no polls at all: every CTA gives up although its
+    copies are on their way, reports it, waits them out with the default limit, and its image passes through
+    unpruned.  Nothing faults; with the default limit restored the same plan passes the parity check."""
+    dev = torch.device("cuda", 0)
+    w = synth.ragged([400, 37, 256, 1, 180, 129], dtype=dtype, params=dict(r_fixed=0.3))
+    plan = binding.Plan(w.d, w.X.dtype, w.batch, w.total_tokens, w.max_tokens, device=dev)
+    try:
+        plan.set_poll_limit(0)
+        fields = {k: (int(v) if k in ("dynamic", "iters") else float(v)) for k, v in w.params.items()}
+        out = binding.Outputs.allocate(w.total_tokens, w.batch, w.d, w.X.dtype, dev)
+        X = w.X.to(dev)
+        for _ in range(2):
+            plan.run(X, torch.from_numpy(w.offsets.copy()).to(dev), binding.make_params(None, **fields), out)
+            assert plan.query_status() == binding.DEV_TIMEOUT
+            lens = torch.from_numpy((w.offsets[1:] - w.offsets[:-1]).copy())
+            assert torch.equal(out.counts.cpu()[:w.batch], lens.to(torch.int32))
+            assert torch.equal(out.out_offsets.cpu(), torch.from_numpy(w.offsets.copy()))
+            assert torch.equal(out.Y, X)                       # every image passed through, bit for bit
+        with pytest.raises(binding.RtpruneError):
+            plan.set_poll_limit(1 << 30)
+        plan.set_poll_limit(-1)
+        rep = parity.check_workload(w, plan=plan)
+        assert rep["mean_retention"] < 0.75
+    finally:
+        plan.close()
