@@ -132,6 +132,39 @@ def document_image(rng: np.random.Generator, n: int, d: int, text_density: float
     return rows[rng.permutation(n)]
 
 
+def paired_image(rng: np.random.Generator, n: int, d: int, r: float, noise: float = 0.3):
+    """An image whose pruning has a known answer: n - B "anchor" tokens with Gaussian directions and lengths in
+    [1.5, 3] sqrt(d), and B = round(r n) "echo" tokens, each a noisy copy of a random anchor's direction with a
+    length in [0.3, 0.8] sqrt(d).  Ranked by norm at ratio r the anchors are kept and the echoes pruned, and every
+    echo's look-alike among the kept tokens is its anchor by a wide margin (cosine about 0.95 against about 0).
+    Returns (rows, echo_of): echo_of[k] = token index of the anchor that token k echoes, -1 for an anchor."""
+    n_echo = int(np.floor(r * n + 0.5))
+    n_anchor = n - n_echo
+    anchors = _unit(rng.standard_normal((n_anchor, d)))
+    src = rng.integers(0, n_anchor, size=n_echo)
+    echoes = _unit(anchors[src] + noise * _unit(rng.standard_normal((n_echo, d))))
+    rows = np.concatenate([anchors * (np.sqrt(d) * rng.uniform(1.5, 3.0, n_anchor))[:, None],
+                           echoes * (np.sqrt(d) * rng.uniform(0.3, 0.8, n_echo))[:, None]])
+    perm = rng.permutation(n)                  # new position p holds old row perm[p]
+    where = np.empty(n, dtype=np.int64)
+    where[perm] = np.arange(n)                 # old row -> new position
+    echo_of = np.full(n, -1, dtype=np.int64)
+    echo_of[where[n_anchor + np.arange(n_echo)]] = where[src]
+    return rows[perm], echo_of
+
+
+def paired(lengths: List[int], r: float, *, seed: int = 3, d: int = D_MODEL,
+           dtype: torch.dtype = torch.bfloat16):
+    """A batch of paired_image images at fixed ratio r.  Returns (workload, [echo_of per image])."""
+    ims, truth = [], []
+    for i, n in enumerate(lengths):
+        rows, echo_of = paired_image(_rng(SEED_BASE + 0x200 + seed, i), n, d, r)
+        ims.append(_space_norms(rows, dtype))
+        truth.append(echo_of)
+    w = _assemble("paired", ims, np.zeros(len(lengths)), dict(dynamic=0, r_fixed=float(r), phi_lo=0.0, phi_hi=1.0, r_max=1.0))
+    return w, truth
+
+
 # Ratio parameters of the dynamic configurations.  phi_hi was chosen so that the Large batch keeps
 # about 84 % of its tokens on average, the retention the paper reports for its dynamic mode.
 DYNAMIC_PARAMS = dict(dynamic=1, r_fixed=0.0, phi_lo=0.0, phi_hi=0.737, r_max=0.5)

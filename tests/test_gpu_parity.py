@@ -69,3 +69,23 @@ def test_sweep_fp32(parity):
 def test_host_buffer_path_matches(parity):
     w = synth.make("base", batch=4)
     parity.check_workload(w, host_path=True)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_known_pairing_is_recovered(parity, dtype):
+    """Images whose answer is known by construction (pruned tokens are low-norm noisy copies of kept tokens):
+    every pair is decisive, so the whole pair output is held to bit-exactness against the oracle, and the
+    partners are the anchors the generator used."""
+    d = 1280 if dtype == torch.bfloat16 else 256
+    w, truth = synth.paired([400] * 6 + [64, 100, 37, 256], 0.25, d=d, dtype=dtype)
+    rep = parity.check_workload(w)
+    assert rep["bit_exact_pair_share"] == 1.0 and rep["pairs"] == 6 * 100 + 16 + 25 + 9 + 64
+    g = parity.run_gpu(w).out
+    for i, echo_of in enumerate(truth):
+        o0 = int(g.out_offsets[i])
+        seg = int(w.offsets[i]) - o0
+        nb = int((echo_of >= 0).sum())
+        kept = g.kept_idx[o0:o0 + int(g.counts[i])].numpy()
+        pruned = g.merged_idx[seg:seg + nb].numpy()
+        partner = g.merge_partner[seg:seg + nb].numpy()
+        np.testing.assert_array_equal(kept[partner], echo_of[pruned])

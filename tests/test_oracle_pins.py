@@ -522,3 +522,26 @@ def test_criterion_ties_keep_lower_index(oracle):
     if order.index(2) < M:
         res = oracle.run_image(T, oracle.Params(r_fixed=(10 - M) / 10.0, criterion=1))
         assert 2 in res.kept and 7 in res.prop
+
+
+def test_echo_tokens_pair_with_their_anchors(oracle):
+    """An input whose answer is known without running anything: the pruned tokens are noisy low-norm copies of
+    kept tokens.  The oracle must keep exactly the anchors and pair every echo with its own anchor, by a wide
+    margin (the generator's construction, not the oracle's arithmetic, is the reference here)."""
+    import torch
+    from paper_2605_00392_b200 import synth
+    w, truth = synth.paired([64, 100, 37], 0.25, d=256, dtype=torch.float32)
+    res = oracle.run_batch(w.X_f64(), w.offsets, oracle.Params(r_fixed=0.25), w.rho, want_plan=True)
+    for i, (im, echo_of) in enumerate(zip(res.images, truth)):
+        anchors = np.nonzero(echo_of < 0)[0]
+        echoes = np.nonzero(echo_of >= 0)[0]
+        np.testing.assert_array_equal(im.kept, anchors)
+        np.testing.assert_array_equal(im.prop, echoes)
+        np.testing.assert_array_equal(im.kept[im.partner], echo_of[echoes])
+        assert im.gap.min() > 0.5            # log P of the anchor stands clear of every other kept token
+        # the exact pairing is one to one: every anchor with echoes is paired with one of its own echoes (a
+        # second echo of the same anchor may find a stranger worth more than the dustbin score, or nobody)
+        ex = oracle.run_image_exact(w.image_f64(i), oracle.Params(r_fixed=0.25))
+        taken = {int(ex.kept[p]): int(ex.prop[j]) for j, p in enumerate(ex.partner) if p >= 0}
+        for a in np.unique(echo_of[echoes]):
+            assert int(a) in taken and echo_of[taken[int(a)]] == a, (i, int(a))
