@@ -339,11 +339,30 @@ def shard_images(batch: int, world_size: int, rank: int):
     return lo, lo + base + (1 if rank < extra else 0)
 
 
-def shard_slice(offsets, world_size: int, rank: int):
-    """What `rank` takes of a ragged batch: (lo, hi) its images, (row_lo, row_hi) its rows of X, and its own
-    offsets array, rebased so that it starts at 0 (what rtprune_run expects for the slice)."""
+def shard_images_by_tokens(offsets, world_size: int, rank: int):
+    """Contiguous range of images [lo, hi) for `rank` on a ragged batch, balanced by work instead of by count:
+    the cut before rank k is the image boundary nearest to k / world_size of the batch's cost, an image of N
+    tokens costing N (the streaming passes) + N^2 / 1600 (scores, Sinkhorn and merge grow with M B <= N^2 / 4;
+    the weight makes the two terms equal at 400 tokens).  Every rank computes the same cuts from the offsets."""
     offsets = np.asarray(offsets, dtype=np.int64)
-    lo, hi = shard_images(len(offsets) - 1, world_size, rank)
+    n = np.diff(offsets).astype(np.float64)
+    cost = np.concatenate([[0.0], np.cumsum(n + n * n / 1600.0)])
+    total = cost[-1]
+    cuts = [0]
+    for k in range(1, world_size):
+        j = int(np.argmin(np.abs(cost - total * k / world_size)))
+        cuts.append(max(j, cuts[-1]))
+    cuts.append(len(n))
+    return cuts[rank], cuts[rank + 1]
+
+
+def shard_slice(offsets, world_size: int, rank: int, *, by_tokens: bool = False):
+    """What `rank` takes of a ragged batch: (lo, hi) its images, (row_lo, row_hi) its rows of X, and its own
+    offsets array, rebased so that it starts at 0 (what rtprune_run expects for the slice).  by_tokens: balance
+    the ranks by work (shard_images_by_tokens) instead of by image count."""
+    offsets = np.asarray(offsets, dtype=np.int64)
+    lo, hi = (shard_images_by_tokens(offsets, world_size, rank) if by_tokens
+              else shard_images(len(offsets) - 1, world_size, rank))
     row_lo, row_hi = int(offsets[lo]), int(offsets[hi])
     return (lo, hi), (row_lo, row_hi), (offsets[lo:hi + 1] - row_lo).astype(np.int32)
 

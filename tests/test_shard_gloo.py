@@ -55,3 +55,26 @@ def test_two_ranks_partition_the_batch():
     assert got_offs == ref.out_offsets.tolist()
     kept = ret[0][3] + ret[1][3]
     assert kept == [im.kept.tolist() for im in ref.images]
+
+
+def test_shards_balanced_by_work_cover_the_batch():
+    """Ragged batches: cuts by work are contiguous, cover every image once, and even out the token counts far
+    better than cuts by image count when the long images sit together."""
+    lens = [1156] * 6 + [456] * 26
+    offsets = np.concatenate([[0], np.cumsum(lens)])
+    for world in (1, 2, 3, 4, 8):
+        ranges = [binding.shard_images_by_tokens(offsets, world, r) for r in range(world)]
+        assert ranges[0][0] == 0 and ranges[-1][1] == len(lens)
+        assert all(ranges[r][1] == ranges[r + 1][0] for r in range(world - 1))
+        assert all(lo <= hi for lo, hi in ranges)
+    by_work = [binding.shard_slice(offsets, 2, r, by_tokens=True)[1] for r in range(2)]
+    by_count = [binding.shard_slice(offsets, 2, r)[1] for r in range(2)]
+    n = np.asarray(lens, dtype=np.float64)
+    cost = np.concatenate([[0.0], np.cumsum(n + n * n / 1600.0)])          # the balancing rule's cost, by image
+    image_of_row = {int(o): i for i, o in enumerate(offsets)}
+    work = lambda rows: [cost[image_of_row[hi]] - cost[image_of_row[lo]] for lo, hi in rows]
+    assert max(work(by_work)) / min(work(by_work)) < 1.1
+    assert max(work(by_count)) / min(work(by_count)) > 1.8
+    # equal images: the same cuts as by count
+    eq = np.arange(0, 401 * 16, 400)
+    assert [binding.shard_images_by_tokens(eq, 4, r) for r in range(4)] == [binding.shard_images(16, 4, r) for r in range(4)]
