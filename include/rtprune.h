@@ -67,7 +67,7 @@ typedef enum { RTPRUNE_BF16 = 0, RTPRUNE_FP32 = 1 } rtprune_dtype_t;
  *           dustbins; the solver finds a vertex by shortest augmenting paths in fp32.  The plan then
  *           holds ones at the pairs and zeros elsewhere, Eq. 7 adds alpha T_p^j to the partner of every
  *           paired token, merge_partner is the kept position or -1 (unpaired: the token is dropped),
- *           merge_weight is 1 or 0, stats[5] counts path-search steps and stats[6] is 0.  eps, iters,
+ *           merge_weight is 1 or 0, stats[5] counts path-search steps and stats[6] the rows paired before any search.  eps, iters,
  *           stop_at_fixed_point, tol and schedule are ignored.  Where several matchings reach the optimum
  *           any one of them may be returned. */
 typedef enum {

@@ -2,13 +2,17 @@
 // program is a maximum-weight partial matching between kept and pruned tokens whose pair (i, j) gains
 // S_ij - z over leaving both in the dustbins; a vertex of the polytope pairs every token at most once.  The
 // kernel finds it by shortest augmenting paths on the gains clipped at zero (a pair of clipped gain 0 is left
-// unpaired afterwards), the smaller side being the one whose tokens are inserted one by one.  Every step of a
-// path search is one pass of the CTA over the other side: relax the reduced costs against the token reached
-// last, take the block-wide minimum (ties to the lower index), shift the potentials by it.
+// unpaired afterwards).  The smaller side are the rows.  Start: every row's price is its best gain and rows
+// whose best column nobody smaller wants take it (those edges are tight).  Then, for every row still free, a
+// shortest-path search over the columns in the reduced costs: every thread owns fixed columns and keeps their
+// distances, predecessors and marks to itself, so a step is one relaxation of the own columns against the
+// column reached last plus one block-wide minimum (ties to the lower index): ONE block barrier per step.  The
+// prices move once per search, after the free column is found (columns in the tree by their distance to it,
+// rows from the tightness of their own edge), never during it.
 //
 // Outputs: the pairs (merge_partner = kept position or -1, merge_weight = 1 or 0) and the plan of zeros and
 // ones that Eq. 7 then uses as it uses Sinkhorn's: alpha at the paired cells of the bf16 plan buffer, or 1 in
-// place in the fp32 workspace tile.  stats[5] = path-search steps taken, stats[6] = 0.
+// place in the fp32 workspace tile.  stats[5] = search steps taken, stats[6] = rows the start assigned.
 #pragma once
 #include "common.cuh"
 #include "sinkhorn.cuh"
@@ -18,9 +22,9 @@ namespace rtp {
 constexpr int kExThreads = 512;
 constexpr int kExWarps = kExThreads / 32;
 
-// Words of shared memory the search arrays take for images of at most max_tokens tokens: two potentials, the
-// reduced-cost minima, the assignment, the path links and the visited marks, each of at most max_tokens + 1.
-__host__ __device__ inline size_t exact_array_words(int max_tokens) { return 6 * (size_t)(max_tokens + 8); }
+// Words of shared memory the search arrays take for images of at most max_tokens tokens: two prices, the
+// distances, the assignment by column and by row, the path links and the marks, each of at most max_tokens + 1.
+__host__ __device__ inline size_t exact_array_words(int max_tokens) { return 7 * (size_t)(max_tokens + 8); }
 
 // Dynamic shared memory of a launch: the arrays, then as many clipped gains as the limit leaves (an image
 // whose n x m gains fit keeps them there, the others read the workspace tile at every step).
@@ -43,6 +47,7 @@ exact_pairing_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     extern __shared__ __align__(16) float sm[];
     __shared__ float s_val[2][kExWarps];
     __shared__ int s_idx[2][kExWarps];
+    __shared__ int s_started;
     const int img = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int t_begin, N;
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
@@ -51,124 +56,186 @@ exact_pairing_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     const bool transposed = B > M;            // rows of the assignment = the smaller side
     const int n = transposed ? M : B, m = transposed ? B : M;
     const int cap = max_tokens + 8;
-    float *u = sm;                            // [n]   potentials of the rows
-    float *v = u + cap;                       // [m+1] potentials of the columns (column m: the root of a search)
-    float *minv = v + cap;                    // [m+1] smallest reduced cost seen for each column in this search
-    int *asg = reinterpret_cast<int *>(minv + cap);   // [m+1] row assigned to each column, -1: free
-    int *way = asg + cap;                     // [m+1] column the search reached this column from
-    int *used = way + cap;                    // [m+1] column is in the search tree
-    float *gains = reinterpret_cast<float *>(used + cap);
+    float *u = sm;                            // [n]   prices of the rows
+    float *v = u + cap;                       // [m]   prices of the columns
+    float *dist = v + cap;                    // [m]   shortest reduced-cost distance found for each column in this search
+    int *asg = reinterpret_cast<int *>(dist + cap);   // [m] row assigned to each column, -1: free
+    int *way = asg + cap;                     // [m]   column the search reached this column from (m: the free row itself)
+    int *used = way + cap;                    // [m]   column is in the search tree
+    int *rowcol = used + cap;                 // [n]   column assigned to each row, -1: free
+    float *gains = reinterpret_cast<float *>(rowcol + cap);
     const bool staged = (long long)n * m <= (long long)smem_words - (long long)exact_array_words(max_tokens);
 
     float *Sg = kmat + kmat_offset(kmat_stride, t_begin, img);
     const int ldS = score_pitch(B);
     const float z = prm.z;
-    // clipped gain of row r, column c
-    auto gain_of = [&](int r, int c) -> float {
+    // clipped gain of row r, column c (the cost of the assignment problem is its negative)
+    auto gain_global = [&](int r, int c) -> float {
         const float s = transposed ? __ldcg(Sg + (size_t)r * ldS + c) : __ldcg(Sg + (size_t)c * ldS + r);
         return fmaxf(s - z, 0.f);
     };
     if (staged)
         for (int idx = tid; idx < n * m; idx += kExThreads) {
             const int r = idx / m, c = idx - r * m;
-            gains[idx] = gain_of(r, c);
+            gains[idx] = gain_global(r, c);
         }
-    for (int r = tid; r < n; r += kExThreads) u[r] = 0.f;
-    for (int c = tid; c <= m; c += kExThreads) {
+    for (int c = tid; c < m; c += kExThreads) {
         v[c] = 0.f;
-        asg[c] = -1;
+        asg[c] = 0x7fffffff;
     }
+    if (tid == 0) s_started = 0;
+    __syncthreads();
+    auto gain_of = [&](int r, int c) -> float { return staged ? gains[(size_t)r * m + c] : gain_global(r, c); };
+
+    // ---- start: u_r = -(best gain of row r); the row takes its best column (lowest index on ties) if no
+    // lower row wants the same one.  Reduced costs -g - u_r - 0 are >= 0, and 0 on the edges taken.
+    for (int r = warp; r < n; r += kExWarps) {
+        float best = -1.f;
+        int bc = 0x7fffffff;
+        for (int c = lane; c < m; c += 32) {
+            const float g = gain_of(r, c);
+            if (g > best) {
+                best = g;
+                bc = c;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oc = __shfl_xor_sync(0xffffffffu, bc, o);
+            if (ob > best || (ob == best && oc < bc)) {
+                best = ob;
+                bc = oc;
+            }
+        }
+        if (lane == 0) {
+            u[r] = -best;
+            way[r] = bc;                      // (scratch until the searches begin)
+            if (bc < m) atomicMin(&asg[bc], r);
+        }
+    }
+    __syncthreads();
+    int started = 0;
+    for (int r = tid; r < n; r += kExThreads) {
+        const int bc = way[r];
+        const bool won = bc < m && asg[bc] == r;
+        rowcol[r] = won ? bc : -1;
+        started += won ? 1 : 0;
+    }
+    if (started) atomicAdd(&s_started, started);
+    __syncthreads();
+    for (int c = tid; c < m; c += kExThreads)
+        if (asg[c] == 0x7fffffff) asg[c] = -1;
     __syncthreads();
 
     int steps = 0;
     bool broken = false;                      // a non-finite score: no minimum exists (uniform over the CTA)
     for (int row = 0; row < n && !broken; ++row) {
+        if (rowcol[row] >= 0) continue;       // (uniform: every thread reads the same word)
+        // distances from the free row; every thread touches only its own columns until the path is flipped
+        const float urow = u[row];
+        float lbest = INFINITY;
+        int lj = 0x7fffffff;
         for (int c = tid; c < m; c += kExThreads) {
-            minv[c] = INFINITY;
+            const float dc = -gain_of(row, c) - urow - v[c];
+            dist[c] = dc;
+            way[c] = m;
             used[c] = 0;
-        }
-        if (tid == 0) {
-            used[m] = 1;
-            asg[m] = row;
-        }
-        __syncthreads();
-        int j0 = m;
-        // each step puts one more column into the tree and there are m of them: the search ends within m steps
-        for (int guard = 0; guard <= m; ++guard) {
-            const int i0 = asg[j0];
-            const float ui0 = u[i0];
-            const float *grow = gains + (size_t)i0 * m;
-            float best = INFINITY;
-            int bj = 0x7fffffff;
-            for (int c = tid; c < m; c += kExThreads) {
-                if (used[c]) continue;
-                const float g = staged ? grow[c] : gain_of(i0, c);
-                const float cur = -g - ui0 - v[c];
-                float mv = minv[c];
-                if (cur < mv) {
-                    mv = cur;
-                    minv[c] = cur;
-                    way[c] = j0;
-                }
-                if (mv < best) {              // c ascends within a thread: strict < keeps the lower column
-                    best = mv;
-                    bj = c;
-                }
+            if (dc < lbest) {                 // c ascends within a thread: strict < keeps the lower column
+                lbest = dc;
+                lj = c;
             }
+        }
+        int sink = -1;
+        float mu = 0.f;
+        // each step puts one more column into the tree and at most `row` of them are taken: the search ends
+        for (int guard = 0; guard <= m; ++guard) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-                const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-                if (ob < best || (ob == best && oj < bj)) {
-                    best = ob;
-                    bj = oj;
+                const float ob = __shfl_xor_sync(0xffffffffu, lbest, o);
+                const int oj = __shfl_xor_sync(0xffffffffu, lj, o);
+                if (ob < lbest || (ob == lbest && oj < lj)) {
+                    lbest = ob;
+                    lj = oj;
                 }
             }
             const int par = steps & 1;
             if (lane == 0) {
-                s_val[par][warp] = best;
-                s_idx[par][warp] = bj;
+                s_val[par][warp] = lbest;
+                s_idx[par][warp] = lj;
             }
             __syncthreads();
-            float delta = s_val[par][0];
-            int j1 = s_idx[par][0];
+            float dmin = s_val[par][0];
+            int jstar = s_idx[par][0];
 #pragma unroll
             for (int w = 1; w < kExWarps; ++w) {
                 const float ob = s_val[par][w];
                 const int oj = s_idx[par][w];
-                if (ob < delta || (ob == delta && oj < j1)) {
-                    delta = ob;
-                    j1 = oj;
+                if (ob < dmin || (ob == dmin && oj < jstar)) {
+                    dmin = ob;
+                    jstar = oj;
                 }
             }
             ++steps;
-            if (j1 == 0x7fffffff) {
+            if (jstar == 0x7fffffff) {
                 broken = true;
                 break;
             }
-            for (int c = tid; c <= m; c += kExThreads) {
-                if (used[c]) {
-                    u[asg[c]] += delta;       // the rows of the tree's columns are distinct
-                    v[c] -= delta;
-                } else {
-                    minv[c] -= delta;
-                }
-                if (c == j1) used[c] = 1;
+            mu = dmin;
+            const int i2 = asg[jstar];
+            if (i2 < 0) {                     // a free column: the shortest path ends here
+                sink = jstar;
+                break;
             }
-            __syncthreads();
-            j0 = j1;
-            if (asg[j0] < 0) break;           // a free column: the path is complete
+            // relax the own columns against the row of the column just reached, and find the next minimum
+            const float base = dmin - u[i2];
+            lbest = INFINITY;
+            lj = 0x7fffffff;
+            for (int c = tid; c < m; c += kExThreads) {
+                if (c == jstar) used[c] = 1;
+                if (used[c]) continue;
+                const float nd = base - gain_of(i2, c) - v[c];
+                float dc = dist[c];
+                if (nd < dc) {
+                    dc = nd;
+                    dist[c] = nd;
+                    way[c] = jstar;
+                }
+                if (dc < lbest) {
+                    lbest = dc;
+                    lj = c;
+                }
+            }
         }
-        if (broken) break;
+        if (broken || sink < 0) {
+            broken = true;
+            break;
+        }
+        // prices of the tree's columns (own columns), while one thread flips the path back to the free row
+        for (int c = tid; c < m; c += kExThreads)
+            if (used[c]) v[c] += dist[c] - mu;
         if (tid == 0) {
-            // flip the path back to the root
-            int c = j0;
-            for (int guard = 0; guard <= m && c != m; ++guard) {
+            int c = sink;
+            for (int guard = 0; guard <= m; ++guard) {
                 const int prev = way[c];
-                asg[c] = asg[prev];
+                if (prev >= m) {
+                    asg[c] = row;
+                    rowcol[row] = c;
+                    break;
+                }
+                const int r = asg[prev];
+                asg[c] = r;
+                rowcol[r] = c;
                 c = prev;
             }
         }
+        __syncthreads();
+        // prices of the tree's rows from the tightness of the edges they now hold
+        for (int c = tid; c < m; c += kExThreads)
+            if (used[c] || c == sink) {
+                const int r = asg[c];
+                u[r] = -gain_of(r, c) - v[c];
+            }
         __syncthreads();
     }
 
@@ -198,7 +265,7 @@ exact_pairing_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     }
     if (tid == 0) {
         stats[(size_t)img * kStats + 5] = (float)steps;
-        stats[(size_t)img * kStats + 6] = 0.f;
+        stats[(size_t)img * kStats + 6] = (float)s_started;
     }
 
     if (pbuf) {
