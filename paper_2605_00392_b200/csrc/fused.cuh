@@ -205,7 +205,7 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
 #pragma unroll
         for (int q = 0; q < NQ; ++q) colacc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         float usum = 0.f;
-        // this round's arrival on the local barrier: the other CTA's ldk column sums and its sum of U
+        // this exchange's arrival on the local barrier: the other CTA's ldk column sums and its sum of U
         if (tid == 0) ptx::mbar_arrive_expect_tx(&sh->xbar[par], (uint32_t)(ldk + 1) * 4u);
 
 #pragma unroll
