@@ -23,8 +23,13 @@ constexpr int kExThreads = 512;
 constexpr int kExWarps = kExThreads / 32;
 
 // Words of shared memory the search arrays take for images of at most max_tokens tokens: two prices, the
-// distances, the assignment by column and by row, the path links and the marks, each of at most max_tokens + 1.
-__host__ __device__ inline size_t exact_array_words(int max_tokens) { return 7 * (size_t)(max_tokens + 8); }
+// distances, the assignment by column and by row and the path links (a word per token each) and the marks (a
+// byte per token): 205 KB at the plan's limit of 8192 tokens.
+__host__ __device__ inline size_t exact_array_words(int max_tokens)
+{
+    const size_t cap = (size_t)(max_tokens + 8);
+    return 6 * cap + (cap + 3) / 4;       // six arrays of words and the marks, a byte each
+}
 
 // Dynamic shared memory of a launch: the arrays, then as many clipped gains as the limit leaves (an image
 // whose n x m gains fit keeps them there, the others read the workspace tile at every step).
@@ -61,9 +66,9 @@ exact_pairing_kernel(const int32_t *__restrict__ offsets, const int32_t *__restr
     float *dist = v + cap;                    // [m]   shortest reduced-cost distance found for each column in this search
     int *asg = reinterpret_cast<int *>(dist + cap);   // [m] row assigned to each column, -1: free
     int *way = asg + cap;                     // [m]   column the search reached this column from (m: the free row itself)
-    int *used = way + cap;                    // [m]   column is in the search tree
-    int *rowcol = used + cap;                 // [n]   column assigned to each row, -1: free
-    float *gains = reinterpret_cast<float *>(rowcol + cap);
+    int *rowcol = way + cap;                  // [n]   column assigned to each row, -1: free
+    unsigned char *used = reinterpret_cast<unsigned char *>(rowcol + cap);   // [m] column is in the search tree
+    float *gains = reinterpret_cast<float *>(sm + exact_array_words(max_tokens));
     const bool staged = (long long)n * m <= (long long)smem_words - (long long)exact_array_words(max_tokens);
 
     float *Sg = kmat + kmat_offset(kmat_stride, t_begin, img);

@@ -97,26 +97,34 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
 
     if (warp == 4) {
         // ---------------- producer: tiled TMA for both operands -----------------------------------
-        if (lane == 0) {
-            ptx::prefetch_tensormap(&tmapX);
-            ptx::prefetch_tensormap(&tmapXp);
+        // The whole warp walks the k-blocks in step; the loads of a k-block are issued by as many lanes at
+        // once (lane 0: the A tile, lanes 1-4: the B boxes) instead of by one thread one after the other.
+        {
+            if (lane == 0) {
+                ptx::prefetch_tensormap(&tmapX);
+                ptx::prefetch_tensormap(&tmapXp);
+            }
             uint32_t it = 0;
-            for (int bt = 0; bt < nbt && !bars->abort_flag; ++bt) {
+            bool alive = true;
+            for (int bt = 0; bt < nbt && alive && !bars->abort_flag; ++bt) {
                 const int nbox = (min(kScBNMax, B - bt * kScBNMax) + kScBBoxRows - 1) / kScBBoxRows;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % kScStages;
-                    if (it >= (uint32_t)kScStages &&
-                        !ptx::mbar_wait(&bars->empty[s], ((it / kScStages) - 1) & 1)) {
+                    const bool ok = it < (uint32_t)kScStages || ptx::mbar_wait(&bars->empty[s], ((it / kScStages) - 1) & 1);
+                    if (!__all_sync(0xffffffffu, ok)) {
                         bars->abort_flag = 1;
-                        atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                        if (lane == 0) atomicOr(&hdr->status, RTPRUNE_DEV_TIMEOUT);
+                        alive = false;
                         break;
                     }
                     const uint32_t a_dst = smem_base + s * stage_bytes;
-                    ptx::mbar_arrive_expect_tx(&bars->full[s], kScABytes + nbox * kScBBoxBytes);
-                    ptx::tma_load_2d(a_dst, &tmapX, &bars->full[s], kb * kScBK, t_begin + mt * kScTileM);
-                    for (int b = 0; b < nbox; ++b)
-                        ptx::tma_load_2d(a_dst + kScABytes + b * kScBBoxBytes, &tmapXp, &bars->full[s],
-                                         kb * kScBK, xp0 + bt * kScBNMax + b * kScBBoxRows);
+                    if (lane == 0) ptx::mbar_arrive_expect_tx(&bars->full[s], kScABytes + nbox * kScBBoxBytes);
+                    __syncwarp();
+                    if (lane == 0)
+                        ptx::tma_load_2d(a_dst, &tmapX, &bars->full[s], kb * kScBK, t_begin + mt * kScTileM);
+                    else if (lane <= nbox)
+                        ptx::tma_load_2d(a_dst + kScABytes + (lane - 1) * kScBBoxBytes, &tmapXp, &bars->full[s],
+                                         kb * kScBK, xp0 + bt * kScBNMax + (lane - 1) * kScBBoxRows);
                 }
             }
         }
