@@ -174,13 +174,11 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
     constexpr int ldk = LR * CPL;
     constexpr int RPS = 32 / LR;
     constexpr int NQ = CPL / 4;
-    constexpr int kVWarps = ldk / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LR, slot = lane / LR;
     const float Bf = (float)B, Mf = (float)M;
 
     for (int j = tid; j <= ldk; j += kFuThreads) sh->vs[j] = (j < B || j == ldk) ? v_init : 0.f;
-    if (tid < kFuWarps) sh->vsum[tid] = (tid == 0) ? Bf * v_init : 0.f;
 #pragma unroll
     for (int s = 0; s < NS; ++s) U[s] = 0.f;
     __syncthreads();
@@ -195,9 +193,13 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
         float4 V[NQ];
 #pragma unroll
         for (int q = 0; q < NQ; ++q) V[q] = *reinterpret_cast<const float4 *>(sh->vs + 4 * (q * LR + sub));
+        // sum of V over the real columns (V is 0 past column B): the LR lanes of a row hold all columns between
+        // them, so the sum comes out of the same shuffles as a row sum, in every thread and in the same order
         float sumV = 0.f;
 #pragma unroll
-        for (int w = 0; w < kVWarps; ++w) sumV += sh->vsum[w];
+        for (int q = 0; q < NQ; ++q) sumV += (V[q].x + V[q].y) + (V[q].z + V[q].w);
+#pragma unroll
+        for (int o = 1; o < LR; o <<= 1) sumV += __shfl_xor_sync(0xffffffffu, sumV, o);
         const float Vd = sh->vs[ldk];
         const float Ud = Bf * rcp_fast(kappa * (sumV + Vd));
         const float kVd = kappa * Vd;
@@ -212,14 +214,16 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
         for (int s = 0; s < NS; ++s) {
             const int i = (s * kFuWarps + warp) * RPS + slot;
             const bool valid = i < Ml;
-            float sd = 0.f;
+            // four partial sums: a chain of NQ dependent multiply-adds instead of 4 NQ
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
-                sd = fmaf(k[s][q].x, V[q].x, sd);
-                sd = fmaf(k[s][q].y, V[q].y, sd);
-                sd = fmaf(k[s][q].z, V[q].z, sd);
-                sd = fmaf(k[s][q].w, V[q].w, sd);
+                s0 = fmaf(k[s][q].x, V[q].x, s0);
+                s1 = fmaf(k[s][q].y, V[q].y, s1);
+                s2 = fmaf(k[s][q].z, V[q].z, s2);
+                s3 = fmaf(k[s][q].w, V[q].w, s3);
             }
+            float sd = (s0 + s1) + (s2 + s3);
 #pragma unroll
             for (int o = 1; o < LR; o <<= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
             const float u = valid ? rcp_fast(sd + kVd) : 0.f;
@@ -257,9 +261,15 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
         int cont = 0;
         float move = 0.f;
         if (tid < ldk) {
-            float cs = 0.f;
+            float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
 #pragma unroll
-            for (int w = 0; w < kFuWarps; ++w) cs += part[w * ldk + tid];
+            for (int w = 0; w < kFuWarps; w += 4) {
+                c0 += part[(w + 0) * ldk + tid];
+                c1 += part[(w + 1) * ldk + tid];
+                c2 += part[(w + 2) * ldk + tid];
+                c3 += part[(w + 3) * ldk + tid];
+            }
+            const float cs = (c0 + c1) + (c2 + c3);
             st_async_peer(xpart_peer + (par * (uint32_t)kFuMaxB + (uint32_t)tid) * 4u, __float_as_uint(cs), xbar_peer + par * 8u);
             if (!ptx::mbar_wait(&sh->xbar[par], phase)) {
                 sh->abort_flag = 1;
@@ -273,8 +283,6 @@ __device__ inline FuIterState fused_iterate(const float4 (&k)[NS][CPL / 4], floa
                 cont = p.tol > 0.f ? (move > p.tol) : (p.stop_fp ? ulp_far(nv, ov) : 1);
                 sh->vs[tid] = nv;
             }
-            const float wv = warp_sum(nv);        // warps 0 .. ldk/32-1 lie entirely inside tid < ldk
-            if (lane == 0) sh->vsum[warp] = wv;
         }
         if (tid == kFuThreads - 1) {              // the dustbin column
             float su = 0.f;
