@@ -19,7 +19,8 @@
 // needs: the kernel is launched as a programmatic dependent and merges the first images on whatever
 // SMs are free while the last ones still iterate.  Warp roles (224 threads):
 // warps 0-3 epilogue (TMEM -> registers -> bf16 -> own row of a padded staging tile -> one bulk store
-// per kept row); warp 4 lane 0 issues the TMA loads; warp 5 owns TMEM and lane 0 issues the UMMAs;
+// per kept row); warp 4 issues the TMA loads (the loads of a k-block from several lanes at once); warp 5 owns TMEM and
+// its lane 0 issues the UMMAs;
 // warp 6 lane 0 is the scheduler: it draws the units, looks up what the other roles need to know about
 // them (a chain of dependent loads from L2) a few units ahead and hands them over through a small queue
 // in shared memory.

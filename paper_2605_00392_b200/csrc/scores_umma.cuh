@@ -10,7 +10,8 @@
 //     box are zeros or another image's tokens; they only reach accumulator columns nobody reads.
 //   * D: 128 TMEM lanes x BN columns (BN = B rounded up to 16, at most 256 per pass).
 // Warp roles (192 threads): warps 0-3 run the epilogue (TMEM -> registers -> divide by the two norms
-// -> global); warp 4 lane 0 issues every TMA load; warp 5 owns TMEM and lane 0 issues the UMMAs.  A
+// -> global); warp 4 issues the TMA loads (those of a k-block from several lanes at once); warp 5 owns TMEM and its
+// lane 0 issues the UMMAs.  A
 // ring of shared-memory stages (as many as fit in 96 KB: 4 for B <= 64, 2 for B = 256) is handed over
 // with mbarriers.  The ring is sized so that two CTAs share an SM: a whole Large batch is one wave.
 #pragma once
