@@ -143,11 +143,12 @@ sinkhorn_reg_kernel(const int32_t *__restrict__ offsets, const int32_t *__restri
     {
         const int qpr = ldk >> 2;                     // float4 per row of K
         const int total_q = Ml * qpr;
-        for (int q0 = tid; q0 < total_q; q0 += kFuThreads * 4) {
-            float4 s4[4];
-            int ii[4], jj[4];
+        constexpr int kInFlight = 8;                  // 16-byte loads a thread has in flight per trip to L2
+        for (int q0 = tid; q0 < total_q; q0 += kFuThreads * kInFlight) {
+            float4 s4[kInFlight];
+            int ii[kInFlight], jj[kInFlight];
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
+            for (int a = 0; a < kInFlight; ++a) {
                 const int q = q0 + a * kFuThreads;
                 ii[a] = q / qpr;
                 jj[a] = (q - ii[a] * qpr) << 2;
@@ -156,7 +157,7 @@ sinkhorn_reg_kernel(const int32_t *__restrict__ offsets, const int32_t *__restri
                             : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
+            for (int a = 0; a < kInFlight; ++a) {
                 const int q = q0 + a * kFuThreads;
                 if (q < total_q) {
                     float4 kv;
