@@ -121,11 +121,16 @@ __device__ inline MergeUnit merge_unit(int u, int mtiles, int nct, const int32_t
             return q;
         }
     }
-    // L2 loads: with a ready list this kernel may have started before the selection wrote these
-    q.valid = image_range(offsets, q.img, max_tokens, total, q.t_begin, q.N) && q.mt * kMgTileM < q.N;
-    q.M = q.valid ? __ldcg(counts + q.img) : 0;
+    // L2 loads (with a ready list this kernel may have started before the selection wrote these), all issued
+    // before the first use: one trip, not one per value (img is a valid image number either way)
+    const int o_lo = __ldcg(offsets + q.img), o_hi = __ldcg(offsets + q.img + 1);
+    const int m_img = __ldcg(counts + q.img), out0 = __ldcg(out_offsets + q.img);
+    q.t_begin = o_lo;
+    q.N = o_hi - o_lo;
+    q.valid = q.N >= 1 && q.N <= max_tokens && o_lo >= 0 && o_hi <= total && q.mt * kMgTileM < q.N;
+    q.M = q.valid ? m_img : 0;
     q.B = q.N - q.M;
-    q.out0 = q.valid ? __ldcg(out_offsets + q.img) : 0;
+    q.out0 = q.valid ? out0 : 0;
     q.nident = (q.N - q.mt * kMgTileM <= kMgBK) ? 1 : kMgIdentKb;
     return q;
 }

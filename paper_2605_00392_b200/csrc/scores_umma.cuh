@@ -53,8 +53,9 @@ scores_umma_kernel(const __grid_constant__ CUtensorMap tmapX, const __grid_const
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();     // counts, order, norms and the compact copy come from the kernels ahead
     int t_begin, N;
+    const int M = __ldcg(counts + img);       // (issued with the two offsets: one trip to L2)
     if (!image_range(offsets, img, max_tokens, total, t_begin, N)) return;
-    const int M = counts[img], B = N - M;
+    const int B = N - M;
     if (mt * kScTileM >= N) return;
     // With scores_done, every tile of a valid image is counted when it is complete (at once if nothing is
     // pruned): the Sinkhorn kernel, launched as a programmatic dependent, starts on an image when its

@@ -120,13 +120,12 @@ sinkhorn_reg_kernel(const int32_t *__restrict__ offsets, const int32_t *__restri
         }
         __syncthreads();
     }
-    const int M = __ldcg(counts + img), B = N - M;
+    const int M = __ldcg(counts + img), out0 = __ldcg(out_offsets + img), B = N - M;     // (one trip to L2 for both)
     if (B == 0) {
         sinkhorn_publish(img, 2u, sink_done, ready_list, hdr);
         if (scores_done) ptx::grid_dep_wait();
         return;
     }
-    const int out0 = __ldcg(out_offsets + img);
     const int half = (M + 1) >> 1;
     const int row_lo = min(M, (int)rank * half);
     const int Ml = min(M, row_lo + half) - row_lo;
