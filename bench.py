@@ -36,8 +36,8 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 f
 REFERENCE_SAMPLE = 64      # images per step of the --impl reference arm: the whole Large batch, as cpu_baseline
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
 # (kernels changed since their capture, or never captured, have no entry and report null)
-NCU_TRAFFIC_BYTES = {"stage1": 66115840, "gather": 10358272, "scores": 85689600, "sinkhorn_reg": 4936704,
-                     "sinkhorn_cluster": 4840960, "merge": 118464768, "density_tile": 318402048}
+NCU_TRAFFIC_BYTES = {"stage1": 66078208, "gather": 10355200, "scores": 87525888, "sinkhorn_reg": 4935424,
+                     "sinkhorn_cluster": 4840960, "merge": 118104064, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
