@@ -37,7 +37,7 @@ REFERENCE_SAMPLE = 64      # images per step of the --impl reference arm: the wh
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture (profiles/), by kernel
 # (kernels changed since their capture, or never captured, have no entry and report null)
 NCU_TRAFFIC_BYTES = {"stage1": 66078208, "gather": 10355200, "scores": 87525888, "sinkhorn_reg": 4935424,
-                     "sinkhorn_cluster": 4840960, "merge": 118104064, "density_tile": 318402048}
+                     "merge": 118104064, "density_tile": 318402048}
 
 
 def cpu_threads() -> int:
